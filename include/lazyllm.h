@@ -1,0 +1,249 @@
+/*
+ * lazyllm.h — C ABI of the token-pruned prefill / decode library (sm_100a).
+ *
+ * The library runs the prefill forward of a Llama-style decoder with dynamic token
+ * pruning, and the decode step that can revive pruned tokens from an Aux Cache.
+ * Paper passages are cited per entry point ("Section 3.2", "Eq. 1", ...).
+ *
+ * Conventions that hold for every call
+ *   - Return value: 0 (LAZY_OK) or a negative lazy_status. Nothing throws, aborts or traps.
+ *   - "device" pointers are CUDA global-memory addresses of the current device; "host"
+ *     pointers are ordinary process memory.  The library never allocates or frees device
+ *     memory: weights, ids, logits and one workspace blob are caller-owned and must outlive
+ *     the context.  The context itself (host metadata only) is owned by the library.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work
+ *     is enqueued asynchronously unless stated otherwise; device-side problems (a bounded
+ *     wait that ran out, an index out of range) are written to a per-device status word and
+ *     surface through lazy_sync_status() / lazy_device_status().
+ *   - Matrices are row-major [out_features, in_features] (K-contiguous), activations are
+ *     row-major [rows, features].  dtype LAZY_BF16: bf16 storage, fp32 accumulation;
+ *     LAZY_F32: fp32 storage and arithmetic (CUDA cores; small models only).
+ *   - A context holds ONE generation state; it is not thread-safe.
+ */
+#ifndef LAZYLLM_H_
+#define LAZYLLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LAZY_OK = 0,
+  LAZY_E_BADARG = -1,      /* null pointer, non-positive size, unsupported shape            */
+  LAZY_E_BADSCHEDULE = -2, /* schedule not strictly increasing / keep fractions increasing  */
+  LAZY_E_CAPACITY = -3,    /* more tokens, sequences or workspace than the context was sized for */
+  LAZY_E_NOT_IN_AUX = -4,  /* a position asked from an Aux Cache is not held there          */
+  LAZY_E_TIMEOUT = -5,     /* a bounded device-side wait ran out                            */
+  LAZY_E_CUDA = -6,        /* a CUDA runtime / driver call failed                           */
+  LAZY_E_STATE = -7        /* call out of order (decode before prefill, ...)                */
+} lazy_status;
+
+enum { LAZY_BF16 = 0, LAZY_F32 = 1 };
+
+typedef struct lazy_ctx lazy_ctx;
+
+/* Model shape (Section 1: Llama 2 7B = 32 layers, model dimension 4096) and capacities. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t dtype;             /* LAZY_BF16 or LAZY_F32                                         */
+  int32_t max_seqs;          /* sequences per batch                                          */
+  int32_t max_prompt_tokens; /* packed total over the batch                                  */
+  int32_t max_new_tokens;    /* decode steps per sequence the caches leave room for          */
+} lazy_model_cfg;
+
+/* Weights, all device memory except the per-layer pointer arrays themselves (host arrays of
+ * n_layers device pointers).  w_qkv = [3d, d] with the q rows first, then k, then v. */
+typedef struct {
+  const void *tok_embed;          /* [vocab, d]                */
+  const void *const *w_qkv;       /* n_layers x [3d, d]        */
+  const void *const *w_o;         /* n_layers x [d, d]         */
+  const void *const *w_gate;      /* n_layers x [d_ffn, d]     */
+  const void *const *w_up;        /* n_layers x [d_ffn, d]     */
+  const void *const *w_down;      /* n_layers x [d, d_ffn]     */
+  const void *const *g_attn;      /* n_layers x [d] RMSNorm gain before attention */
+  const void *const *g_mlp;       /* n_layers x [d] RMSNorm gain before the MLP   */
+  const void *g_final;            /* [d]                       */
+  const void *w_lm_head;          /* [vocab, d]                */
+} lazy_weights;
+
+/* Layer-wise keep schedule (Section 3.2, progressive token pruning; the three knobs of
+ * Section 4.2: how many pruning layers, where, how many tokens).  Point i says: the set that
+ * ENTERS layer layer_entered[i] holds ceil(keep_bp[i]/10000 * N) tokens of the N-token
+ * prompt, chosen by the Eq. 1 score of layer layer_entered[i]-1.  Layer 0 sees everything.
+ * layer_entered strictly increasing in (0, n_layers); keep_bp in 1..10000, non-increasing. */
+typedef struct {
+  int32_t n_points;
+  const int32_t *layer_entered; /* host */
+  const uint32_t *keep_bp;      /* host */
+} lazy_schedule;
+
+/* Counters of the latest prefill / decode call (Section 4.3 "% of prompt tokens computed",
+ * Section 4.5 cumulative token usage = KV-cache size per layer). Host struct, filled by
+ * lazy_get_stats. Arrays are indexed by layer, up to LAZY_MAX_LAYERS. */
+#define LAZY_MAX_LAYERS 128
+typedef struct {
+  int32_t n_layers;
+  int32_t rows_computed[LAZY_MAX_LAYERS]; /* rows that went through each layer in the latest call */
+  int32_t kv_rows[LAZY_MAX_LAYERS];       /* tokens whose K/V exist at each layer (all sequences)  */
+  int32_t aux_rows[LAZY_MAX_LAYERS];      /* tokens held by the Aux Cache that follows each layer  */
+  int32_t revived[LAZY_MAX_LAYERS];       /* rows revived into each layer in the latest call       */
+  int64_t kernel_launches;                /* kernels enqueued by the latest call                   */
+} lazy_stats;
+
+/* ---- context ------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context of this shape and schedule needs (0 on bad args). */
+size_t lazy_prefill_workspace_bytes(const lazy_model_cfg *cfg, const lazy_schedule *sched);
+
+/* Validates cfg and schedule, records the weight pointers and carves `d_workspace`
+ * (256-byte aligned, at least lazy_prefill_workspace_bytes).  Enqueues a few small set-up
+ * kernels (RoPE table) on the default stream and synchronises before returning.  On success
+ * *out owns host memory only. */
+int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const lazy_schedule *sched,
+                      void *d_workspace, size_t workspace_bytes, lazy_ctx **out);
+
+/* Token-pruned prefill (Section 3.1 prefilling stage; Section 3.2 progressive token pruning,
+ * Eq. 1, Aux Cache).  d_prompt_ids: device int32, the prompts packed back to back;
+ * h_cu_seqlens: host int32[n_seqs+1], cumulative lengths (h_cu_seqlens[0] = 0).
+ * Writes fp32 next-token logits [n_seqs, vocab] to d_logits (device) and leaves per-layer KV
+ * caches and Aux Caches in the workspace for decode.  Resets any earlier generation state.
+ * Row counts follow from (lengths, schedule) alone, so nothing is read back: the call only
+ * enqueues work on `stream`. */
+int lazy_prefill_run(lazy_ctx *ctx, void *stream, const int32_t *d_prompt_ids,
+                     const int32_t *h_cu_seqlens, int32_t n_seqs, float *d_logits);
+
+/* One decode step for every sequence of the batch (Section 3.1 decoding stage; Section 3.2:
+ * each step re-selects its context set by the new token's Eq. 1 score and may revive pruned
+ * tokens from the Aux Cache instead of recomputing them).  d_new_ids: device int32[n_seqs],
+ * the token appended to each sequence.  d_logits: device fp32 [n_seqs, vocab].  d_next_ids:
+ * device int32[n_seqs] greedy argmax (lowest id on ties) or NULL.  How many rows are revived
+ * depends on the data: at every scheduled layer the call reads a few counters back
+ * (a stream synchronisation), so it returns with the step's selection already decided. */
+int lazy_decode_step(lazy_ctx *ctx, void *stream, const int32_t *d_new_ids, float *d_logits,
+                     int32_t *d_next_ids);
+
+/* Reads hidden states of pruned tokens from the Aux Cache that follows `layer` (Section 3.2,
+ * Aux Cache: hidden states of tokens whose KV is absent from the next layer's cache).
+ * d_positions: device int32[n] original token positions of sequence `seq`; d_hidden_out:
+ * device [n, d_model] in the context's dtype.  The entries stay in the cache.  Synchronises
+ * the stream; a position not held there gives LAZY_E_NOT_IN_AUX (rows of found positions are
+ * still written). */
+int aux_cache_revive(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq,
+                     const int32_t *d_positions, int32_t n, void *d_hidden_out);
+
+/* ---- introspection (parity checks, replay of another implementation's kept sets) ------- */
+
+/* Kept set entering `layer_entered` (a schedule point) of sequence `seq` in the latest call, as
+ * original token positions ascending; d_pos: device int32 with room for the count (may be NULL
+ * to query the count only).  Synchronises the stream. */
+int lazy_get_kept(lazy_ctx *ctx, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
+                  int32_t *h_count);
+/* Eq. 1 scores of `layer` for sequence `seq` in the latest call, one per candidate row in
+ * ascending position order (prefill: the rows present at that layer). */
+int lazy_get_scores(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, float *d_scores,
+                    int32_t *h_count);
+/* Test hook: the NEXT prefill (decode step) takes this kept set (positions, ascending, device
+ * int32[n]; the last token is kept regardless) at the schedule point instead of selecting by
+ * score.  n = 0 clears the hook for that point.  The array must stay valid until that call
+ * has run. */
+int lazy_set_forced_keep(lazy_ctx *ctx, int32_t layer_entered, int32_t seq, const int32_t *d_pos,
+                         int32_t n);
+/* With capture on, every prefill also keeps the residual stream after each layer
+ * (workspace must have been sized with capture in mind: see lazy_prefill_workspace_bytes_ex). */
+size_t lazy_prefill_workspace_bytes_ex(const lazy_model_cfg *cfg, const lazy_schedule *sched,
+                                       int32_t debug_capture);
+int lazy_set_debug_capture(lazy_ctx *ctx, int32_t on);
+/* Residual stream after layer `layer` of the latest PREFILL, all sequences packed:
+ * d_out [rows, d_model] (context dtype; may be NULL to query rows).  LAZY_E_STATE if capture
+ * was off. */
+int lazy_get_hidden(lazy_ctx *ctx, void *stream, int32_t layer, void *d_out, int32_t *h_rows);
+/* KV-cache / Aux-Cache contents of a layer for sequence `seq`: positions in order of insertion
+ * and the rows.  Any of the device outputs may be NULL. */
+int lazy_get_kv(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t *d_pos, void *d_k,
+                void *d_v, int32_t *h_count);
+int lazy_get_aux(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t *d_pos,
+                 void *d_hidden, int32_t *h_count);
+int lazy_get_stats(lazy_ctx *ctx, lazy_stats *out);
+/* Synchronises `stream` and returns the first device-side error recorded since the last call
+ * of this function (LAZY_OK if none), clearing it. */
+int lazy_sync_status(lazy_ctx *ctx, void *stream);
+/* Same, for the context-free calls below. */
+int lazy_device_status(void *stream);
+void lazy_destroy(lazy_ctx *ctx);
+const char *lazy_strerror(int status);
+
+/* ---- single-layer pruning op ------------------------------------------------------------ */
+
+/* One layer's attention half followed by the cut (Section 3.2): RMSNorm, QKV projection, RoPE,
+ * causal attention, output projection + residual, Eq. 1 score of the last row, top-percentile
+ * selection, then gather of the kept hidden / K / V / position rows and scatter of the pruned
+ * hidden rows into an Aux Cache.  All pointers device, bf16 (dtype LAZY_BF16) or fp32.
+ *   x [n, d] hidden states entering the layer; pos int32[n] ascending positions;
+ *   w_qkv [3d, d], w_o [d, d], g_attn [d]; keep_bp: keep ceil(keep_bp/10000*n) rows;
+ *   max_pos: every position is < max_pos (sizes the RoPE table kept in the workspace).
+ * Outputs: scores fp32[n]; keep_idx int32[n_keep], drop_idx int32[n-n_keep] (row indices,
+ * ascending); hidden_kept [n_keep, d], k_kept / v_kept [n_keep, d] (k rotated),
+ * pos_kept int32[n_keep]; aux_hidden [n-n_keep, d], aux_pos int32[n-n_keep].
+ * d_workspace: lazy_prune_op_workspace_bytes(...) bytes.  forced_keep_idx (device, may be NULL):
+ * n_forced row indices ascending that replace the score-based choice (test hook). */
+size_t lazy_prune_op_workspace_bytes(int32_t n, int32_t d_model, int32_t n_heads, int32_t head_dim,
+                                     int32_t dtype, int32_t max_pos);
+int lazy_prune_op(void *stream, int32_t dtype, int32_t n, int32_t d_model, int32_t n_heads,
+                  int32_t head_dim, int32_t max_pos, float rms_eps, float rope_theta, uint32_t keep_bp,
+                  const void *x, const int32_t *pos, const void *w_qkv, const void *w_o,
+                  const void *g_attn, const int32_t *forced_keep_idx, int32_t n_forced,
+                  float *scores, int32_t *keep_idx, int32_t *drop_idx, void *hidden_kept,
+                  void *k_kept, void *v_kept, int32_t *pos_kept, void *aux_hidden,
+                  int32_t *aux_pos, void *d_workspace, size_t workspace_bytes);
+
+/* ---- individual steps of the path (each also used inside the calls above) ----------------- */
+
+/* y[r,:] = x[r,:] * rsqrt(mean(x[r,:]^2) + eps) * g  (Llama-2 pre-norm). x, y [n, d]. */
+int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, void *y, int32_t n,
+                   int32_t d, float eps);
+/* C[M,N] = A[M,K] * B[N,K]^T (+ R[M,N] if R != NULL). bf16: tcgen05 tensor cores, TMA-fed;
+ * fp32: CUDA cores. lda = K, ldc = N (dense).  K and N multiples of 8.  impl: 0 = the
+ * dtype's production kernel, 1 = the CUDA-core kernel (cross-check). */
+int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B,
+                const void *R, void *C, int32_t M, int32_t N, int32_t K);
+/* C[M,F] = silu(A Bg^T) * (A Bu^T), Bg, Bu [F, K] (SwiGLU, first half of the MLP). */
+int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
+                       const void *Bu, void *C, int32_t M, int32_t F, int32_t K);
+/* In-place RoPE of q and k inside qkv [n, 3*H*dh] by positions pos[n]; rotated k and v are
+ * also written to kcache / vcache [n, H*dh].  rope_table: device fp32[max_pos*head_dim] scratch
+ * that the call fills first. */
+int lazy_k_rope_kv(void *stream, int32_t dtype, void *qkv, const int32_t *pos, float *rope_table,
+                   void *kcache, void *vcache, int32_t n, int32_t n_heads, int32_t head_dim,
+                   int32_t max_pos, float theta);
+/* Causal multi-head attention over packed sequences. q: rows of stride ldq elements, k/v rows of
+ * stride ldkv; o [n, H*dh] dense. d_cu_seqlens: device int32[n_seqs+1]. */
+int lazy_k_attention(void *stream, int32_t dtype, const void *q, int32_t ldq, const void *k,
+                     const void *v, int32_t ldkv, void *o, const int32_t *d_cu_seqlens,
+                     int32_t n_seqs, int32_t max_len, int32_t n_total, int32_t n_heads,
+                     int32_t head_dim);
+/* Eq. 1: s[j] = (1/H) sum_h softmax_j(q_last,h . k_j,h / sqrt(dh)) per sequence, q_last = the
+ * sequence's last row. scratch: device fp32[lazy_k_score_scratch_floats(...)]. */
+size_t lazy_k_score_scratch_floats(int32_t n_seqs, int32_t n_total, int32_t n_heads);
+int lazy_k_score(void *stream, int32_t dtype, const void *q, int32_t ldq, const void *k,
+                 int32_t ldkv, const int32_t *d_cu_seqlens, int32_t n_seqs, int32_t n_total,
+                 int32_t n_heads, int32_t head_dim, float *scratch, float *scores);
+/* Top-percentile selection per sequence (Section 3.2): keeps n_keep[s] rows with the largest
+ * score, the last row always, ties to the lower index.  d_cu_in / d_cu_keep: device
+ * int32[n_seqs+1] prefix sums of rows in / rows kept.  keep_idx / drop_idx receive packed row
+ * indices (global, ascending within a sequence); drop rows of sequence s start at
+ * d_cu_in[s]-d_cu_keep[s]. */
+int lazy_k_select(void *stream, const float *scores, const int32_t *d_cu_in,
+                  const int32_t *d_cu_keep, int32_t n_seqs, int32_t *keep_idx, int32_t *drop_idx);
+/* dst[i,:] = src[idx[i],:] for i < n (row gather), rows of `row_bytes` bytes (multiple of 16);
+ * src has src_rows rows (indices outside are reported, not dereferenced). */
+int lazy_k_gather_rows(void *stream, const void *src, const int32_t *idx, void *dst, int32_t n,
+                       int32_t row_bytes, int32_t src_rows);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAZYLLM_H_ */

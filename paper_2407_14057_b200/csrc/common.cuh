@@ -1,0 +1,186 @@
+// Shared declarations of the CUDA side: status word, launch helpers, storage-type traits.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lazyllm.h"
+
+namespace lazy {
+
+// ---- device status word -------------------------------------------------------------------
+// First error wins.  `where` identifies the wait or check that failed.
+struct DevStatus {
+  int code;
+  int where;
+  int a;
+  int b;
+};
+
+enum DevWhere {
+  W_GEMM_PRODUCER = 1,
+  W_GEMM_MMA_FULL = 2,
+  W_GEMM_MMA_TMEM = 3,
+  W_GEMM_EPILOGUE = 4,
+  W_GATHER_INDEX = 5,
+  W_AUX_LOOKUP = 6,
+  W_EMBED_ID = 7,
+  W_SELECT = 8,
+  W_DECODE = 9,
+  W_ROPE_POS = 10,
+};
+
+__device__ __forceinline__ void dev_fail(DevStatus *st, int code, int where, int a = 0, int b = 0) {
+  if (atomicCAS(&st->code, 0, code) == 0) {
+    st->where = where;
+    st->a = a;
+    st->b = b;
+  }
+}
+
+// Address of this device's status word (a __device__ global of the library); NULL on failure.
+DevStatus *dev_status_ptr();
+// Synchronises the stream, returns and clears the status word.
+int sync_and_take_status(cudaStream_t stream, int *where_out);
+
+// ---- storage types --------------------------------------------------------------------------
+typedef __nv_bfloat16 bf16;
+
+template <typename T>
+struct Elem;
+template <>
+struct Elem<float> {
+  static constexpr int kPerVec = 4;  // elements per 16-byte vector
+  __device__ static __forceinline__ float to_f(float v) { return v; }
+  __device__ static __forceinline__ float from_f(float v) { return v; }
+};
+template <>
+struct Elem<bf16> {
+  static constexpr int kPerVec = 8;
+  __device__ static __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+  __device__ static __forceinline__ bf16 from_f(float v) { return __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ void bf16x2_unpack(uint32_t u, float &lo, float &hi) {
+  lo = __uint_as_float(u << 16);
+  hi = __uint_as_float(u & 0xffff0000u);
+}
+__device__ __forceinline__ uint32_t bf16x2_pack(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// 16-byte vector of T, unpacked to floats and back.
+template <typename T>
+struct Vec16 {
+  uint4 raw;
+  __device__ __forceinline__ void load(const T *p) { raw = *reinterpret_cast<const uint4 *>(p); }
+  __device__ __forceinline__ void store(T *p) const { *reinterpret_cast<uint4 *>(p) = raw; }
+  __device__ __forceinline__ void unpack(float *f) const;
+  __device__ __forceinline__ void pack(const float *f);
+};
+template <>
+__device__ __forceinline__ void Vec16<float>::unpack(float *f) const {
+  f[0] = __uint_as_float(raw.x);
+  f[1] = __uint_as_float(raw.y);
+  f[2] = __uint_as_float(raw.z);
+  f[3] = __uint_as_float(raw.w);
+}
+template <>
+__device__ __forceinline__ void Vec16<float>::pack(const float *f) {
+  raw = make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                   __float_as_uint(f[3]));
+}
+template <>
+__device__ __forceinline__ void Vec16<bf16>::unpack(float *f) const {
+  bf16x2_unpack(raw.x, f[0], f[1]);
+  bf16x2_unpack(raw.y, f[2], f[3]);
+  bf16x2_unpack(raw.z, f[4], f[5]);
+  bf16x2_unpack(raw.w, f[6], f[7]);
+}
+template <>
+__device__ __forceinline__ void Vec16<bf16>::pack(const float *f) {
+  raw = make_uint4(bf16x2_pack(f[0], f[1]), bf16x2_pack(f[2], f[3]), bf16x2_pack(f[4], f[5]),
+                   bf16x2_pack(f[6], f[7]));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+inline int elem_bytes(int dtype) { return dtype == LAZY_F32 ? 4 : 2; }
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Number of SMs of the current device (cached).
+int sm_count();
+// Counts kernels enqueued by this library (per process); used for the launch statistics.
+extern long long g_launches;
+#define LAZY_COUNT_LAUNCH() (++::lazy::g_launches)
+
+#define LAZY_CUDA_OK(expr)                      \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return LAZY_E_CUDA; \
+  } while (0)
+#define LAZY_TRY(expr)                \
+  do {                                \
+    int rc__ = (expr);                \
+    if (rc__ != LAZY_OK) return rc__; \
+  } while (0)
+
+inline int launch_ok() { return cudaPeekAtLastError() == cudaSuccess ? LAZY_OK : LAZY_E_CUDA; }
+
+// ---- launchers (one per step of the path); all enqueue on `st` and return a lazy_status ----
+int launch_embed(cudaStream_t st, int dtype, const void *table, const int32_t *ids, void *x, int n,
+                 int d, int vocab, DevStatus *status);
+int launch_rmsnorm(cudaStream_t st, int dtype, const void *x, const void *g, void *y, int n, int d,
+                   float eps);
+// rows listed in row_idx (or rows 0..n-1 if NULL) of x -> y rows 0..n-1
+int launch_rmsnorm_rows(cudaStream_t st, int dtype, const void *x, const int32_t *row_idx,
+                        const void *g, void *y, int n, int d, float eps);
+int launch_rope_table(cudaStream_t st, float *table, int max_pos, int head_dim, float theta);
+// q rotated in place inside qkv; rotated k and v written to the caches at row kv_row[r]
+// (or kv_row_offset + r if kv_row is NULL) together with the position tag.
+int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, const float *table,
+                   void *kcache, void *vcache, int32_t *kv_pos, const int32_t *kv_row, int n,
+                   int n_heads, int head_dim, int max_pos, DevStatus *status);
+int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
+                int M, int N, int K, DevStatus *status);
+int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
+                       void *C, int M, int F, int K, DevStatus *status);
+int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
+                     const void *R, void *C, int M, int N, int K, int swiglu);
+// Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows
+// kv_base[s] + j of k/v (kv_base NULL: same rows as q). Query row i sees keys j <= i (prefill).
+int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
+                     const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
+                     int n_seqs, int max_len, int n_total, int n_heads, int head_dim);
+size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
+int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
+                 const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
+                 int n_heads, int head_dim, float *scratch, float *scores);
+int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
+                  const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
+                  DevStatus *status);
+// scores[r] = 2 if pos[r] is in the ascending list forced[0..n_forced), else 0 (rows r0..r0+n)
+int launch_forced_scores(cudaStream_t st, const int32_t *pos, int r0, int n, const int32_t *forced,
+                         int n_forced, float *scores);
+int launch_gather_rows(cudaStream_t st, const void *src, const int32_t *idx, void *dst, int n,
+                       int row_bytes, int src_rows, DevStatus *status);
+int launch_gather_i32(cudaStream_t st, const int32_t *src, const int32_t *idx, int32_t *dst, int n);
+int launch_lm_head(cudaStream_t st, int dtype, const void *h, const void *w, float *logits,
+                   int n_rows, int d, int vocab);
+int launch_argmax(cudaStream_t st, const float *logits, int32_t *out, int n_rows, int vocab);
+int launch_fill_i32(cudaStream_t st, int32_t *p, int32_t v, size_t n);
+int launch_iota_pos(cudaStream_t st, int32_t *pos, const int32_t *cu, int n_seqs, int n_total);
+
+}  // namespace lazy

@@ -1,0 +1,612 @@
+// Context set-up, the token-pruned prefill, Aux-Cache reads and the introspection calls.
+#include <string.h>
+
+#include <new>
+
+#include "runtime.cuh"
+
+namespace lazy {
+
+// ---- small kernels used only by the runtime ---------------------------------------------------
+__global__ void move_rows_kernel(const uint4 *__restrict__ src, const int32_t *__restrict__ src_idx,
+                                 uint4 *__restrict__ dst, const int32_t *__restrict__ dst_idx, int n,
+                                 int vec_per_row, int src_rows, int dst_rows, DevStatus *status) {
+  for (int r = blockIdx.x; r < n; r += gridDim.x) {
+    const int s = src_idx ? src_idx[r] : r;
+    const int t = dst_idx ? dst_idx[r] : r;
+    if (s < 0 || s >= src_rows || t < 0 || t >= dst_rows) {
+      if (threadIdx.x == 0) dev_fail(status, LAZY_E_BADARG, W_GATHER_INDEX, s, t);
+      continue;
+    }
+    const uint4 *sp = src + (size_t)s * vec_per_row;
+    uint4 *dp = dst + (size_t)t * vec_per_row;
+    for (int i = threadIdx.x; i < vec_per_row; i += blockDim.x) dp[i] = sp[i];
+  }
+}
+int launch_move_rows(cudaStream_t st, const void *src, const int32_t *src_idx, void *dst,
+                     const int32_t *dst_idx, int n, int row_bytes, int src_rows, int dst_rows,
+                     DevStatus *status) {
+  if (n == 0) return LAZY_OK;
+  int blocks = n < sm_count() * 16 ? n : sm_count() * 16;
+  move_rows_kernel<<<blocks, 128, 0, st>>>((const uint4 *)src, src_idx, (uint4 *)dst, dst_idx, n,
+                                           row_bytes / 16, src_rows, dst_rows, status);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+__global__ void move_i32_kernel(const int32_t *src, const int32_t *src_idx, int32_t *dst,
+                                const int32_t *dst_idx, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[dst_idx ? dst_idx[i] : i] = src[src_idx ? src_idx[i] : i];
+}
+int launch_move_i32(cudaStream_t st, const int32_t *src, const int32_t *src_idx, int32_t *dst,
+                    const int32_t *dst_idx, int n) {
+  if (n == 0) return LAZY_OK;
+  move_i32_kernel<<<cdiv(n, 256), 256, 0, st>>>(src, src_idx, dst, dst_idx, n);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+__global__ void seg_rows_kernel(const int32_t *cu, const int32_t *base, int n_seqs, int n_total,
+                                int32_t *out) {
+  int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= n_total) return;
+  int lo = 0, hi = n_seqs;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= r) lo = mid; else hi = mid;
+  }
+  out[r] = base[lo] + (r - cu[lo]);
+}
+int launch_seg_rows(cudaStream_t st, const int32_t *cu, const int32_t *base, int n_seqs, int n_total,
+                    int32_t *out) {
+  if (n_total == 0) return LAZY_OK;
+  seg_rows_kernel<<<cdiv(n_total, 256), 256, 0, st>>>(cu, base, n_seqs, n_total, out);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+// For each requested position: the Aux row that holds it (scan of the sequence's region), or -1.
+__global__ void aux_find_kernel(const int32_t *__restrict__ aux_pos, int region0, int count,
+                                const int32_t *__restrict__ want, int n, int32_t *__restrict__ found,
+                                DevStatus *status) {
+  const int i = blockIdx.x;
+  if (i >= n) return;
+  const int p = want[i];
+  __shared__ int hit;
+  if (threadIdx.x == 0) hit = -1;
+  __syncthreads();
+  for (int j = threadIdx.x; j < count; j += blockDim.x)
+    if (aux_pos[region0 + j] == p) hit = region0 + j;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    found[i] = hit;
+    if (hit < 0) dev_fail(status, LAZY_E_NOT_IN_AUX, W_AUX_LOOKUP, i, p);
+  }
+}
+
+// ---- validation ------------------------------------------------------------------------------------
+int validate_cfg(const lazy_model_cfg *c) {
+  if (!c) return LAZY_E_BADARG;
+  if (c->n_layers < 1 || c->n_layers > LAZY_MAX_LAYERS || c->d_model < 1 || c->n_heads < 1 ||
+      c->head_dim < 1 || c->d_ffn < 1 || c->vocab < 1)
+    return LAZY_E_BADARG;
+  if (c->n_heads * c->head_dim != c->d_model) return LAZY_E_BADARG;
+  if (c->dtype != LAZY_BF16 && c->dtype != LAZY_F32) return LAZY_E_BADARG;
+  // 16-byte vectors everywhere; RoPE pairs 16-byte vectors of the two halves of a head;
+  // the generic attention kernel gives each lane head_dim/32 output columns.
+  const int v = c->dtype == LAZY_F32 ? 4 : 8;
+  if (c->d_model % 8 || c->d_ffn % 8 || (c->head_dim / 2) % v || c->head_dim % 32 || c->head_dim > 256)
+    return LAZY_E_BADARG;
+  const int lpk = c->head_dim / v;
+  if (lpk > 32 || (lpk & (lpk - 1))) return LAZY_E_BADARG;
+  if (c->max_seqs < 1 || c->max_prompt_tokens < 1 || c->max_new_tokens < 0) return LAZY_E_BADARG;
+  if (!(c->rms_eps > 0.f) || !(c->rope_theta > 0.f)) return LAZY_E_BADARG;
+  return LAZY_OK;
+}
+
+int validate_schedule(const lazy_model_cfg *c, const lazy_schedule *s) {
+  if (!s || s->n_points < 0 || s->n_points >= LAZY_MAX_LAYERS) return LAZY_E_BADSCHEDULE;
+  if (s->n_points > 0 && (!s->layer_entered || !s->keep_bp)) return LAZY_E_BADSCHEDULE;
+  int prev_e = 0;
+  uint32_t prev_bp = 10000;
+  for (int i = 0; i < s->n_points; ++i) {
+    const int e = s->layer_entered[i];
+    const uint32_t bp = s->keep_bp[i];
+    if (!(prev_e < e && e < c->n_layers)) return LAZY_E_BADSCHEDULE;
+    if (bp < 1 || bp > 10000 || bp > prev_bp) return LAZY_E_BADSCHEDULE;
+    prev_e = e;
+    prev_bp = bp;
+  }
+  return LAZY_OK;
+}
+
+// ---- workspace carve-up -------------------------------------------------------------------------------
+struct Carver {
+  char *base;
+  size_t off;
+  explicit Carver(char *b) : base(b), off(0) {}
+  char *take(size_t bytes) {
+    char *p = base ? base + off : nullptr;
+    off += align_up(bytes ? bytes : 1, 256);
+    return p;
+  }
+};
+
+// Fills the pointers of `c` (all NULL-based offsets when base is NULL) and returns the bytes needed.
+static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
+  Carver k(base);
+  const size_t rb = c->row_bytes();
+  const size_t R = (size_t)c->cap_rows, KV = (size_t)c->cap_kv;
+  const int P = c->P, L = c->L;
+  c->x = k.take(R * rb);
+  c->x2 = k.take(R * rb);
+  c->h = k.take(R * rb);
+  c->qkv = k.take(R * rb * 3);
+  c->attn = k.take(R * rb);
+  c->act = k.take(R * (size_t)c->F * c->eb);
+  c->h_last = k.take((size_t)c->S * rb);
+  c->pos_seg.assign(P + 1, nullptr);
+  c->kv_row.assign(P + 1, nullptr);
+  for (int g = 0; g <= P; ++g) {
+    c->pos_seg[g] = (int32_t *)k.take(R * 4);
+    c->kv_row[g] = (int32_t *)k.take(R * 4);
+  }
+  c->scores = (float *)k.take((size_t)L * R * 4);
+  c->sel_scores = (float *)k.take(R * 4);
+  c->score_scratch = (float *)k.take(score_scratch_floats(c->S, c->cap_kv, c->H) * 4);
+  c->keep_idx.assign(P, nullptr);
+  c->drop_idx.assign(P, nullptr);
+  c->aux_dst.assign(P, nullptr);
+  for (int p = 0; p < P; ++p) {
+    c->keep_idx[p] = (int32_t *)k.take(R * 4);
+    c->drop_idx[p] = (int32_t *)k.take(R * 4);
+    c->aux_dst[p] = (int32_t *)k.take(R * 4);
+  }
+  c->rope_table = (float *)k.take((size_t)c->max_pos * c->dh * 4);
+  c->kcache = k.take((size_t)L * KV * rb);
+  c->vcache = k.take((size_t)L * KV * rb);
+  c->kv_pos = (int32_t *)k.take((size_t)L * KV * 4);
+  c->aux_rows = k.take((size_t)P * KV * rb);
+  c->aux_pos = (int32_t *)k.take((size_t)P * KV * 4);
+  c->d_ints = (int32_t *)k.take((size_t)(2 * P + 8) * (c->S + 1) * 4);
+  c->d_found = (int32_t *)k.take(KV * 4);
+  c->kv_map = (int32_t *)k.take((size_t)L * KV * 4);
+  c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
+  c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)64 * (c->S + 1) * 4);
+  c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
+  c->capture = with_capture ? k.take((size_t)L * R * rb) : nullptr;
+  return k.off;
+}
+
+static void fill_shape(lazy_ctx *c, const lazy_model_cfg *cfg, const lazy_schedule *s) {
+  c->cfg = *cfg;
+  c->L = cfg->n_layers;
+  c->d = cfg->d_model;
+  c->H = cfg->n_heads;
+  c->dh = cfg->head_dim;
+  c->F = cfg->d_ffn;
+  c->V = cfg->vocab;
+  c->dtype = cfg->dtype;
+  c->eb = elem_bytes(cfg->dtype);
+  c->S = cfg->max_seqs;
+  c->P = s->n_points;
+  c->sched_layer.assign(s->layer_entered, s->layer_entered + s->n_points);
+  c->sched_bp.assign(s->keep_bp, s->keep_bp + s->n_points);
+  c->point_at.assign(c->L + 1, -1);
+  for (int p = 0; p < c->P; ++p) c->point_at[c->sched_layer[p]] = p;
+  c->cap_rows = cfg->max_prompt_tokens;
+  c->cap_kv = cfg->max_prompt_tokens + cfg->max_seqs * cfg->max_new_tokens;
+  c->max_pos = cfg->max_prompt_tokens + cfg->max_new_tokens;
+}
+
+}  // namespace lazy
+
+using namespace lazy;
+
+// =====================================================================================================
+extern "C" {
+
+size_t lazy_prefill_workspace_bytes_ex(const lazy_model_cfg *cfg, const lazy_schedule *sched,
+                                       int32_t debug_capture) {
+  if (validate_cfg(cfg) != LAZY_OK || validate_schedule(cfg, sched) != LAZY_OK) return 0;
+  lazy_ctx tmp;
+  fill_shape(&tmp, cfg, sched);
+  return carve(&tmp, nullptr, debug_capture != 0);
+}
+size_t lazy_prefill_workspace_bytes(const lazy_model_cfg *cfg, const lazy_schedule *sched) {
+  return lazy_prefill_workspace_bytes_ex(cfg, sched, 0);
+}
+
+int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const lazy_schedule *sched,
+                      void *d_workspace, size_t workspace_bytes, lazy_ctx **out) {
+  if (!out) return LAZY_E_BADARG;
+  *out = nullptr;
+  LAZY_TRY(validate_cfg(cfg));
+  int rc = validate_schedule(cfg, sched);
+  if (rc != LAZY_OK) return rc;
+  if (!w || !d_workspace || ((uintptr_t)d_workspace & 255)) return LAZY_E_BADARG;
+  if (!w->tok_embed || !w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn ||
+      !w->g_mlp || !w->g_final || !w->w_lm_head)
+    return LAZY_E_BADARG;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const void *ps[7] = {w->w_qkv[l], w->w_o[l], w->w_gate[l], w->w_up[l], w->w_down[l], w->g_attn[l],
+                         w->g_mlp[l]};
+    for (const void *p : ps)
+      if (!p || ((uintptr_t)p & 15)) return LAZY_E_BADARG;
+  }
+  lazy_ctx *c = new (std::nothrow) lazy_ctx();
+  if (!c) return LAZY_E_BADARG;
+  fill_shape(c, cfg, sched);
+  const size_t need = carve(c, nullptr, false);
+  const size_t need_cap = carve(c, nullptr, true);
+  if (workspace_bytes < need) {
+    delete c;
+    return LAZY_E_CAPACITY;
+  }
+  c->capture_sized = workspace_bytes >= need_cap;
+  carve(c, (char *)d_workspace, c->capture_sized);
+  c->ws_base = (char *)d_workspace;
+  c->ws_bytes = workspace_bytes;
+  c->capture_on = false;
+  c->tok_embed = w->tok_embed;
+  c->g_final = w->g_final;
+  c->w_lm_head = w->w_lm_head;
+  c->w_qkv.assign(w->w_qkv, w->w_qkv + c->L);
+  c->w_o.assign(w->w_o, w->w_o + c->L);
+  c->w_gate.assign(w->w_gate, w->w_gate + c->L);
+  c->w_up.assign(w->w_up, w->w_up + c->L);
+  c->w_down.assign(w->w_down, w->w_down + c->L);
+  c->g_attn.assign(w->g_attn, w->g_attn + c->L);
+  c->g_mlp.assign(w->g_mlp, w->g_mlp + c->L);
+  c->have_prefill = false;
+  c->maps_built = false;
+  c->n_seqs = 0;
+  memset(&c->stats, 0, sizeof(c->stats));
+  if (!dev_status_ptr()) {
+    delete c;
+    return LAZY_E_CUDA;
+  }
+  rc = launch_rope_table(0, c->rope_table, c->max_pos, c->dh, cfg->rope_theta);
+  if (rc == LAZY_OK && cudaStreamSynchronize(0) != cudaSuccess) rc = LAZY_E_CUDA;
+  if (rc != LAZY_OK) {
+    delete c;
+    return rc;
+  }
+  *out = c;
+  return LAZY_OK;
+}
+
+void lazy_destroy(lazy_ctx *ctx) { delete ctx; }
+
+const char *lazy_strerror(int status) {
+  switch (status) {
+    case LAZY_OK: return "ok";
+    case LAZY_E_BADARG: return "bad argument";
+    case LAZY_E_BADSCHEDULE: return "bad keep schedule";
+    case LAZY_E_CAPACITY: return "capacity exceeded";
+    case LAZY_E_NOT_IN_AUX: return "position not held by the Aux Cache";
+    case LAZY_E_TIMEOUT: return "bounded device-side wait ran out";
+    case LAZY_E_CUDA: return "CUDA call failed";
+    case LAZY_E_STATE: return "call out of order";
+    default: return "unknown status";
+  }
+}
+
+int lazy_set_debug_capture(lazy_ctx *c, int32_t on) {
+  if (!c) return LAZY_E_BADARG;
+  if (on && !c->capture_sized) return LAZY_E_CAPACITY;
+  c->capture_on = on != 0;
+  return LAZY_OK;
+}
+
+int lazy_set_forced_keep(lazy_ctx *c, int32_t layer_entered, int32_t seq, const int32_t *d_pos,
+                         int32_t n) {
+  if (!c || layer_entered < 0 || layer_entered > c->L || seq < 0 || seq >= c->S || n < 0)
+    return LAZY_E_BADARG;
+  const int p = c->point_at[layer_entered];
+  if (p < 0) return LAZY_E_BADARG;
+  if (n == 0) {
+    c->forced.erase(std::make_pair(p, (int)seq));
+    return LAZY_OK;
+  }
+  if (!d_pos) return LAZY_E_BADARG;
+  c->forced[std::make_pair(p, (int)seq)] = std::make_pair(d_pos, (int)n);
+  return LAZY_OK;
+}
+
+// ---------------------------------------------------------------------------------------- prefill
+int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
+                     const int32_t *h_cu_seqlens, int32_t n_seqs, float *d_logits) {
+  if (!c || !d_prompt_ids || !h_cu_seqlens || !d_logits || n_seqs < 1) return LAZY_E_BADARG;
+  if (n_seqs > c->S) return LAZY_E_CAPACITY;
+  if (h_cu_seqlens[0] != 0) return LAZY_E_BADARG;
+  for (int s = 0; s < n_seqs; ++s)
+    if (h_cu_seqlens[s + 1] <= h_cu_seqlens[s]) return LAZY_E_BADARG;  // empty prompts not allowed
+  const int N = h_cu_seqlens[n_seqs];
+  if (N > c->cap_rows) return LAZY_E_CAPACITY;
+  cudaStream_t st = (cudaStream_t)stream;
+  DevStatus *status = dev_status_ptr();
+  if (!status) return LAZY_E_CUDA;
+  const long long launches0 = g_launches;
+  const int P = c->P, L = c->L, d = c->d, dt = c->dtype;
+  const size_t rb = c->row_bytes();
+
+  // ---- host bookkeeping: every row count follows from the lengths and the schedule
+  c->have_prefill = false;
+  c->maps_built = false;
+  c->n_seqs = n_seqs;
+  c->prompt_len.resize(n_seqs);
+  c->n_tokens.resize(n_seqs);
+  c->seq_base.resize(n_seqs);
+  int max_len = 0;
+  for (int s = 0; s < n_seqs; ++s) {
+    c->prompt_len[s] = h_cu_seqlens[s + 1] - h_cu_seqlens[s];
+    c->n_tokens[s] = c->prompt_len[s];
+    c->seq_base[s] = h_cu_seqlens[s] + s * c->cfg.max_new_tokens;
+    if (c->prompt_len[s] > max_len) max_len = c->prompt_len[s];
+    if (c->prompt_len[s] + c->cfg.max_new_tokens > c->max_pos) return LAZY_E_CAPACITY;
+  }
+  c->seg_cu.assign(P + 1, std::vector<int>(n_seqs + 1, 0));
+  for (int s = 0; s <= n_seqs; ++s) c->seg_cu[0][s] = h_cu_seqlens[s];
+  std::vector<std::vector<int>> cu_drop(P, std::vector<int>(n_seqs + 1, 0));
+  for (int p = 0; p < P; ++p) {
+    for (int s = 0; s < n_seqs; ++s) {
+      const int present = c->seg_cu[p][s + 1] - c->seg_cu[p][s];
+      int keep = keep_count(c->prompt_len[s], c->sched_bp[p], present);
+      auto it = c->forced.find(std::make_pair(p, s));
+      if (it != c->forced.end()) {
+        keep = it->second.second;
+        if (keep < 1 || keep > present) return LAZY_E_BADARG;
+      }
+      c->seg_cu[p + 1][s + 1] = c->seg_cu[p + 1][s] + keep;
+      cu_drop[p][s + 1] = cu_drop[p][s] + (present - keep);
+    }
+  }
+  c->kv_count.assign(L, std::vector<int>(n_seqs, 0));
+  c->aux_count.assign(P, std::vector<int>(n_seqs, 0));
+  memset(&c->stats, 0, sizeof(c->stats));
+  c->stats.n_layers = L;
+
+  // ---- integer tables to the device: segment cu arrays, drop cu arrays, bases, last rows
+  const int W = c->S + 1;
+  std::vector<int32_t> ints((size_t)(2 * P + 8) * W, 0);
+  auto tab = [&](int i) { return ints.data() + (size_t)i * W; };
+  for (int g = 0; g <= P; ++g)
+    for (int s = 0; s <= n_seqs; ++s) tab(g)[s] = c->seg_cu[g][s];
+  for (int p = 0; p < P; ++p)
+    for (int s = 0; s <= n_seqs; ++s) tab(P + 1 + p)[s] = cu_drop[p][s];
+  for (int s = 0; s < n_seqs; ++s) {
+    tab(2 * P + 1)[s] = c->seq_base[s];
+    tab(2 * P + 2)[s] = c->seg_cu[P][s + 1] - 1;  // last row of the sequence in the final segment
+  }
+  LAZY_CUDA_OK(cudaMemcpyAsync(c->d_ints, ints.data(), ints.size() * 4, cudaMemcpyHostToDevice, st));
+  auto d_cu = [&](int g) { return c->d_ints + (size_t)g * W; };
+  auto d_cu_drop = [&](int p) { return c->d_ints + (size_t)(P + 1 + p) * W; };
+  const int32_t *d_base = c->d_ints + (size_t)(2 * P + 1) * W;
+  const int32_t *d_last = c->d_ints + (size_t)(2 * P + 2) * W;
+
+  for (int g = 0; g <= P; ++g)
+    LAZY_TRY(launch_seg_rows(st, d_cu(g), d_base, n_seqs, c->seg_cu[g][n_seqs], c->kv_row[g]));
+  for (int p = 0; p < P; ++p)
+    LAZY_TRY(launch_seg_rows(st, d_cu_drop(p), d_base, n_seqs, cu_drop[p][n_seqs], c->aux_dst[p]));
+
+  // ---- embedding, positions
+  LAZY_TRY(launch_embed(st, dt, c->tok_embed, d_prompt_ids, c->x, N, d, c->V, status));
+  LAZY_TRY(launch_iota_pos(st, c->pos_seg[0], d_cu(0), n_seqs, N));
+
+  char *x = c->x, *x2 = c->x2;
+  int g = 0;
+  for (int l = 0; l < L; ++l) {
+    const int n = c->seg_cu[g][n_seqs];
+    const int32_t *pos = c->pos_seg[g];
+    char *kc = c->kcache + (size_t)l * c->cap_kv * rb;
+    char *vc = c->vcache + (size_t)l * c->cap_kv * rb;
+    int32_t *kvp = c->kv_pos + (size_t)l * c->cap_kv;
+    float *sc = c->scores + (size_t)l * c->cap_rows;
+    int seg_max = 0;
+    for (int s = 0; s < n_seqs; ++s) {
+      const int ns = c->seg_cu[g][s + 1] - c->seg_cu[g][s];
+      c->kv_count[l][s] = ns;
+      if (ns > seg_max) seg_max = ns;
+    }
+    c->stats.rows_computed[l] = n;
+    c->stats.kv_rows[l] = n;
+
+    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
+    LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
+    LAZY_TRY(launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H,
+                            c->dh, c->max_pos, status));
+    LAZY_TRY(launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs,
+                              seg_max, n, c->H, c->dh));
+    LAZY_TRY(launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H,
+                          c->dh, c->score_scratch, sc));
+    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status));
+
+    const int p = c->point_at[l + 1];
+    if (p >= 0) {
+      // cut between attention and MLP: the MLP of this layer already runs on the kept rows
+      const float *sel = sc;
+      bool any_forced = false;
+      for (int s = 0; s < n_seqs; ++s)
+        if (c->forced.count(std::make_pair(p, s))) any_forced = true;
+      if (any_forced) {
+        LAZY_CUDA_OK(cudaMemcpyAsync(c->sel_scores, sc, (size_t)n * 4, cudaMemcpyDeviceToDevice, st));
+        for (int s = 0; s < n_seqs; ++s) {
+          auto it = c->forced.find(std::make_pair(p, s));
+          if (it == c->forced.end()) continue;
+          LAZY_TRY(launch_forced_scores(st, pos, c->seg_cu[g][s], c->seg_cu[g][s + 1] - c->seg_cu[g][s],
+                                        it->second.first, it->second.second, c->sel_scores));
+        }
+        sel = c->sel_scores;
+      }
+      const int n_keep = c->seg_cu[g + 1][n_seqs], n_drop = n - n_keep;
+      LAZY_TRY(launch_select(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->keep_idx[p], c->drop_idx[p], status));
+      char *ar = c->aux_rows + (size_t)p * c->cap_kv * rb;
+      int32_t *ap = c->aux_pos + (size_t)p * c->cap_kv;
+      LAZY_TRY(launch_move_rows(st, x, c->drop_idx[p], ar, c->aux_dst[p], n_drop, (int)rb, n, c->cap_kv, status));
+      LAZY_TRY(launch_move_i32(st, pos, c->drop_idx[p], ap, c->aux_dst[p], n_drop));
+      LAZY_TRY(launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
+      LAZY_TRY(launch_move_i32(st, pos, c->keep_idx[p], c->pos_seg[g + 1], nullptr, n_keep));
+      for (int s = 0; s < n_seqs; ++s) c->aux_count[p][s] = cu_drop[p][s + 1] - cu_drop[p][s];
+      c->stats.aux_rows[l] = n_drop;
+      char *t = x; x = x2; x2 = t;
+      ++g;
+    }
+    const int n2 = c->seg_cu[g][n_seqs];
+    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
+    LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status));
+    LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status));
+    if (c->capture_on && c->capture)
+      LAZY_CUDA_OK(cudaMemcpyAsync(c->capture + (size_t)l * c->cap_rows * rb, x, (size_t)n2 * rb,
+                                   cudaMemcpyDeviceToDevice, st));
+  }
+  // ---- first-token logits from the last row of every sequence
+  LAZY_TRY(launch_rmsnorm_rows(st, dt, x, d_last, c->g_final, c->h_last, n_seqs, d, c->cfg.rms_eps));
+  LAZY_TRY(launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, n_seqs, d, c->V));
+  // the residual stream may live in either ping-pong buffer; decode does not need it
+  c->forced.clear();
+  c->have_prefill = true;
+  c->stats.kernel_launches = g_launches - launches0;
+  return LAZY_OK;
+}
+
+// ---------------------------------------------------------------------------------------- Aux read
+int aux_cache_revive(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, const int32_t *d_positions,
+                     int32_t n, void *d_hidden_out) {
+  if (!c || layer < 0 || layer + 1 > c->L || seq < 0 || n < 0 || (n > 0 && (!d_positions || !d_hidden_out)))
+    return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int p = c->point_at[layer + 1];
+  if (p < 0) return n == 0 ? LAZY_OK : LAZY_E_NOT_IN_AUX;  // no Aux Cache follows this layer
+  if (n > c->cap_kv) return LAZY_E_CAPACITY;
+  cudaStream_t st = (cudaStream_t)stream;
+  DevStatus *status = dev_status_ptr();
+  if (!status) return LAZY_E_CUDA;
+  if (n == 0) return LAZY_OK;
+  const size_t rb = c->row_bytes();
+  const int32_t *ap = c->aux_pos + (size_t)p * c->cap_kv;
+  const char *ar = c->aux_rows + (size_t)p * c->cap_kv * rb;
+  // a pending device error of an earlier call must not be mistaken for a miss of this one
+  int rc = sync_and_take_status(st, nullptr);
+  if (rc != LAZY_OK) return rc;
+  aux_find_kernel<<<n, 128, 0, st>>>(ap, c->seq_base[seq], c->aux_count[p][seq], d_positions, n,
+                                     c->d_found, status);
+  LAZY_COUNT_LAUNCH();
+  LAZY_TRY(launch_ok());
+  // rows of found positions are copied; misses (index -1) are skipped and reported
+  LAZY_TRY(launch_move_rows(st, ar, c->d_found, d_hidden_out, nullptr, n, (int)rb, c->cap_kv, n, status));
+  rc = sync_and_take_status(st, nullptr);
+  if (rc == LAZY_E_BADARG) rc = LAZY_E_NOT_IN_AUX;
+  return rc;
+}
+
+int lazy_decode_step(lazy_ctx *c, void *stream, const int32_t *d_new_ids, float *d_logits,
+                     int32_t *d_next_ids) {
+  if (!c || !d_new_ids || !d_logits) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  return decode_step_impl(c, (cudaStream_t)stream, d_new_ids, d_logits, d_next_ids);
+}
+
+// ---------------------------------------------------------------------------------------- introspection
+int lazy_get_kept(lazy_ctx *c, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
+                  int32_t *h_count) {
+  if (!c || layer_entered < 0 || layer_entered > c->L || seq < 0) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int p = c->point_at[layer_entered];
+  if (p < 0) return LAZY_E_BADARG;
+  const int a = c->seg_cu[p + 1][seq], b = c->seg_cu[p + 1][seq + 1];
+  if (h_count) *h_count = b - a;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_pos)
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_pos, c->pos_seg[p + 1] + a, (size_t)(b - a) * 4, cudaMemcpyDeviceToDevice, st));
+  LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_scores(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, float *d_scores,
+                    int32_t *h_count) {
+  if (!c || layer < 0 || layer >= c->L || seq < 0) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int g = c->seg_of_layer(layer);
+  const int a = c->seg_cu[g][seq], b = c->seg_cu[g][seq + 1];
+  if (h_count) *h_count = b - a;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_scores)
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_scores, c->scores + (size_t)layer * c->cap_rows + a, (size_t)(b - a) * 4,
+                                 cudaMemcpyDeviceToDevice, st));
+  LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_hidden(lazy_ctx *c, void *stream, int32_t layer, void *d_out, int32_t *h_rows) {
+  if (!c || layer < 0 || layer >= c->L) return LAZY_E_BADARG;
+  if (!c->have_prefill || !c->capture_on || !c->capture) return LAZY_E_STATE;
+  int g = c->seg_of_layer(layer);
+  if (c->point_at[layer + 1] >= 0) g += 1;  // the layer's MLP already ran on the kept rows
+  const int rows = c->seg_cu[g][c->n_seqs];
+  if (h_rows) *h_rows = rows;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t rb = c->row_bytes();
+  if (d_out)
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_out, c->capture + (size_t)layer * c->cap_rows * rb, (size_t)rows * rb,
+                                 cudaMemcpyDeviceToDevice, st));
+  LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_kv(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t *d_pos, void *d_k,
+                void *d_v, int32_t *h_count) {
+  if (!c || layer < 0 || layer >= c->L || seq < 0) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int cnt = c->kv_count[layer][seq];
+  const size_t rb = c->row_bytes();
+  const size_t row0 = (size_t)layer * c->cap_kv + c->seq_base[seq];
+  if (h_count) *h_count = cnt;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_pos) LAZY_CUDA_OK(cudaMemcpyAsync(d_pos, c->kv_pos + row0, (size_t)cnt * 4, cudaMemcpyDeviceToDevice, st));
+  if (d_k) LAZY_CUDA_OK(cudaMemcpyAsync(d_k, c->kcache + row0 * rb, (size_t)cnt * rb, cudaMemcpyDeviceToDevice, st));
+  if (d_v) LAZY_CUDA_OK(cudaMemcpyAsync(d_v, c->vcache + row0 * rb, (size_t)cnt * rb, cudaMemcpyDeviceToDevice, st));
+  LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_aux(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t *d_pos, void *d_hidden,
+                 int32_t *h_count) {
+  if (!c || layer < 0 || layer >= c->L || seq < 0) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int p = layer + 1 <= c->L ? c->point_at[layer + 1] : -1;
+  if (p < 0) {
+    if (h_count) *h_count = 0;
+    return LAZY_OK;
+  }
+  const int cnt = c->aux_count[p][seq];
+  const size_t rb = c->row_bytes();
+  const size_t row0 = (size_t)p * c->cap_kv + c->seq_base[seq];
+  if (h_count) *h_count = cnt;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (d_pos) LAZY_CUDA_OK(cudaMemcpyAsync(d_pos, c->aux_pos + row0, (size_t)cnt * 4, cudaMemcpyDeviceToDevice, st));
+  if (d_hidden)
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_hidden, c->aux_rows + row0 * rb, (size_t)cnt * rb, cudaMemcpyDeviceToDevice, st));
+  LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_stats(lazy_ctx *c, lazy_stats *out) {
+  if (!c || !out) return LAZY_E_BADARG;
+  *out = c->stats;
+  return LAZY_OK;
+}
+
+int lazy_sync_status(lazy_ctx *c, void *stream) {
+  if (!c) return LAZY_E_BADARG;
+  return sync_and_take_status((cudaStream_t)stream, nullptr);
+}
+int lazy_device_status(void *stream) { return sync_and_take_status((cudaStream_t)stream, nullptr); }
+
+}  // extern "C"

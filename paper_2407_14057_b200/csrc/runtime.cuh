@@ -1,0 +1,101 @@
+// Host-side context of one generation state: shapes, weight pointers, the carved workspace and
+// the bookkeeping that prefill leaves for decode.  No device memory is owned here.
+#pragma once
+
+#include <map>
+#include <utility>
+#include <vector>
+
+#include "common.cuh"
+
+struct lazy_ctx {
+  lazy_model_cfg cfg;
+  int L, d, H, dh, F, V, dtype, eb;
+  int P;  // schedule points
+  std::vector<int> sched_layer;
+  std::vector<uint32_t> sched_bp;
+  std::vector<int> point_at;  // [L+1]: index of the schedule point entering that layer, or -1
+
+  const void *tok_embed, *g_final, *w_lm_head;
+  std::vector<const void *> w_qkv, w_o, w_gate, w_up, w_down, g_attn, g_mlp;
+
+  // capacities
+  int cap_rows;  // activation rows (packed prompt tokens; decode in-flight rows)
+  int cap_kv;    // rows of every per-layer cache: prompt tokens + max_seqs * max_new_tokens
+  int max_pos;   // positions per sequence the RoPE table covers
+  int S;         // max_seqs
+
+  // workspace carve-up (device)
+  char *ws_base;
+  size_t ws_bytes;
+  char *x, *x2, *h, *qkv, *attn, *act, *h_last;
+  std::vector<int32_t *> pos_seg;  // [P+1] positions of the rows of each segment
+  float *scores;                   // [L, cap_rows]
+  float *sel_scores;               // [cap_rows] scores handed to the selection when a set is forced
+  float *score_scratch;
+  std::vector<int32_t *> keep_idx, drop_idx;  // [P] x [cap_rows]
+  std::vector<int32_t *> aux_dst;             // [P] x [cap_rows] Aux row of the i-th dropped row
+  std::vector<int32_t *> kv_row;              // [P+1] x [cap_rows] cache row of packed row r
+  float *rope_table;
+  char *kcache, *vcache;  // [L, cap_kv, d]
+  int32_t *kv_pos;        // [L, cap_kv]
+  char *aux_rows;         // [P, cap_kv, d]
+  int32_t *aux_pos;       // [P, cap_kv]
+  int32_t *d_ints;        // small integer tables uploaded per call (cu arrays, bases, last rows)
+  int32_t *d_found;       // [cap_rows] scratch for Aux lookups
+  char *capture;          // [L, cap_rows, d] or NULL
+  // decode-only buffers
+  int32_t *kv_map;   // [L, cap_kv]: cache row of (sequence base + position), -1 if absent
+  int32_t *aux_map;  // [P, cap_kv]: Aux row of (sequence base + position), -1 if absent
+  int32_t *dec_i32;  // integer scratch of the decode step
+  float *dec_f32;
+
+  bool capture_on, capture_sized;
+
+  // ---- state of the latest call (host)
+  bool have_prefill;
+  bool maps_built;
+  int n_seqs;
+  std::vector<int> prompt_len;             // [n_seqs]
+  std::vector<int> n_tokens;               // [n_seqs] tokens so far (prompt + generated)
+  std::vector<int> seq_base;               // [n_seqs] first cache row of the sequence's region
+  std::vector<std::vector<int>> seg_cu;    // [P+1][n_seqs+1] packed row offsets per segment
+  std::vector<std::vector<int>> kv_count;  // [L][n_seqs]
+  std::vector<std::vector<int>> aux_count; // [P][n_seqs]
+  std::map<std::pair<int, int>, std::pair<const int32_t *, int>> forced;  // (point, seq) -> list
+  lazy_stats stats;
+
+  size_t row_bytes() const { return (size_t)d * eb; }
+  int seg_of_layer(int l) const {  // segment whose rows enter layer l
+    int g = 0;
+    for (int p = 0; p < P; ++p)
+      if (sched_layer[p] <= l) g = p + 1;
+    return g;
+  }
+};
+
+namespace lazy {
+
+int validate_cfg(const lazy_model_cfg *cfg);
+int validate_schedule(const lazy_model_cfg *cfg, const lazy_schedule *s);
+inline int keep_count(long long n_total, long long bp, int n_present) {
+  long long c = (n_total * bp + 9999) / 10000;
+  if (c > n_present) c = n_present;
+  if (c < 1) c = 1;
+  return (int)c;
+}
+
+// rows moved with optional source and destination index lists
+int launch_move_rows(cudaStream_t st, const void *src, const int32_t *src_idx, void *dst,
+                     const int32_t *dst_idx, int n, int row_bytes, int src_rows, int dst_rows,
+                     DevStatus *status);
+int launch_move_i32(cudaStream_t st, const int32_t *src, const int32_t *src_idx, int32_t *dst,
+                    const int32_t *dst_idx, int n);
+// out[r] = base[s] + (r - cu[s]) for the sequence s owning packed row r
+int launch_seg_rows(cudaStream_t st, const int32_t *cu, const int32_t *base, int n_seqs, int n_total,
+                    int32_t *out);
+
+int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, float *d_logits,
+                     int32_t *d_next_ids);
+
+}  // namespace lazy

@@ -1,0 +1,271 @@
+// Importance score (Eq. 1) and top-percentile selection (Section 3.2).
+//
+// Score: s_j = (1/H) sum_h softmax_j(q_last,h . k_j,h / sqrt(dh)).  Three small kernels:
+//   1. logits[h][j] for every key of every sequence: K is read once with 16-byte loads, a group of
+//      dh/8 (bf16) lanes per key, partial dot products combined with shuffles;
+//   2. per (sequence, head) max and 1/sum of exp;
+//   3. head mean of the normalised probabilities.
+// Scratch: fp32 logits [H, n_total] plus (max, 1/sum) per (sequence, head).
+//
+// Select: one CTA per sequence.  The n_keep-th largest score is found with a 4-pass, 8-bit-per-pass
+// radix select over the fp32 bit patterns (the last row is given the maximal key so it always
+// survives); a final pass in index order emits kept and dropped row indices with ballot / popcount
+// prefix sums, taking ties at the threshold in ascending index order until n_keep is reached.
+#include "common.cuh"
+
+namespace lazy {
+
+namespace {
+
+template <typename T>
+__global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *__restrict__ k,
+                                    int ldkv, const int32_t *__restrict__ cu_q,
+                                    const int32_t *__restrict__ kv_base, int n_total, int head_dim,
+                                    float *__restrict__ logits) {
+  constexpr int V = Elem<T>::kPerVec;
+  const int seq = blockIdx.z, h = blockIdx.y;
+  const int q_start = cu_q[seq];
+  const int n = cu_q[seq + 1] - q_start;
+  const int lpk = head_dim / V;       // lanes per key (power of two, <= 32)
+  const int kpw = 32 / lpk;           // keys per warp per iteration
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps = blockDim.x >> 5;
+  const int sub = lane % lpk, kslot = lane / lpk;
+  const size_t kb = kv_base ? (size_t)kv_base[seq] : (size_t)q_start;
+  if (n == 0) return;
+  // this lane's slice of the last row's query, pre-scaled
+  float qf[V];
+  {
+    Vec16<T> qv;
+    qv.load(q + (size_t)(q_start + n - 1) * ldq + h * head_dim + sub * V);
+    qv.unpack(qf);
+    const float scale = rsqrtf((float)head_dim);
+#pragma unroll
+    for (int i = 0; i < V; ++i) qf[i] *= scale;
+  }
+  const int keys_per_block = warps * kpw * 4;
+  const int j_begin = blockIdx.x * keys_per_block;
+  const int j_end = min(n, j_begin + keys_per_block);
+  for (int j0 = j_begin + warp * kpw; j0 < j_end; j0 += warps * kpw) {
+    const int j = j0 + kslot;
+    float dot = 0.f;
+    if (j < j_end) {
+      Vec16<T> kv;
+      kv.load(k + (kb + j) * ldkv + h * head_dim + sub * V);
+      float kf[V];
+      kv.unpack(kf);
+#pragma unroll
+      for (int i = 0; i < V; ++i) dot += qf[i] * kf[i];
+    }
+    for (int o = lpk >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (j < j_end && sub == 0) logits[(size_t)h * n_total + q_start + j] = dot;
+  }
+}
+
+__global__ void score_stats_kernel(const float *__restrict__ logits, const int32_t *__restrict__ cu_q,
+                                   int n_total, int n_heads, float *__restrict__ stats) {
+  const int h = blockIdx.x, seq = blockIdx.y;
+  const int q_start = cu_q[seq];
+  const int n = cu_q[seq + 1] - q_start;
+  const float *row = logits + (size_t)h * n_total + q_start;
+  __shared__ float red[32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, warps = blockDim.x >> 5;
+  float m = -INFINITY;
+  for (int j = threadIdx.x; j < n; j += blockDim.x) m = fmaxf(m, row[j]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = -INFINITY;
+  for (int w = 0; w < warps; ++w) m = fmaxf(m, red[w]);
+  __syncthreads();
+  float s = 0.f;
+  for (int j = threadIdx.x; j < n; j += blockDim.x) s += __expf(row[j] - m);
+  s = warp_sum(s);
+  if (lane == 0) red[warp] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < warps; ++w) t += red[w];
+    stats[((size_t)seq * n_heads + h) * 2 + 0] = m;
+    stats[((size_t)seq * n_heads + h) * 2 + 1] = n > 0 ? 1.f / t : 0.f;
+  }
+}
+
+__global__ void score_mean_kernel(const float *__restrict__ logits, const float *__restrict__ stats,
+                                  const int32_t *__restrict__ cu_q, int n_seqs, int n_total,
+                                  int n_heads, float *__restrict__ scores) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= n_total) return;
+  int lo = 0, hi = n_seqs;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu_q[mid] <= r) lo = mid; else hi = mid;
+  }
+  const float *st = stats + (size_t)lo * n_heads * 2;
+  float acc = 0.f;
+  for (int h = 0; h < n_heads; ++h)
+    acc += __expf(logits[(size_t)h * n_total + r] - st[2 * h]) * st[2 * h + 1];
+  scores[r] = acc / (float)n_heads;
+}
+
+// ------------------------------------------------------------------------------------------ select
+constexpr int SEL_THREADS = 1024;
+
+__device__ __forceinline__ uint32_t score_key(float s) {
+  uint32_t u = __float_as_uint(s);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // monotone for every finite float
+}
+
+// Exclusive prefix of `flag` over the CTA in thread order; total returned through *total.
+__device__ __forceinline__ int block_excl_scan(int flag, int *warp_tot /*[32]*/, int *total) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t b = __ballot_sync(0xffffffffu, flag);
+  const int within = __popc(b & ((1u << lane) - 1u));
+  __syncthreads();  // warp_tot may still be read from the previous scan
+  if (lane == 0) warp_tot[warp] = __popc(b);
+  __syncthreads();
+  int before = 0, tot = 0;
+  for (int w = 0; w < SEL_THREADS / 32; ++w) {
+    const int c = warp_tot[w];
+    if (w < warp) before += c;
+    tot += c;
+  }
+  *total = tot;
+  return before + within;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_in,
+              const int32_t *__restrict__ cu_keep, int32_t *__restrict__ keep_idx,
+              int32_t *__restrict__ drop_idx, DevStatus *status) {
+  const int seq = blockIdx.x;
+  const int in0 = cu_in[seq], n = cu_in[seq + 1] - in0;
+  const int k0 = cu_keep[seq], n_keep = cu_keep[seq + 1] - k0;
+  const int d0 = in0 - k0;
+  if (n == 0) return;
+  if (n_keep < 1 || n_keep > n) {
+    if (threadIdx.x == 0) dev_fail(status, LAZY_E_BADARG, W_SELECT, seq, n_keep);
+    return;
+  }
+  const float *s = scores + in0;
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_k;
+
+  // ---- radix select of the n_keep-th largest key
+  uint32_t prefix = 0, mask = 0;
+  int k = n_keep;  // still looking for the k-th largest among keys matching `prefix` under `mask`
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += SEL_THREADS) {
+      const uint32_t key = (i == n - 1) ? 0xffffffffu : score_key(s[i]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int above = 0, b = 255;
+      for (; b > 0; --b) {
+        if (above + hist[b] >= k) break;
+        above += hist[b];
+      }
+      sh_prefix = prefix | ((uint32_t)b << shift);
+      sh_k = k - above;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    k = sh_k;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t tau = prefix;  // key of the n_keep-th largest; k = how many keys == tau to keep
+
+  // ---- emit in index order
+  int kept_so_far = 0, eq_so_far = 0;
+  for (int base = 0; base < n; base += SEL_THREADS) {
+    const int i = base + threadIdx.x;
+    uint32_t key = 0;
+    const bool valid = i < n;
+    if (valid) key = (i == n - 1) ? 0xffffffffu : score_key(s[i]);
+    const int is_eq = valid && key == tau;
+    int eq_total;
+    const int eq_rank = eq_so_far + block_excl_scan(is_eq, warp_tot, &eq_total);
+    const int keep = valid && (key > tau || (is_eq && eq_rank < k));
+    int keep_total;
+    const int keep_rank = kept_so_far + block_excl_scan(keep, warp_tot, &keep_total);
+    if (valid) {
+      if (keep) keep_idx[k0 + keep_rank] = in0 + i;
+      else drop_idx[d0 + (i - keep_rank)] = in0 + i;
+    }
+    eq_so_far += eq_total;
+    kept_so_far += keep_total;
+  }
+  if (threadIdx.x == 0 && kept_so_far != n_keep) dev_fail(status, LAZY_E_STATE, W_SELECT, seq, kept_so_far);
+}
+
+__global__ void forced_scores_kernel(const int32_t *__restrict__ pos, int r0, int n,
+                                     const int32_t *__restrict__ forced, int n_forced,
+                                     float *__restrict__ scores) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int p = pos[r0 + i];
+  int lo = 0, hi = n_forced;  // first index with forced[idx] >= p
+  while (lo < hi) {
+    int mid = (lo + hi) >> 1;
+    if (forced[mid] < p) lo = mid + 1; else hi = mid;
+  }
+  scores[r0 + i] = (lo < n_forced && forced[lo] == p) ? 2.f : 0.f;
+}
+
+}  // namespace
+
+size_t score_scratch_floats(int n_seqs, int n_total, int n_heads) {
+  return (size_t)n_heads * n_total + (size_t)2 * n_heads * n_seqs;
+}
+
+int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
+                 const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
+                 int n_heads, int head_dim, float *scratch, float *scores) {
+  if (n_total == 0 || n_seqs == 0) return LAZY_OK;
+  const int V = dtype == LAZY_F32 ? 4 : 8;
+  const int lpk = head_dim / V;
+  if (head_dim % V || lpk < 1 || lpk > 32 || (lpk & (lpk - 1))) return LAZY_E_BADARG;
+  float *logits = scratch;
+  float *stats = scratch + (size_t)n_heads * n_total;
+  const int threads = 256;
+  const int keys_per_block = (threads / 32) * (32 / lpk) * 4;
+  dim3 grid(cdiv(max_len, keys_per_block), n_heads, n_seqs);
+  if (dtype == LAZY_F32)
+    score_logits_kernel<float><<<grid, threads, 0, st>>>((const float *)q, ldq, (const float *)k, ldkv,
+                                                         cu_q, kv_base, n_total, head_dim, logits);
+  else
+    score_logits_kernel<bf16><<<grid, threads, 0, st>>>((const bf16 *)q, ldq, (const bf16 *)k, ldkv,
+                                                        cu_q, kv_base, n_total, head_dim, logits);
+  LAZY_COUNT_LAUNCH();
+  score_stats_kernel<<<dim3(n_heads, n_seqs), 256, 0, st>>>(logits, cu_q, n_total, n_heads, stats);
+  LAZY_COUNT_LAUNCH();
+  score_mean_kernel<<<cdiv(n_total, 256), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
+                                                        scores);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
+                  const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
+                  DevStatus *status) {
+  if (n_seqs == 0) return LAZY_OK;
+  select_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, cu_keep, keep_idx, drop_idx, status);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+int launch_forced_scores(cudaStream_t st, const int32_t *pos, int r0, int n, const int32_t *forced,
+                         int n_forced, float *scores) {
+  if (n == 0) return LAZY_OK;
+  forced_scores_kernel<<<cdiv(n, 256), 256, 0, st>>>(pos, r0, n, forced, n_forced, scores);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+}  // namespace lazy
