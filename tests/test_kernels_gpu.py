@@ -1,0 +1,222 @@
+"""Per-kernel parity: each step of the path, called through the C ABI, against the CPU oracle's
+definition of that step on the same seeded inputs.
+
+Tolerances (per-tensor max|a-b| <= tol * max|b|): bf16 2e-2 is the bound for hidden states and
+logits over a whole layer stack; a single step rounds once, so single steps are held to 1e-2;
+fp32 mode 1e-4; Eq. 1 scores 1e-3 absolute; indices bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import lazyllm_oracle as O
+from paper_2407_14057_b200 import binding as B
+from paper_2407_14057_b200 import build, synth
+from helpers import rel_err, to_np
+
+pytestmark = pytest.mark.gpu
+
+BF16_STEP_TOL = 1e-2
+F32_TOL = 1e-4
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.lib()
+    yield
+    B.lazy_device_status()
+
+
+def _rand(shape, seed, dtype, std=1.0):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(shape, generator=g, dtype=torch.float32) * std).to(dtype)
+
+
+def _tol(dtype):
+    return F32_TOL if dtype == torch.float32 else BF16_STEP_TOL
+
+
+# ------------------------------------------------------------------------------------------ rmsnorm
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n,d", [(1, 256), (37, 256), (300, 4096)])
+def test_rmsnorm(dtype, n, d):
+    x = _rand((n, d), 1, dtype, 3.0)
+    g = (1 + 0.1 * _rand((d,), 2, torch.float32)).to(dtype)
+    y = B.lazy_k_rmsnorm(x.cuda(), g.cuda(), 1e-6)
+    ref = O.rmsnorm(to_np(x), to_np(g), 1e-6)
+    assert rel_err(to_np(y), ref) < _tol(dtype)
+
+
+# ------------------------------------------------------------------------------------------ GEMM
+GEMM_SHAPES = [(128, 256, 64), (1, 256, 64), (300, 512, 320), (257, 1376, 688), (129, 768, 256),
+               (1000, 4096, 4096)]
+
+
+@pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("residual", [False, True])
+def test_gemm_bf16_tensor_core(M, N, K, residual):
+    A = _rand((M, K), 3, torch.bfloat16)
+    Bm = _rand((N, K), 4, torch.bfloat16, 0.05)
+    R = _rand((M, N), 5, torch.bfloat16) if residual else None
+    out = B.lazy_k_gemm(A.cuda(), Bm.cuda(), None if R is None else R.cuda())
+    B.lazy_device_status()
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T
+    if residual:
+        ref = ref + O.f64(to_np(R))
+    assert rel_err(to_np(out), ref) < BF16_STEP_TOL
+    # element-wise: bf16 rounding of the exact value, plus fp32 accumulation noise
+    err = np.abs(to_np(out).astype(np.float64) - ref)
+    assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-3 * np.max(np.abs(ref)))
+
+
+def test_gemm_bf16_in_place_residual_and_cuda_core_cross_check():
+    M, N, K = 200, 512, 1408
+    A = _rand((M, K), 6, torch.bfloat16).cuda()
+    Bm = _rand((N, K), 7, torch.bfloat16, 0.05).cuda()
+    x = _rand((M, N), 8, torch.bfloat16).cuda()
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(x))
+    simt = B.lazy_k_gemm(A, Bm, x, impl=1)
+    B.lazy_k_gemm(A, Bm, x, out=x)          # x += A B^T in place
+    B.lazy_device_status()
+    assert rel_err(to_np(x), ref) < BF16_STEP_TOL
+    assert rel_err(to_np(simt), ref) < BF16_STEP_TOL
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 256, 64), (70, 688, 256), (33, 256, 688)])
+def test_gemm_fp32(M, N, K):
+    A = _rand((M, K), 9, torch.float32)
+    Bm = _rand((N, K), 10, torch.float32, 0.05)
+    R = _rand((M, N), 11, torch.float32)
+    out = B.lazy_k_gemm(A.cuda(), Bm.cuda(), R.cuda())
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(R))
+    assert rel_err(to_np(out), ref) < F32_TOL
+
+
+@pytest.mark.parametrize("dtype,M,F,K", [(torch.bfloat16, 300, 1408, 512), (torch.bfloat16, 128, 128, 64),
+                                         (torch.bfloat16, 77, 688, 256), (torch.bfloat16, 500, 11008, 4096),
+                                         (torch.float32, 70, 688, 256)])
+def test_gemm_swiglu(dtype, M, F, K):
+    A = _rand((M, K), 12, dtype)
+    Bg = _rand((F, K), 13, dtype, 0.05)
+    Bu = _rand((F, K), 14, dtype, 0.05)
+    out = B.lazy_k_gemm_swiglu(A.cuda(), Bg.cuda(), Bu.cuda())
+    B.lazy_device_status()
+    a = O.f64(to_np(A))
+    ref = O.silu(a @ O.f64(to_np(Bg)).T) * (a @ O.f64(to_np(Bu)).T)
+    assert rel_err(to_np(out), ref) < _tol(dtype)
+
+
+def test_gemm_empty_rows_is_a_no_op():
+    A = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    Bm = _rand((256, 64), 1, torch.bfloat16).cuda()
+    assert B.lazy_k_gemm(A, Bm).shape == (0, 256)
+
+
+# ------------------------------------------------------------------------------------------ RoPE
+@pytest.mark.parametrize("dtype,H,dh", [(torch.float32, 4, 64), (torch.bfloat16, 4, 128)])
+def test_rope_and_kv_write(dtype, H, dh):
+    n, d = 50, H * dh
+    qkv = _rand((n, 3 * d), 15, dtype)
+    pos = torch.tensor(sorted(np.random.default_rng(0).choice(4000, n, replace=False)), dtype=torch.int32)
+    dev = qkv.cuda()
+    kc, vc = B.lazy_k_rope_kv(dev, pos.cuda(), H, dh, 4096, 1e4)
+    B.lazy_device_status()
+    x = to_np(qkv)
+    q_ref = O.rope(x[:, :d].reshape(n, H, dh), to_np(pos), 1e4).reshape(n, d)
+    k_ref = O.rope(x[:, d:2 * d].reshape(n, H, dh), to_np(pos), 1e4).reshape(n, d)
+    got = to_np(dev)
+    assert rel_err(got[:, :d], q_ref) < _tol(dtype)
+    assert rel_err(to_np(kc), k_ref) < _tol(dtype)
+    assert np.array_equal(to_np(vc), x[:, 2 * d:])           # v is a plain copy
+    assert np.array_equal(got[:, 2 * d:], x[:, 2 * d:])
+
+
+# ------------------------------------------------------------------------------------------ attention
+def _attention_case(dtype, H, dh, lengths, seed):
+    n = sum(lengths)
+    d = H * dh
+    q = _rand((n, d), seed, dtype)
+    k = _rand((n, d), seed + 1, dtype)
+    v = _rand((n, d), seed + 2, dtype)
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    o = B.lazy_k_attention(q.cuda(), d, k.cuda(), v.cuda(), d, torch.tensor(cu).cuda(), max(lengths), n, H, dh)
+    s = B.lazy_k_score(q.cuda(), d, k.cuda(), d, torch.tensor(cu).cuda(), n, H, dh)
+    B.lazy_device_status()
+    o_ref = np.zeros((n, d))
+    s_ref = np.zeros(n)
+    for a, b in zip(cu[:-1], cu[1:]):
+        pos = np.arange(b - a)
+        oo, ss = O.attend(to_np(q)[a:b].reshape(-1, H, dh), to_np(k)[a:b].reshape(-1, H, dh),
+                          to_np(v)[a:b].reshape(-1, H, dh), pos, pos, -1)
+        o_ref[a:b], s_ref[a:b] = oo, ss
+    return to_np(o), o_ref, to_np(s), s_ref, cu
+
+
+@pytest.mark.parametrize("dtype,H,dh,lengths", [
+    (torch.float32, 4, 64, [70]), (torch.float32, 2, 64, [1, 33, 5]),
+    (torch.bfloat16, 4, 128, [1]), (torch.bfloat16, 4, 128, [64]), (torch.bfloat16, 3, 128, [200]),
+    (torch.bfloat16, 2, 128, [65, 1, 130, 17]), (torch.bfloat16, 2, 128, [513]),
+    (torch.bfloat16, 4, 64, [45]),
+])
+def test_attention_and_score(dtype, H, dh, lengths):
+    o, o_ref, s, s_ref, cu = _attention_case(dtype, H, dh, lengths, 20)
+    assert rel_err(o, o_ref) < _tol(dtype)
+    assert np.max(np.abs(s - s_ref)) < 1e-3
+    assert np.max(np.abs(s - s_ref) / s_ref.clip(1e-12)) < (1e-4 if dtype == torch.float32 else 2e-2)
+    for a, b in zip(cu[:-1], cu[1:]):
+        assert abs(s[a:b].sum() - 1) < 1e-4
+
+
+# ------------------------------------------------------------------------------------------ select
+def _select_case(score_list, keep_list):
+    cu_in = np.concatenate([[0], np.cumsum([len(s) for s in score_list])]).astype(np.int32)
+    cu_keep = np.concatenate([[0], np.cumsum(keep_list)]).astype(np.int32)
+    scores = torch.cat(score_list)
+    keep, drop = B.lazy_k_select(scores.cuda(), torch.tensor(cu_in).cuda(), torch.tensor(cu_keep).cuda())
+    B.lazy_device_status()
+    keep, drop = to_np(keep), to_np(drop)
+    for s in range(len(score_list)):
+        n = len(score_list[s])
+        k_ref, d_ref = O.select_top(score_list[s].numpy(), keep_list[s], n - 1)
+        got_k = keep[cu_keep[s]:cu_keep[s + 1]] - cu_in[s]
+        d0 = cu_in[s] - cu_keep[s]
+        got_d = drop[d0:d0 + n - keep_list[s]] - cu_in[s]
+        assert np.array_equal(got_k, k_ref), (s, n, keep_list[s])
+        assert np.array_equal(got_d, d_ref)
+
+
+@pytest.mark.parametrize("kind", ["random", "uniform", "zeros", "duplicates", "lognormal"])
+@pytest.mark.parametrize("n", [1, 2, 127, 128, 129, 1025, 3376, 4096, 65536])
+def test_select_bit_exact(kind, n):
+    s = synth.make_scores(n, kind, seed=n)
+    for n_keep in sorted({1, max(1, (n * 3 + 9) // 10), max(1, (n * 7 + 9) // 10), n}):
+        _select_case([s], [n_keep])
+
+
+def test_select_per_sequence_batch():
+    lens = [5, 1, 300, 2049, 64]
+    scores = [synth.make_scores(n, k, seed=i) for i, (n, k) in
+              enumerate(zip(lens, ["duplicates", "random", "zeros", "lognormal", "uniform"]))]
+    _select_case(scores, [3, 1, 150, 615, 64])
+
+
+# ------------------------------------------------------------------------------------------ gather
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 4096), (torch.float32, 256)])
+def test_gather_rows_is_an_exact_copy(dtype, d):
+    src = _rand((500, d), 30, dtype)
+    idx = torch.tensor(sorted(np.random.default_rng(1).choice(500, 301, replace=False)), dtype=torch.int32)
+    out = B.lazy_k_gather_rows(src.cuda(), idx.cuda())
+    B.lazy_device_status()
+    assert torch.equal(out.cpu(), src[idx.long()])
+    assert B.lazy_k_gather_rows(src.cuda(), idx[:0].cuda()).shape[0] == 0
+
+
+def test_gather_rows_reports_a_bad_index_instead_of_reading_it():
+    src = _rand((10, 64), 31, torch.bfloat16).cuda()
+    idx = torch.tensor([0, 3, 10], dtype=torch.int32).cuda()      # 10 is out of range
+    B.lazy_k_gather_rows(src, idx)
+    with pytest.raises(B.LazyError) as e:
+        B.lazy_device_status()
+    assert e.value.status == -1
+    B.lazy_device_status()                                          # cleared

@@ -1,0 +1,278 @@
+"""End-to-end parity of the token-pruned prefill (and the single-layer pruning op) against the
+CPU oracle, through the C ABI.
+
+Protocol.  The GPU run selects its own kept sets.  (1) Scores are compared directly wherever both
+sides still hold the same rows; (2) a kept-set difference is accepted only for tokens whose oracle
+score lies within the band of the threshold (1e-3 absolute as the stated bound, and a relative
+band that is not vacuous at long prompts); (3) because one flipped token changes every deeper
+tensor, hidden states, caches and logits are compared with the oracle re-run on the GPU's kept
+sets (forced replay); (4) the GPU is also re-run on the oracle's kept sets.
+Tolerances: per-tensor max|a-b| <= tol*max|b| with tol 2e-2 (bf16) / 1e-4 (fp32); scores 1e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+import lazyllm_oracle as O
+from paper_2407_14057_b200 import binding as B
+from paper_2407_14057_b200 import build, synth
+from helpers import rel_err, to_np, weights_to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.lib()
+
+
+def _to_cuda(W):
+    out = {k: v.cuda() for k, v in W.items() if k != "layers"}
+    out["layers"] = [{k: v.cuda() for k, v in lw.items()} for lw in W["layers"]]
+    return out
+
+
+def _tols(dtype):
+    return (1e-4, 1e-5) if dtype == torch.float32 else (2e-2, 3e-2)   # tensor tol, relative score band
+
+
+def _check_set_difference(gpu_pos, ref_pos, ref_scores, ref_score_pos, band_rel):
+    """Tokens kept by one side only must sit at the threshold."""
+    g, r = set(gpu_pos.tolist()), set(ref_pos.tolist())
+    assert len(g) == len(r)
+    diff = g ^ r
+    if not diff:
+        return 0
+    s_of = dict(zip(ref_score_pos.tolist(), ref_scores.tolist()))
+    last = int(ref_score_pos[-1])
+    tau = min(s_of[p] for p in r if p != last)
+    for p in diff:
+        assert abs(s_of[p] - tau) <= 1e-3, (p, s_of[p], tau)
+        assert abs(s_of[p] - tau) <= band_rel * tau, (p, s_of[p], tau)
+    return len(diff)
+
+
+def run_model_case(shape, schedule, lengths, dtype, seed, perturb=True, max_new=0):
+    bf16 = dtype == torch.bfloat16
+    tol, band = _tols(dtype)
+    W = synth.make_weights(shape, seed, bf16=bf16)
+    if perturb:
+        synth.perturb_gains(W, seed + 100)
+    Wn = weights_to_np(W)
+    ids, cu = synth.make_varlen_batch(shape.vocab, lengths, seed + 1)
+    n_seqs = len(lengths)
+    eng = B.LazyPrefill(shape, _to_cuda(W), schedule, dtype, max_seqs=n_seqs,
+                        max_prompt_tokens=sum(lengths), max_new_tokens=max_new, debug_capture=True)
+    logits = torch.empty((n_seqs, shape.vocab), dtype=torch.float32, device="cuda")
+    d_ids = ids.cuda()
+    eng.lazy_prefill_run(d_ids, cu, logits)
+    eng.lazy_sync_status()
+    stats = eng.lazy_get_stats()
+    points = [e for e, _ in schedule]
+    flips = 0
+    hidden = [to_np(eng.lazy_get_hidden(l)) for l in range(shape.n_layers)]
+    row_off = [0] * shape.n_layers
+    for s in range(n_seqs):
+        sid = to_np(ids)[cu[s]:cu[s + 1]]
+        free = O.prefill(shape, Wn, sid, schedule)
+        gpu_kept = {e: to_np(eng.lazy_get_kept(e, s)).astype(np.int64) for e in points}
+        # (1) scores before the first cut see identical rows on both sides
+        first = points[0] if points else shape.n_layers
+        for l in range(first):
+            sc = to_np(eng.lazy_get_scores(l, s))
+            assert np.max(np.abs(sc - free.scores[l])) < 1e-3
+            assert abs(sc.sum() - 1.0) < 1e-3 and sc.min() >= 0
+        # (2)+(3) walk the cuts: compare against the oracle replayed on the GPU's sets so far
+        replay = O.prefill(shape, Wn, sid, schedule, forced_keep=gpu_kept)
+        prev = None
+        for e in points:
+            partial = {k: v for k, v in gpu_kept.items() if k < e}
+            ref = O.prefill(shape, Wn, sid, schedule, forced_keep=partial) if partial else free
+            flips += _check_set_difference(gpu_kept[e], ref.kept_pos[e], ref.scores[e - 1],
+                                           ref.score_pos[e - 1], band)
+            assert np.all(np.diff(gpu_kept[e]) > 0) and gpu_kept[e][-1] == len(sid) - 1
+            if prev is not None:
+                assert set(gpu_kept[e].tolist()) <= set(prev.tolist())       # subset property
+            prev = gpu_kept[e]
+        for l in range(shape.n_layers):
+            sc = to_np(eng.lazy_get_scores(l, s))
+            assert sc.shape == replay.scores[l].shape
+            assert np.max(np.abs(sc - replay.scores[l])) < 1e-3
+            n_l = replay.hidden_out[l].shape[0]
+            got = hidden[l][row_off[l]:row_off[l] + n_l]
+            row_off[l] += n_l
+            assert rel_err(got, replay.hidden_out[l]) < tol, (l, rel_err(got, replay.hidden_out[l]))
+            kpos, kk, vv = eng.lazy_get_kv(l, s)
+            assert np.array_equal(to_np(kpos), replay.rows_pos[l])
+            kr, vr = replay.layers[l].rows(replay.rows_pos[l])
+            assert rel_err(to_np(kk), kr.reshape(len(kpos), -1)) < tol
+            assert rel_err(to_np(vv), vr.reshape(len(kpos), -1)) < tol
+            apos, ahid = eng.lazy_get_aux(l, s)
+            want = sorted(replay.layers[l].aux.keys())
+            assert to_np(apos).tolist() == want
+            if want:
+                ref_rows = np.stack([replay.layers[l].aux[p] for p in want])
+                assert rel_err(to_np(ahid), ref_rows) < tol
+                rev = eng.aux_cache_revive(l, s, apos[: min(5, len(want))].contiguous())
+                assert torch.equal(rev, ahid[: min(5, len(want))])
+        assert rel_err(to_np(logits[s]), replay.logits) < tol
+        # (4) GPU on the oracle's own kept sets
+        for e in points:
+            eng.lazy_set_forced_keep(e, s, torch.tensor(free.kept_pos[e], dtype=torch.int32).cuda())
+    if points:
+        logits2 = torch.empty_like(logits)
+        eng.lazy_prefill_run(d_ids, cu, logits2)
+        eng.lazy_sync_status()
+        for s in range(n_seqs):
+            free = O.prefill(shape, Wn, to_np(ids)[cu[s]:cu[s + 1]], schedule)
+            for e in points:
+                assert np.array_equal(to_np(eng.lazy_get_kept(e, s)), free.kept_pos[e])
+            assert rel_err(to_np(logits2[s]), free.logits) < tol
+            assert int(torch.argmax(logits2[s])) == O.greedy(free.logits) or bf16
+    assert stats.kernel_launches > 0
+    eng.close()
+    return flips
+
+
+def test_tiny_fp32_config():
+    """2 layers, d=256, 4x64 heads, ffn 688, vocab 1024, one 256-token prompt, keep 50 % entering
+    layer 1, next-token logits; fp32 mode."""
+    flips = run_model_case(synth.TINY, synth.SCHEDULE_TINY, [256], torch.float32, seed=0, perturb=False)
+    assert flips == 0
+
+
+def test_tiny_fp32_three_cuts_and_ragged_lengths():
+    shape = synth.TINY.with_layers(4)
+    run_model_case(shape, ((1, 7000), (2, 5000), (3, 3000)), [129], torch.float32, seed=3)
+
+
+def test_fp32_varlen_batch():
+    shape = synth.TINY.with_layers(3)
+    run_model_case(shape, ((1, 6000), (2, 2500)), [70, 1, 33, 150], torch.float32, seed=4)
+
+
+def test_full_keep_schedule_is_standard_prefill():
+    shape = synth.TINY
+    W = synth.make_weights(shape, 7, bf16=False)
+    ids = synth.make_prompt(shape.vocab, 100, 8)
+    out = []
+    for sched in ((), ((1, 10000),)):
+        eng = B.LazyPrefill(shape, _to_cuda(W), sched, torch.float32, 1, 100)
+        lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+        eng.lazy_prefill_run(ids.cuda(), [0, 100], lg)
+        eng.lazy_sync_status()
+        out.append(lg.cpu())
+        eng.close()
+    assert torch.equal(out[0], out[1])
+    ref = O.prefill(shape, weights_to_np(W), to_np(ids), ())
+    assert rel_err(to_np(out[0][0]), ref.logits) < 1e-4
+
+
+def test_small_bf16_model_multi_tile():
+    """head_dim 128 model on the tensor-core kernels: 300 rows = several GEMM and attention tiles
+    with ragged tails, three cuts."""
+    run_model_case(synth.SMALL, ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16, seed=5)
+
+
+def test_small_bf16_varlen_batch():
+    run_model_case(synth.SMALL.with_layers(3), ((1, 6000), (2, 3000)), [200, 65, 1, 131], torch.bfloat16, seed=6)
+
+
+def test_capacity_and_argument_errors():
+    shape = synth.TINY
+    W = _to_cuda(synth.make_weights(shape, 1, bf16=False))
+    eng = B.LazyPrefill(shape, W, synth.SCHEDULE_TINY, torch.float32, 1, 64)
+    lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+    ids = synth.make_prompt(shape.vocab, 65, 1).cuda()
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_prefill_run(ids, [0, 65], lg)
+    assert e.value.status == -3
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_prefill_run(ids, [0, 10, 20], lg)                    # two sequences, room for one
+    assert e.value.status == -3
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_get_kept(1, 0)                                       # nothing has run yet
+    assert e.value.status == -7
+    bad = ids.clone()
+    bad[3] = shape.vocab + 5                                          # id out of range: reported
+    eng.lazy_prefill_run(bad[:64].contiguous(), [0, 64], lg)
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_sync_status()
+    assert e.value.status == -1
+    eng.lazy_prefill_run(ids[:64].contiguous(), [0, 64], lg)
+    eng.lazy_sync_status()
+    pos, _ = eng.lazy_get_aux(0, 0)
+    kept = eng.lazy_get_kept(1, 0)
+    with pytest.raises(B.LazyError) as e:
+        eng.aux_cache_revive(0, 0, kept[:1].contiguous())             # a kept token is not in Aux
+    assert e.value.status == -4
+    assert eng.aux_cache_revive(0, 0, pos[:3].contiguous()).shape == (3, shape.d_model)
+    eng.close()
+
+
+# ------------------------------------------------------------------------------------------ prune op
+def _prune_case(dtype, n, H, dh, keep_bp, seed, pos=None):
+    d = H * dh
+    bf16 = dtype == torch.bfloat16
+    tol, band = _tols(dtype)
+    shape = synth.ModelShape(1, d, H, dh, 8, 8)
+    g = torch.Generator().manual_seed(seed)
+    lw = {"w_qkv": torch.empty(3 * d, d).normal_(0, 0.02, generator=g).to(dtype),
+          "w_o": torch.empty(d, d).normal_(0, 0.02, generator=g).to(dtype),
+          "g_attn": torch.ones(d, dtype=dtype)}
+    x = synth.make_hidden(n, d, seed + 1, bf16)
+    pos = torch.arange(n, dtype=torch.int32) if pos is None else pos
+    max_pos = int(pos.max()) + 1
+    out = B.lazy_prune_op(x.cuda(), pos.cuda(), lw["w_qkv"].cuda(), lw["w_o"].cuda(), lw["g_attn"].cuda(),
+                          H, dh, keep_bp, max_pos)
+    B.lazy_device_status()
+    lwn = {k: to_np(v) for k, v in lw.items()}
+    ref = O.prune_op(shape, lwn, to_np(x), to_np(pos), keep_bp)
+    sc = to_np(out["scores"])
+    assert np.max(np.abs(sc - ref["scores"])) < 1e-3
+    assert np.max(np.abs(sc - ref["scores"]) / ref["scores"].clip(1e-30)) < band
+    keep = to_np(out["keep_idx"]).astype(np.int64)
+    drop = to_np(out["drop_idx"]).astype(np.int64)[: out["n_drop"]]
+    assert len(keep) == len(ref["keep"]) and keep[-1] == n - 1
+    assert sorted(keep.tolist() + drop.tolist()) == list(range(n))
+    flips = _check_set_difference(keep, ref["keep"], ref["scores"], np.arange(n), band)
+    # the selection itself is bit-exact given the GPU's own scores
+    k2, d2 = O.select_top(sc, len(keep), n - 1)
+    assert np.array_equal(keep, k2) and np.array_equal(drop, d2)
+    rep = O.prune_op(shape, lwn, to_np(x), to_np(pos), keep_bp, forced_keep_rows=keep)
+    assert rel_err(to_np(out["hidden_kept"]), rep["hidden_kept"]) < tol
+    assert rel_err(to_np(out["k_kept"]), rep["k_kept"].reshape(len(keep), d)) < tol
+    assert rel_err(to_np(out["v_kept"]), rep["v_kept"].reshape(len(keep), d)) < tol
+    assert np.array_equal(to_np(out["pos_kept"]), rep["pos_kept"])
+    if out["n_drop"]:
+        assert rel_err(to_np(out["aux_hidden"])[: out["n_drop"]], rep["aux_rows"]) < tol
+        assert np.array_equal(to_np(out["aux_pos"])[: out["n_drop"]], rep["aux_pos"])
+    # GPU forced onto the oracle's set: gathered rows are exact copies of rows the op itself made
+    forced = B.lazy_prune_op(x.cuda(), pos.cuda(), lw["w_qkv"].cuda(), lw["w_o"].cuda(), lw["g_attn"].cuda(),
+                             H, dh, keep_bp, max_pos,
+                             forced_keep_idx=torch.tensor(ref["keep"], dtype=torch.int32).cuda())
+    B.lazy_device_status()
+    assert np.array_equal(to_np(forced["keep_idx"]), ref["keep"])
+    assert rel_err(to_np(forced["hidden_kept"]), ref["hidden_kept"]) < tol
+    return flips
+
+
+def test_prune_op_fp32_small():
+    assert _prune_case(torch.float32, 200, 4, 64, 6000, seed=1) == 0
+
+
+def test_prune_op_bf16_multi_tile_with_position_gaps():
+    pos = torch.tensor(sorted(np.random.default_rng(3).choice(5000, 700, replace=False)), dtype=torch.int32)
+    _prune_case(torch.bfloat16, 700, 4, 128, 6000, seed=2, pos=pos)
+
+
+def test_prune_op_keep_everything_and_keep_one():
+    _prune_case(torch.float32, 64, 4, 64, 10000, seed=4)
+    _prune_case(torch.float32, 64, 4, 64, 1, seed=5)
+
+
+def test_prune_op_full_size_bf16():
+    """The single-layer pruning op at its full size: hidden [4096, 4096], 32 heads x 128, keep 60 %
+    (2458 kept / 1638 to the Aux Cache)."""
+    _prune_case(torch.bfloat16, 4096, 32, 128, 6000, seed=1)
