@@ -17,7 +17,9 @@ int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, vo
 
 int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B, const void *R,
                 void *C, int32_t M, int32_t N, int32_t K) {
-  if (bad_dtype(dtype) || !A || !B || !C || M < 0 || N < 1 || K < 1 || N % 8 || K % 8) return LAZY_E_BADARG;
+  if (bad_dtype(dtype) || M < 0 || N < 1 || K < 1 || N % 8 || K % 8) return LAZY_E_BADARG;
+  if (M == 0) return LAZY_OK;  // nothing to compute; an empty matrix may have no address
+  if (!A || !B || !C) return LAZY_E_BADARG;
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, B, nullptr, R, C, M, N, K, 0);
@@ -26,8 +28,9 @@ int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const 
 
 int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
                        const void *Bu, void *C, int32_t M, int32_t F, int32_t K) {
-  if (bad_dtype(dtype) || !A || !Bg || !Bu || !C || M < 0 || F < 1 || K < 1 || F % 8 || K % 8)
-    return LAZY_E_BADARG;
+  if (bad_dtype(dtype) || M < 0 || F < 1 || K < 1 || F % 8 || K % 8) return LAZY_E_BADARG;
+  if (M == 0) return LAZY_OK;
+  if (!A || !Bg || !Bu || !C) return LAZY_E_BADARG;
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
@@ -85,7 +88,9 @@ int lazy_k_select(void *stream, const float *scores, const int32_t *d_cu_in, con
 
 int lazy_k_gather_rows(void *stream, const void *src, const int32_t *idx, void *dst, int32_t n,
                        int32_t row_bytes, int32_t src_rows) {
-  if (!src || !dst || n < 0 || row_bytes < 16 || row_bytes % 16 || src_rows < 0) return LAZY_E_BADARG;
+  if (n < 0 || row_bytes < 16 || row_bytes % 16 || src_rows < 0) return LAZY_E_BADARG;
+  if (n == 0) return LAZY_OK;
+  if (!src || !dst) return LAZY_E_BADARG;
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   return launch_gather_rows((cudaStream_t)stream, src, idx, dst, n, row_bytes, src_rows, status);
