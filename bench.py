@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the token-pruned prefill on the Llama-2-7B shape.
+
+One "step" = one whole prefill (every layer, every pruning point, first-token logits) of one
+3376-token synthetic prompt with cumulative keep 100/70/50/30 % entering layers 0/8/16/24.
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of the
+same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+N_PROMPT = 3376
+METRIC = "prefill tokens/s (TTFT), 7B-shape 3376-token prompt, token-pruned"
+UNIT = "tokens/s"
+WORKLOAD = ("llama2-7b-shape prefill (32 layers, d=4096, 32x128 heads, ffn 11008, vocab 32000), batch 1, "
+            "3376-token prompt, keep 100/70/50/30% entering layers 0/8/16/24")
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle leg
+def _rows_per_layer(n_layers, schedule, n):
+    """(rows in attention, rows in MLP) of every layer under a schedule of (layer_entered, bp)."""
+    pts = dict(schedule)
+    rows, out = n, []
+    for l in range(n_layers):
+        n_attn = rows
+        if (l + 1) in pts:
+            rows = max(1, min(rows, (n * pts[l + 1] + 9999) // 10000))
+        out.append((n_attn, rows))
+    return out
+
+
+def _algorithmic_flops(shape, schedule, n):
+    d, F = shape.d_model, shape.d_ffn
+    tot = 0.0
+    for n_attn, n_mlp in _rows_per_layer(shape.n_layers, schedule, n):
+        tot += n_attn * (2.0 * 3 * d * d + 2.0 * d * d) + 2.0 * d * n_attn * (n_attn + 1.0) + n_mlp * 6.0 * d * F
+    return tot + 2.0 * d * shape.vocab
+
+
+class OracleSample:
+    """The CPU oracle on a bounded sample of the workload: a shallow stack of the 7B widths that
+    visits the same row counts (4 layers, cuts entering layers 1/2/3: 3376/2364/1688/1013 rows; or
+    2 layers, 3376 -> 1013 rows, when many steps are asked for).  The whole-prompt time is taken as
+    the sample's time scaled by the ratio of algorithmic FLOPs (32-layer workload / sample)."""
+
+    def __init__(self, n_prompt: int, small: bool):
+        import torch  # noqa: F401
+        sys.path.insert(0, os.path.join(ROOT, "oracle"))
+        import lazyllm_oracle as O
+        from paper_2407_14057_b200 import synth
+        self.O = O
+        self.n = n_prompt
+        if small:
+            self.shape, self.schedule = synth.LLAMA7B.with_layers(2), ((1, 3000),)
+        else:
+            self.shape, self.schedule = synth.LLAMA7B.with_layers(4), ((1, 7000), (2, 5000), (3, 3000))
+        W = synth.make_weights(self.shape, 0, bf16=True)
+        self.W = {k: v.float().numpy() for k, v in W.items() if k != "layers"}
+        self.W["layers"] = [{k: v.float().numpy() for k, v in lw.items()} for lw in W["layers"]]
+        self.ids = synth.make_prompt(self.shape.vocab, n_prompt, 1).numpy()
+        self.scale = (_algorithmic_flops(synth.LLAMA7B, synth.SCHEDULE_7B, n_prompt)
+                      / _algorithmic_flops(self.shape, self.schedule, n_prompt))
+        self.cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+        try:
+            from threadpoolctl import threadpool_info
+            nt = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+            if nt:
+                self.cores = min(self.cores, max(nt))
+        except Exception:
+            pass
+        rows = "/".join(str(r) for r, _ in _rows_per_layer(self.shape.n_layers, self.schedule, n_prompt))
+        self.sample = (f"{self.shape.n_layers} of 32 layers at 7B widths, one layer per visited segment "
+                       f"({rows} rows), fp64 numpy oracle; whole-prompt time = sample time x "
+                       f"{self.scale:.2f} (ratio of algorithmic FLOPs)")
+
+    def step_seconds(self) -> float:
+        t0 = time.perf_counter()
+        self.O.prefill(self.shape, self.W, self.ids, self.schedule, keep_records=False)
+        return (time.perf_counter() - t0) * self.scale
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(args.prompt, small=(args.steps + args.warmup) > 13)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = smp.step_seconds()
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * sum(times) / len(times)
+    value = args.prompt / (ms / 1e3)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": WORKLOAD, "batch": 1, "seq_len": args.prompt},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                            "sample": smp.sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU leg
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_14057_b200 import binding as B
+    from paper_2407_14057_b200 import build, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    B.lib()
+    peaks = _peaks()
+
+    shape = synth.LLAMA7B
+    if args.layers:
+        shape = shape.with_layers(args.layers)
+    schedule = synth.SCHEDULE_7B if shape.n_layers == 32 else synth.scaled_schedule(shape.n_layers)
+    n = args.prompt
+    # Replicas only: every rank holds all weights and its own prompt; there is no collective.
+    W = synth.make_weights(shape, 2, bf16=True, device="cuda")
+    ids_host = synth.make_prompt(shape.vocab, n, 100 + rank).pin_memory()
+    ids = ids_host.cuda()
+    logits = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+    logits_host = torch.empty((1, shape.vocab), dtype=torch.float32).pin_memory()
+    eng = B.LazyPrefill(shape, W, schedule, torch.bfloat16, 1, n)
+    full = B.LazyPrefill(shape, W, (), torch.bfloat16, 1, n)
+    cu = [0, n]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(engine, steps, warmup, timing=False):
+        for _ in range(warmup):
+            engine.lazy_prefill_run(ids, cu, logits)
+        engine.lazy_sync_status()
+        engine.lazy_set_kernel_timing(timing)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        per_kind = None
+        e0.record()
+        for _ in range(steps):
+            engine.lazy_prefill_run(ids, cu, logits)
+            if timing:   # event pairs belong to one run: collect them before the next one reuses them
+                kt = engine.lazy_get_kernel_times()
+                if per_kind is None:
+                    per_kind = {k: dict(v) for k, v in kt.items()}
+                else:
+                    for k, v in kt.items():
+                        for f in ("ms", "launches", "flops", "bytes"):
+                            per_kind[k][f] += v[f]
+        e1.record()
+        barrier()
+        engine.lazy_sync_status()
+        engine.lazy_set_kernel_timing(False)
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, per_kind
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms_pruned, _ = timed(eng, args.steps, args.warmup)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = eng.lazy_get_stats().kernel_launches * args.steps
+    ms_full, _ = timed(full, max(2, args.steps // 2), 2)
+    # per-kernel device times: a separate pass with every launch bracketed by events on the same stream
+    _, kinds = timed(eng, max(2, min(5, args.steps)), 1, timing=True)
+    ksteps = max(2, min(5, args.steps))
+
+    # end to end through the public call with host buffers: pinned ids in, logits out, every step
+    def e2e_step():
+        ids.copy_(ids_host, non_blocking=True)
+        eng.lazy_prefill_run(ids, cu, logits)
+        logits_host.copy_(logits, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        e2e_step()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    eng.lazy_sync_status()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    gemm = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down"]
+    g_ms = sum(kinds[k]["ms"] for k in gemm) / ksteps
+    g_fl = sum(kinds[k]["flops"] for k in gemm) / ksteps
+    g_launch = sum(kinds[k]["launches"] for k in gemm) / ksteps
+    achieved = g_fl / (g_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    breakdown = {}
+    for k, v in kinds.items():
+        if v["launches"] == 0:
+            continue
+        ms = v["ms"] / ksteps
+        ent = {"ms": round(ms, 4), "launches": int(v["launches"] / ksteps)}
+        if v["flops"] > 0:
+            ent["tflops"] = round(v["flops"] / ksteps / (ms * 1e-3) / 1e12, 1)
+        if v["bytes"] > 0:
+            ent["gbs"] = round(v["bytes"] / ksteps / (ms * 1e-3) / 1e9, 1)
+        breakdown[k] = ent
+    value = world * n / (ms_pruned * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_pruned, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD if (shape.n_layers == 32 and n == N_PROMPT) else
+                   f"REDUCED (profiling only): {shape.n_layers} layers, {n}-token prompt, schedule {schedule}",
+                   "batch": 1, "seq_len": n, "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "inputs (13.5 GB of weights) larger than L2"},
+        "ttft_ms_pruned": ms_pruned, "ttft_ms_full_keep": ms_full, "pruned_speedup": ms_full / ms_pruned,
+        "tokens_per_s_full_keep": world * n / (ms_full * 1e-3),
+        "clocks": clocks,
+        "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": n * 4, "d2h_bytes_per_step": shape.vocab * 4},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel (QKV, O, gate/up+SwiGLU, down)",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_kind": f"sustained bf16, {peaks['source']}", "launches_per_step": g_launch,
+                     "ms_per_step": g_ms, "traffic": None},
+        "kernels": breakdown,
+    }
+    if not args.no_cpu:
+        smp = OracleSample(n, small=False)
+        dt = smp.step_seconds()
+        out["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                               "sample": smp.sample, "whole_prompt_seconds": dt}
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="reduced depth (profiling captures only)")
+    ap.add_argument("--prompt", type=int, default=N_PROMPT)
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

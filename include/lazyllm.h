@@ -168,6 +168,24 @@ int lazy_get_kv(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t
 int lazy_get_aux(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t *d_pos,
                  void *d_hidden, int32_t *h_count);
 int lazy_get_stats(lazy_ctx *ctx, lazy_stats *out);
+/* Per-step device times.  With timing on, every kernel launch of lazy_prefill_run is bracketed by
+ * CUDA events on the caller's stream; lazy_get_kernel_times synchronises the stream and returns,
+ * per kind of step, the summed event time of the latest run together with the ALGORITHMIC work of
+ * those launches (floating-point operations for the tensor-core steps, bytes that must move for
+ * the memory-bound ones).  Event creation happens inside lazy_set_kernel_timing. */
+enum {
+  LAZY_K_GEMM_QKV = 0, LAZY_K_GEMM_O, LAZY_K_GEMM_GATE_UP, LAZY_K_GEMM_DOWN, LAZY_K_ATTENTION,
+  LAZY_K_SCORE, LAZY_K_SELECT, LAZY_K_COMPACT, LAZY_K_RMSNORM, LAZY_K_ROPE_KV, LAZY_K_EMBED,
+  LAZY_K_LM_HEAD, LAZY_K_OTHER, LAZY_N_KERNEL_KINDS
+};
+typedef struct {
+  float ms[LAZY_N_KERNEL_KINDS];
+  int32_t launches[LAZY_N_KERNEL_KINDS];
+  double flops[LAZY_N_KERNEL_KINDS];
+  double bytes[LAZY_N_KERNEL_KINDS];
+} lazy_kernel_times;
+int lazy_set_kernel_timing(lazy_ctx *ctx, int32_t on);
+int lazy_get_kernel_times(lazy_ctx *ctx, void *stream, lazy_kernel_times *out);
 /* Synchronises `stream` and returns the first device-side error recorded since the last call
  * of this function (LAZY_OK if none), clearing it. */
 int lazy_sync_status(lazy_ctx *ctx, void *stream);

@@ -55,6 +55,16 @@ class lazy_stats(C.Structure):
                 ("revived", C.c_int32 * LAZY_MAX_LAYERS), ("kernel_launches", C.c_int64)]
 
 
+LAZY_N_KERNEL_KINDS = 13
+KERNEL_KINDS = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "attention", "score", "select",
+                "compact", "rmsnorm", "rope_kv", "embed", "lm_head", "other"]
+
+
+class lazy_kernel_times(C.Structure):
+    _fields_ = [("ms", C.c_float * LAZY_N_KERNEL_KINDS), ("launches", C.c_int32 * LAZY_N_KERNEL_KINDS),
+                ("flops", C.c_double * LAZY_N_KERNEL_KINDS), ("bytes", C.c_double * LAZY_N_KERNEL_KINDS)]
+
+
 # name -> (restype, argtypes); the list mirrors include/lazyllm.h
 _P, _I, _F, _U, _Z = C.c_void_p, C.c_int32, C.c_float, C.c_uint32, C.c_size_t
 _SIGNATURES = {
@@ -73,6 +83,8 @@ _SIGNATURES = {
     "lazy_get_kv": (_I, [_P, _P, _I, _I, _P, _P, _P, C.POINTER(_I)]),
     "lazy_get_aux": (_I, [_P, _P, _I, _I, _P, _P, C.POINTER(_I)]),
     "lazy_get_stats": (_I, [_P, C.POINTER(lazy_stats)]),
+    "lazy_set_kernel_timing": (_I, [_P, _I]),
+    "lazy_get_kernel_times": (_I, [_P, _P, C.POINTER(lazy_kernel_times)]),
     "lazy_sync_status": (_I, [_P, _P]),
     "lazy_device_status": (_I, [_P]),
     "lazy_destroy": (None, [_P]),
@@ -267,6 +279,15 @@ class LazyPrefill:
         s = lazy_stats()
         _check("lazy_get_stats", lib().lazy_get_stats(self.ctx, C.byref(s)))
         return s
+
+    def lazy_set_kernel_timing(self, on: bool) -> None:
+        _check("lazy_set_kernel_timing", lib().lazy_set_kernel_timing(self.ctx, 1 if on else 0))
+
+    def lazy_get_kernel_times(self) -> Dict[str, Dict[str, float]]:
+        t = lazy_kernel_times()
+        _check("lazy_get_kernel_times", lib().lazy_get_kernel_times(self.ctx, _stream(), C.byref(t)))
+        return {name: {"ms": t.ms[i], "launches": t.launches[i], "flops": t.flops[i], "bytes": t.bytes[i]}
+                for i, name in enumerate(KERNEL_KINDS)}
 
     def lazy_sync_status(self) -> None:
         _check("lazy_sync_status", lib().lazy_sync_status(self.ctx, _stream()))

@@ -204,6 +204,35 @@ static void fill_shape(lazy_ctx *c, const lazy_model_cfg *cfg, const lazy_schedu
 
 using namespace lazy;
 
+lazy_ctx::~lazy_ctx() {
+  for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
+}
+int lazy_ctx::time_begin(cudaStream_t st, int kind, double flops, double bytes) {
+  if (!timing_on) return -1;
+  k_flops[kind] += flops;
+  k_bytes[kind] += bytes;
+  const int slot = (int)ev_kind.size();
+  while ((int)ev_pool.size() < 2 * (slot + 1)) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return -1;
+    ev_pool.push_back(e);
+  }
+  ev_kind.push_back(kind);
+  cudaEventRecord(ev_pool[2 * slot], st);
+  return slot;
+}
+void lazy_ctx::time_end(cudaStream_t st, int slot) {
+  if (slot >= 0) cudaEventRecord(ev_pool[2 * slot + 1], st);
+}
+// Runs one launcher call bracketed by an event pair when timing is on.
+#define TIMED(kind, flops, bytes, call)                                  \
+  do {                                                                   \
+    const int slot__ = c->time_begin(st, (kind), (double)(flops), (double)(bytes)); \
+    const int rc__ = (call);                                             \
+    c->time_end(st, slot__);                                             \
+    if (rc__ != LAZY_OK) return rc__;                                    \
+  } while (0)
+
 // =====================================================================================================
 extern "C" {
 
@@ -331,6 +360,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   const long long launches0 = g_launches;
   const int P = c->P, L = c->L, d = c->d, dt = c->dtype;
   const size_t rb = c->row_bytes();
+  c->ev_kind.clear();
+  for (int i = 0; i < LAZY_N_KERNEL_KINDS; ++i) c->k_flops[i] = c->k_bytes[i] = 0.0;
 
   // ---- host bookkeeping: every row count follows from the lengths and the schedule
   c->have_prefill = false;
@@ -392,7 +423,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     LAZY_TRY(launch_seg_rows(st, d_cu_drop(p), d_base, n_seqs, cu_drop[p][n_seqs], c->aux_dst[p]));
 
   // ---- embedding, positions
-  LAZY_TRY(launch_embed(st, dt, c->tok_embed, d_prompt_ids, c->x, N, d, c->V, status));
+  TIMED(LAZY_K_EMBED, 0, 2.0 * N * rb, launch_embed(st, dt, c->tok_embed, d_prompt_ids, c->x, N, d, c->V, status));
   LAZY_TRY(launch_iota_pos(st, c->pos_seg[0], d_cu(0), n_seqs, N));
 
   char *x = c->x, *x2 = c->x2;
@@ -413,15 +444,24 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     c->stats.rows_computed[l] = n;
     c->stats.kv_rows[l] = n;
 
-    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
-    LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
-    LAZY_TRY(launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H,
-                            c->dh, c->max_pos, status));
-    LAZY_TRY(launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs,
-                              seg_max, n, c->H, c->dh));
-    LAZY_TRY(launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H,
-                          c->dh, c->score_scratch, sc));
-    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status));
+    double attn_flops = 0.0;
+    for (int s = 0; s < n_seqs; ++s) {
+      const double ns = c->seg_cu[g][s + 1] - c->seg_cu[g][s];
+      attn_flops += 2.0 * d * ns * (ns + 1.0);
+    }
+    TIMED(LAZY_K_RMSNORM, 0, 2.0 * n * rb, launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
+    TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
+          launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
+    TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
+          launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
+                         c->max_pos, status));
+    TIMED(LAZY_K_ATTENTION, attn_flops, 0,
+          launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
+                           c->H, c->dh));
+    TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
+          launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
+                       c->score_scratch, sc));
+    TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status));
 
     const int p = c->point_at[l + 1];
     if (p >= 0) {
@@ -441,29 +481,37 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
         sel = c->sel_scores;
       }
       const int n_keep = c->seg_cu[g + 1][n_seqs], n_drop = n - n_keep;
-      LAZY_TRY(launch_select(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->keep_idx[p], c->drop_idx[p], status));
+      TIMED(LAZY_K_SELECT, 0, 8.0 * n,
+            launch_select(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->keep_idx[p], c->drop_idx[p], status));
       char *ar = c->aux_rows + (size_t)p * c->cap_kv * rb;
       int32_t *ap = c->aux_pos + (size_t)p * c->cap_kv;
-      LAZY_TRY(launch_move_rows(st, x, c->drop_idx[p], ar, c->aux_dst[p], n_drop, (int)rb, n, c->cap_kv, status));
-      LAZY_TRY(launch_move_i32(st, pos, c->drop_idx[p], ap, c->aux_dst[p], n_drop));
-      LAZY_TRY(launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
-      LAZY_TRY(launch_move_i32(st, pos, c->keep_idx[p], c->pos_seg[g + 1], nullptr, n_keep));
+      TIMED(LAZY_K_COMPACT, 0, 2.0 * n_drop * rb,
+            launch_move_rows(st, x, c->drop_idx[p], ar, c->aux_dst[p], n_drop, (int)rb, n, c->cap_kv, status));
+      TIMED(LAZY_K_COMPACT, 0, 8.0 * n_drop, launch_move_i32(st, pos, c->drop_idx[p], ap, c->aux_dst[p], n_drop));
+      TIMED(LAZY_K_COMPACT, 0, 2.0 * n_keep * rb,
+            launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
+      TIMED(LAZY_K_COMPACT, 0, 8.0 * n_keep,
+            launch_move_i32(st, pos, c->keep_idx[p], c->pos_seg[g + 1], nullptr, n_keep));
       for (int s = 0; s < n_seqs; ++s) c->aux_count[p][s] = cu_drop[p][s + 1] - cu_drop[p][s];
       c->stats.aux_rows[l] = n_drop;
       char *t = x; x = x2; x2 = t;
       ++g;
     }
     const int n2 = c->seg_cu[g][n_seqs];
-    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
-    LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status));
-    LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status));
+    TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb, launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
+    TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
+          launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status));
+    TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
+          launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status));
     if (c->capture_on && c->capture)
       LAZY_CUDA_OK(cudaMemcpyAsync(c->capture + (size_t)l * c->cap_rows * rb, x, (size_t)n2 * rb,
                                    cudaMemcpyDeviceToDevice, st));
   }
   // ---- first-token logits from the last row of every sequence
-  LAZY_TRY(launch_rmsnorm_rows(st, dt, x, d_last, c->g_final, c->h_last, n_seqs, d, c->cfg.rms_eps));
-  LAZY_TRY(launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, n_seqs, d, c->V));
+  TIMED(LAZY_K_RMSNORM, 0, 2.0 * n_seqs * rb,
+        launch_rmsnorm_rows(st, dt, x, d_last, c->g_final, c->h_last, n_seqs, d, c->cfg.rms_eps));
+  TIMED(LAZY_K_LM_HEAD, 0, (double)c->V * rb,
+        launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, n_seqs, d, c->V));
   // the residual stream may live in either ping-pong buffer; decode does not need it
   c->forced.clear();
   c->have_prefill = true;
@@ -600,6 +648,36 @@ int lazy_get_aux(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t 
 int lazy_get_stats(lazy_ctx *c, lazy_stats *out) {
   if (!c || !out) return LAZY_E_BADARG;
   *out = c->stats;
+  return LAZY_OK;
+}
+
+int lazy_set_kernel_timing(lazy_ctx *c, int32_t on) {
+  if (!c) return LAZY_E_BADARG;
+  c->timing_on = on != 0;
+  if (on) {  // create the events now so that the timed run itself creates none
+    while (c->ev_pool.size() < 2048) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return LAZY_E_CUDA;
+      c->ev_pool.push_back(e);
+    }
+  }
+  return LAZY_OK;
+}
+
+int lazy_get_kernel_times(lazy_ctx *c, void *stream, lazy_kernel_times *out) {
+  if (!c || !out) return LAZY_E_BADARG;
+  LAZY_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  memset(out, 0, sizeof(*out));
+  for (size_t i = 0; i < c->ev_kind.size(); ++i) {
+    float ms = 0.f;
+    LAZY_CUDA_OK(cudaEventElapsedTime(&ms, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+    out->ms[c->ev_kind[i]] += ms;
+    out->launches[c->ev_kind[i]] += 1;
+  }
+  for (int k = 0; k < LAZY_N_KERNEL_KINDS; ++k) {
+    out->flops[k] = c->k_flops[k];
+    out->bytes[k] = c->k_bytes[k];
+  }
   return LAZY_OK;
 }
 

@@ -65,6 +65,16 @@ struct lazy_ctx {
   std::map<std::pair<int, int>, std::pair<const int32_t *, int>> forced;  // (point, seq) -> list
   lazy_stats stats;
 
+  // ---- optional per-kernel event timing
+  bool timing_on = false;
+  std::vector<cudaEvent_t> ev_pool;  // pairs: 2*i start, 2*i+1 stop
+  std::vector<int> ev_kind;          // kind of each used pair
+  double k_flops[LAZY_N_KERNEL_KINDS], k_bytes[LAZY_N_KERNEL_KINDS];
+  // Returns the index of a fresh event pair (or -1) after recording its start.
+  int time_begin(cudaStream_t st, int kind, double flops, double bytes);
+  void time_end(cudaStream_t st, int slot);
+  ~lazy_ctx();
+
   size_t row_bytes() const { return (size_t)d * eb; }
   int seg_of_layer(int l) const {  // segment whose rows enter layer l
     int g = 0;
