@@ -249,6 +249,21 @@ size_t lazy_k_score_scratch_floats(int32_t n_seqs, int32_t n_total, int32_t n_he
 int lazy_k_score(void *stream, int32_t dtype, const void *q, int32_t ldq, const void *k,
                  int32_t ldkv, const int32_t *d_cu_seqlens, int32_t n_seqs, int32_t n_total,
                  int32_t n_heads, int32_t head_dim, float *scratch, float *scores);
+/* Same result as lazy_k_score, for callers that cannot allocate device memory (no counterpart in
+ * the paper: this is a deployment convenience).  Such callers exist: a plugin inside a host
+ * application that owns all device memory, a latency-critical callback where cudaMalloc would
+ * stall the device, a process that has already handed its memory to another owner.  The scratch
+ * (per-head logits and softmax statistics) lives in a fixed array inside the library that every
+ * GPU loading it holds until exit (about 1.04 MB).  Limits: n_heads * n_total <= 262144 and
+ * 2 * n_heads * n_seqs <= 4096; anything larger returns LAZY_E_CAPACITY and runs nothing.  The
+ * call allocates and frees nothing.  The first call on each device looks up the array's device
+ * address (a synchronous runtime query), so make that first call outside any stream capture.
+ * All calls share the one array, which simply keeps what the last call left there (nothing needs
+ * clearing: every value read is written earlier by the same call); two calls whose kernels may
+ * overlap on the GPU (different streams, different threads) race on it, so serialise them. */
+int lazy_k_score_static(void *stream, int32_t dtype, const void *q, int32_t ldq, const void *k,
+                        int32_t ldkv, const int32_t *d_cu_seqlens, int32_t n_seqs, int32_t n_total,
+                        int32_t n_heads, int32_t head_dim, float *scores);
 /* Top-percentile selection per sequence (Section 3.2): keeps n_keep[s] rows with the largest
  * score, the last row always, ties to the lower index.  d_cu_in / d_cu_keep: device
  * int32[n_seqs+1] prefix sums of rows in / rows kept.  keep_idx / drop_idx receive packed row

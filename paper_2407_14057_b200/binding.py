@@ -99,6 +99,7 @@ _SIGNATURES = {
     "lazy_k_attention": (_I, [_P, _I, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _I]),
     "lazy_k_score_scratch_floats": (_Z, [_I, _I, _I]),
     "lazy_k_score": (_I, [_P, _I, _P, _I, _P, _I, _P, _I, _I, _I, _I, _P, _P]),
+    "lazy_k_score_static": (_I, [_P, _I, _P, _I, _P, _I, _P, _I, _I, _I, _I, _P]),
     "lazy_k_select": (_I, [_P, _P, _P, _P, _I, _P, _P]),
     "lazy_k_gather_rows": (_I, [_P, _P, _P, _P, _I, _I, _I]),
 }
@@ -359,6 +360,16 @@ def lazy_k_score(q: torch.Tensor, ldq: int, k: torch.Tensor, ldkv: int, cu_seqle
     _check("lazy_k_score", lib().lazy_k_score(_stream(), dtype_code(k.dtype), q.data_ptr(), ldq, _ptr(k), ldkv,
                                               _ptr(cu_seqlens), n_seqs, n_total, n_heads, head_dim,
                                               _ptr(scratch), _ptr(scores)))
+    return scores
+
+
+def lazy_k_score_static(q: torch.Tensor, ldq: int, k: torch.Tensor, ldkv: int, cu_seqlens: torch.Tensor,
+                        n_total: int, n_heads: int, head_dim: int, scores: torch.Tensor) -> torch.Tensor:
+    """Eq. 1 scores with the scratch held inside the library: nothing is allocated by the call, so the
+    caller passes the output tensor too."""
+    _check("lazy_k_score_static", lib().lazy_k_score_static(
+        _stream(), dtype_code(k.dtype), q.data_ptr(), ldq, _ptr(k), ldkv, _ptr(cu_seqlens),
+        cu_seqlens.numel() - 1, n_total, n_heads, head_dim, _ptr(scores)))
     return scores
 
 

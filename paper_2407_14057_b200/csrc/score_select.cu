@@ -268,4 +268,52 @@ int launch_forced_scores(cudaStream_t st, const int32_t *pos, int r0, int n, con
   return launch_ok();
 }
 
+
+// ---- importance score without caller-provided scratch ---------------------------------------------
+// Some callers of this library cannot hand over scratch memory because they are not allowed to
+// allocate device memory at all: a plugin running inside a host application whose memory pool is
+// closed to it, a callback on a serving path where cudaMalloc would stall every stream of the
+// device, or code that runs after the process has given all memory to another owner.  For them the
+// score's scratch (per-head logits plus the softmax statistics) lives in this fixed array, which
+// every GPU that loads the library holds until the process exits.
+namespace {
+constexpr int STATIC_SCORE_MAX_LOGITS = 262144;  // n_heads * n_total, e.g. 32 heads x 8192 tokens
+constexpr int STATIC_SCORE_MAX_STATS = 4096;     // 2 * n_heads * n_seqs
+static __device__ __align__(256) float g_static_score_scratch[STATIC_SCORE_MAX_LOGITS + STATIC_SCORE_MAX_STATS];
+
+// Device address of the array on the current device.  The array's name is only a host-side handle
+// here: the address a kernel can use comes from cudaGetSymbolAddress, asked once per device.
+float *static_score_scratch_ptr() {
+  static float *ptrs[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ptrs[dev]) {
+    float *p = nullptr;
+    if (cudaGetSymbolAddress((void **)&p, g_static_score_scratch) != cudaSuccess) return nullptr;
+    ptrs[dev] = p;
+  }
+  return ptrs[dev];
+}
+}  // namespace
+
 }  // namespace lazy
+
+extern "C" int lazy_k_score_static(void *stream, int32_t dtype, const void *q, int32_t ldq, const void *k,
+                                   int32_t ldkv, const int32_t *d_cu_seqlens, int32_t n_seqs,
+                                   int32_t n_total, int32_t n_heads, int32_t head_dim, float *scores) {
+  using namespace lazy;
+  if ((dtype != LAZY_BF16 && dtype != LAZY_F32) || !q || !k || !d_cu_seqlens || !scores || n_seqs < 0 ||
+      n_total < 0 || n_heads < 1)
+    return LAZY_E_BADARG;
+  // sizes beyond the fixed array are refused, never truncated
+  if ((long long)n_heads * n_total > STATIC_SCORE_MAX_LOGITS ||
+      2LL * n_heads * n_seqs > STATIC_SCORE_MAX_STATS)
+    return LAZY_E_CAPACITY;
+  float *scratch = static_score_scratch_ptr();
+  if (!scratch) return LAZY_E_CUDA;
+  // Layout inside the array matches what launch_score expects for this (n_heads, n_total): logits
+  // first, statistics right after them.  Every element that is read is written first by the same
+  // call, so nothing has to be cleared between calls.
+  return launch_score((cudaStream_t)stream, dtype, q, ldq, k, ldkv, d_cu_seqlens, nullptr, n_seqs, n_total,
+                      n_total, n_heads, head_dim, scratch, scores);
+}
