@@ -137,13 +137,15 @@ int aux_cache_revive(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq,
 
 /* ---- introspection (parity checks, replay of another implementation's kept sets) ------- */
 
-/* Kept set entering `layer_entered` (a schedule point) of sequence `seq` in the latest call, as
+/* Kept set entering `layer_entered` (a schedule point) of sequence `seq` in the latest call
+ * (after a decode step: the context re-selected there, the new token included), as
  * original token positions ascending; d_pos: device int32 with room for the count (may be NULL
  * to query the count only).  Synchronises the stream. */
 int lazy_get_kept(lazy_ctx *ctx, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
                   int32_t *h_count);
 /* Eq. 1 scores of `layer` for sequence `seq` in the latest call, one per candidate row in
- * ascending position order (prefill: the rows present at that layer). */
+ * ascending position order (prefill: the rows present at that layer; decode: the context the new
+ * token attended at that layer, itself last). */
 int lazy_get_scores(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, float *d_scores,
                     int32_t *h_count);
 /* Test hook: the NEXT prefill (decode step) takes this kept set (positions, ascending, device
@@ -167,6 +169,11 @@ int lazy_get_kv(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t
                 void *d_v, int32_t *h_count);
 int lazy_get_aux(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_t *d_pos,
                  void *d_hidden, int32_t *h_count);
+/* Positions (ascending) of the tokens of sequence `seq` that the latest decode step revived from
+ * the Aux Cache into `layer_entered` (Section 3.2: hidden states fetched from the Aux Cache of the
+ * previous layer instead of being recomputed).  Zero after a prefill. */
+int lazy_get_revived(lazy_ctx *ctx, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
+                     int32_t *h_count);
 int lazy_get_stats(lazy_ctx *ctx, lazy_stats *out);
 /* Per-step device times.  With timing on, every kernel launch of lazy_prefill_run is bracketed by
  * CUDA events on the caller's stream; lazy_get_kernel_times synchronises the stream and returns,

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "lazy_get_hidden": (_I, [_P, _P, _I, _P, C.POINTER(_I)]),
     "lazy_get_kv": (_I, [_P, _P, _I, _I, _P, _P, _P, C.POINTER(_I)]),
     "lazy_get_aux": (_I, [_P, _P, _I, _I, _P, _P, C.POINTER(_I)]),
+    "lazy_get_revived": (_I, [_P, _P, _I, _I, _P, C.POINTER(_I)]),
     "lazy_get_stats": (_I, [_P, C.POINTER(lazy_stats)]),
     "lazy_set_kernel_timing": (_I, [_P, _I]),
     "lazy_get_kernel_times": (_I, [_P, _P, C.POINTER(lazy_kernel_times)]),
@@ -275,6 +276,15 @@ class LazyPrefill:
         _check("lazy_get_aux", lib().lazy_get_aux(self.ctx, _stream(), layer, seq, _ptr(pos), _ptr(hid),
                                                   C.byref(cnt)))
         return pos, hid
+
+    def lazy_get_revived(self, layer_entered: int, seq: int = 0) -> torch.Tensor:
+        cnt = C.c_int32()
+        _check("lazy_get_revived", lib().lazy_get_revived(self.ctx, _stream(), layer_entered, seq, None,
+                                                          C.byref(cnt)))
+        out = torch.empty(cnt.value, dtype=torch.int32, device="cuda")
+        _check("lazy_get_revived", lib().lazy_get_revived(self.ctx, _stream(), layer_entered, seq, _ptr(out),
+                                                          C.byref(cnt)))
+        return out
 
     def lazy_get_stats(self) -> lazy_stats:
         s = lazy_stats()

@@ -20,7 +20,10 @@ template <typename T>
 __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *__restrict__ k,
                                     const T *__restrict__ v, int ldkv, T *__restrict__ o,
                                     const int32_t *__restrict__ cu_q,
-                                    const int32_t *__restrict__ kv_base, int n_seqs, int n_total,
+                                    const int32_t *__restrict__ kv_base,
+                                    const int32_t *__restrict__ cu_kv,
+                                    const int32_t *__restrict__ kv_idx,
+                                    const int32_t *__restrict__ q_kvlen, int n_seqs, int n_total,
                                     int n_heads, int head_dim) {
   extern __shared__ float qs_all[];  // [warps][head_dim]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -32,8 +35,11 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
     int mid = (lo + hi) >> 1;
     if (cu_q[mid] <= r) lo = mid; else hi = mid;
   }
-  const int i = r - cu_q[lo];
+  // keys visible to this row: the first `vis` entries of the sequence's key list
+  const int vis = q_kvlen ? q_kvlen[r] : r - cu_q[lo] + 1;
+  const int i = vis - 1;
   const size_t kbase = kv_base ? (size_t)kv_base[lo] : (size_t)cu_q[lo];
+  const int32_t *kidx = kv_idx ? kv_idx + cu_kv[lo] : nullptr;
   float *qs = qs_all + warp * head_dim;
   const float scale = rsqrtf((float)head_dim);
   for (int t = lane; t < head_dim; t += 32)
@@ -48,7 +54,7 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
     const int j = j0 + lane;
     float s = -INFINITY;
     if (j <= i) {
-      const T *kr = k + (kbase + j) * ldkv + h * head_dim;
+      const T *kr = k + (kidx ? (size_t)kidx[j] : kbase + j) * ldkv + h * head_dim;
       float dot = 0.f;
       for (int t = 0; t < head_dim; ++t) dot += qs[t] * Elem<T>::to_f(kr[t]);
       s = dot;
@@ -63,7 +69,7 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
     const int cnt = min(32, i - j0 + 1);
     for (int jj = 0; jj < cnt; ++jj) {
       const float pj = __shfl_sync(0xffffffffu, p, jj);
-      const T *vr = v + (kbase + j0 + jj) * ldkv + h * head_dim;
+      const T *vr = v + (kidx ? (size_t)kidx[j0 + jj] : kbase + j0 + jj) * ldkv + h * head_dim;
 #pragma unroll
       for (int t = 0; t < 8; ++t)
         if (t < per_lane) acc[t] += pj * Elem<T>::to_f(vr[lane + 32 * t]);
@@ -117,19 +123,24 @@ __device__ __forceinline__ void mma_bf16(float *c, const uint32_t *a, uint32_t b
 
 // Copies 64 rows x 256 B (one head's slice) into a swizzled tile.  Rows past `n_valid` re-read the
 // last valid row so that shared memory never holds uninitialised (possibly non-finite) data.
-__device__ __forceinline__ void load_tile(uint32_t tile, const bf16 *base, int ld, int row0, int n_valid) {
+// With `idx`, list entry j names the cache row to read (decode: keys picked by position).
+__device__ __forceinline__ void load_tile(uint32_t tile, const bf16 *base, int ld, int row0, int n_valid,
+                                          const int32_t *idx = nullptr) {
   for (int t = threadIdx.x; t < FA_BN * 16; t += FA_THREADS) {
     const int r = t >> 4, c = t & 15;
     int gr = row0 + r;
     if (gr > n_valid - 1) gr = n_valid - 1;
-    cp_async16(tile + sw_off(r, c), base + (size_t)gr * ld + c * 8);
+    const size_t src = idx ? (size_t)idx[gr] : (size_t)gr;
+    cp_async16(tile + sw_off(r, c), base + src * ld + c * 8);
   }
 }
 
 __global__ void __launch_bounds__(FA_THREADS)
 attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
                 const bf16 *__restrict__ v, int ldkv, bf16 *__restrict__ o,
-                const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base, int n_heads) {
+                const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base,
+                const int32_t *__restrict__ cu_kv, const int32_t *__restrict__ kv_idx,
+                const int32_t *__restrict__ q_kvlen, int n_heads) {
   extern __shared__ __align__(128) uint8_t fa_smem[];
   const int seq = blockIdx.z, h = blockIdx.y;
   const int q_start = cu_q[seq];
@@ -138,7 +149,10 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   if ((int)blockIdx.x >= q_tiles) return;
   const int qt = q_tiles - 1 - blockIdx.x;  // longest rows first
   const int q0 = qt * FA_BM;
-  const size_t kb = kv_base ? (size_t)kv_base[seq] : (size_t)q_start;
+  // keys: either the sequence's contiguous cache rows, or the rows a list names (decode)
+  const int32_t *kidx = kv_idx ? kv_idx + cu_kv[seq] : nullptr;
+  const int n_kv = kv_idx ? cu_kv[seq + 1] - cu_kv[seq] : n;
+  const size_t kb = kv_idx ? 0 : (kv_base ? (size_t)kv_base[seq] : (size_t)q_start);
   const bf16 *qg = q + (size_t)q_start * ldq + h * FA_D;
   const bf16 *kg = k + kb * ldkv + h * FA_D;
   const bf16 *vg = v + kb * ldkv + h * FA_D;
@@ -149,10 +163,18 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t4 = lane & 3;
 
-  const int n_kt = (min(q0 + FA_BM, n) + FA_BN - 1) / FA_BN;  // key tiles up to the diagonal
+  // Row i sees the first vis(i) keys; vis is non-decreasing in i (prefill: i + 1).
+  const int last_row = min(q0 + FA_BM, n) - 1;
+  const int vis_tile = q_kvlen ? min(q_kvlen[q_start + last_row], n_kv) : last_row + 1;
+  const int n_kt = (vis_tile + FA_BN - 1) / FA_BN;  // key tiles up to the diagonal
+  const int wrow0 = min(q0 + warp * 16 + g, n - 1), wrow1 = min(q0 + warp * 16 + g + 8, n - 1);
+  const int vis0 = q_kvlen ? q_kvlen[q_start + wrow0] : wrow0 + 1;
+  const int vis1 = q_kvlen ? q_kvlen[q_start + wrow1] : wrow1 + 1;
+  const int wfirst = min(q0 + warp * 16, n - 1);
+  const int vis_first = q_kvlen ? q_kvlen[q_start + wfirst] : wfirst + 1;
   load_tile(sQ, qg, ldq, q0, n);
-  load_tile(sK, kg, ldkv, 0, n);
-  load_tile(sV, vg, ldkv, 0, n);
+  load_tile(sK, kg, ldkv, 0, n_kv, kidx);
+  load_tile(sV, vg, ldkv, 0, n_kv, kidx);
   cp_async_commit();
 
   uint32_t qf[8][4];
@@ -165,8 +187,8 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   for (int kt = 0; kt < n_kt; ++kt) {
     const int buf = kt & 1;
     if (kt + 1 < n_kt) {  // prefetch the next K/V tile into the other buffer
-      load_tile(sK + (buf ^ 1) * FA_TILE_BYTES, kg, ldkv, (kt + 1) * FA_BN, n);
-      load_tile(sV + (buf ^ 1) * FA_TILE_BYTES, vg, ldkv, (kt + 1) * FA_BN, n);
+      load_tile(sK + (buf ^ 1) * FA_TILE_BYTES, kg, ldkv, (kt + 1) * FA_BN, n_kv, kidx);
+      load_tile(sV + (buf ^ 1) * FA_TILE_BYTES, vg, ldkv, (kt + 1) * FA_BN, n_kv, kidx);
       cp_async_commit();
       cp_async_wait<1>();
     } else {
@@ -197,10 +219,9 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
         mma_bf16(s[2 * np + 1], qf[ks], b2, b3);
       }
     }
-    // scale, causal mask (key index > query index), running max
-    const int qrow0 = q0 + warp * 16 + g;  // rows qrow0 and qrow0 + 8
+    // scale, causal mask (key index >= keys visible to the row), running max
     const int kcol0 = kt * FA_BN + 2 * t4;
-    const bool diag = (kt + 1) * FA_BN > q0 + warp * 16;  // tile may cross this warp's diagonal
+    const bool diag = (kt + 1) * FA_BN > vis_first;  // tile may cross this warp's diagonal
     float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -209,8 +230,7 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
         float val = s[i][e] * sl2;
         if (diag) {
           const int col = kcol0 + i * 8 + (e & 1);
-          const int row = qrow0 + ((e >> 1) << 3);
-          if (col > row) val = -INFINITY;
+          if (col >= ((e >> 1) ? vis1 : vis0)) val = -INFINITY;
         }
         s[i][e] = val;
         mx[e >> 1] = fmaxf(mx[e >> 1], val);
@@ -285,6 +305,14 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                      const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                      int n_seqs, int max_len, int n_total, int n_heads, int head_dim) {
+  return launch_attention_ex(st, dtype, q, ldq, k, v, ldkv, o, cu_q, kv_base, nullptr, nullptr, nullptr,
+                             n_seqs, max_len, n_total, n_heads, head_dim);
+}
+
+int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
+                        const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
+                        const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
+                        int max_len, int n_total, int n_heads, int head_dim) {
   if (n_total == 0 || n_seqs == 0) return LAZY_OK;
   if (dtype == LAZY_BF16 && head_dim == FA_D && (ldq % 8) == 0 && (ldkv % 8) == 0) {
     static bool attr_set = false;
@@ -296,7 +324,7 @@ int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const v
     dim3 grid(cdiv(max_len, FA_BM), n_heads, n_seqs);
     attn_mma_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>((const bf16 *)q, ldq, (const bf16 *)k,
                                                              (const bf16 *)v, ldkv, (bf16 *)o, cu_q,
-                                                             kv_base, n_heads);
+                                                             kv_base, cu_kv, kv_idx, q_kvlen, n_heads);
     LAZY_COUNT_LAUNCH();
     return launch_ok();
   }
@@ -307,11 +335,13 @@ int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const v
   if (dtype == LAZY_F32)
     attn_rowwarp_kernel<float><<<grid, warps * 32, smem, st>>>((const float *)q, ldq, (const float *)k,
                                                               (const float *)v, ldkv, (float *)o, cu_q,
-                                                              kv_base, n_seqs, n_total, n_heads, head_dim);
+                                                              kv_base, cu_kv, kv_idx, q_kvlen, n_seqs, n_total,
+                                                              n_heads, head_dim);
   else
     attn_rowwarp_kernel<bf16><<<grid, warps * 32, smem, st>>>((const bf16 *)q, ldq, (const bf16 *)k,
                                                              (const bf16 *)v, ldkv, (bf16 *)o, cu_q,
-                                                             kv_base, n_seqs, n_total, n_heads, head_dim);
+                                                             kv_base, cu_kv, kv_idx, q_kvlen, n_seqs, n_total,
+                                                             n_heads, head_dim);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

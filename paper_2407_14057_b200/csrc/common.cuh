@@ -164,10 +164,23 @@ int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, 
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                      const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                      int n_seqs, int max_len, int n_total, int n_heads, int head_dim);
+// General form (decode): sequence s has query rows [cu_q[s], cu_q[s+1]) and a key LIST
+// kv_idx[cu_kv[s] .. cu_kv[s+1]) of cache rows in ascending position order; query row r sees the
+// first q_kvlen[r] entries of its sequence's list.
+int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
+                        const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
+                        const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
+                        int max_len, int n_total, int n_heads, int head_dim);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                  const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
                  int n_heads, int head_dim, float *scratch, float *scores);
+// General form (decode): sequence s scores the key LIST key_rows[cu_q[s] .. cu_q[s+1]) (cache rows)
+// with the query in row q_rows[s].
+int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
+                    const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
+                    const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,
+                    int head_dim, float *scratch, float *scores);
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
                   const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
                   DevStatus *status);

@@ -149,10 +149,10 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->pos_seg.assign(P + 1, nullptr);
   c->kv_row.assign(P + 1, nullptr);
   for (int g = 0; g <= P; ++g) {
-    c->pos_seg[g] = (int32_t *)k.take(R * 4);
+    c->pos_seg[g] = (int32_t *)k.take(KV * 4);
     c->kv_row[g] = (int32_t *)k.take(R * 4);
   }
-  c->scores = (float *)k.take((size_t)L * R * 4);
+  c->scores = (float *)k.take((size_t)L * KV * 4);
   c->sel_scores = (float *)k.take(R * 4);
   c->score_scratch = (float *)k.take(score_scratch_floats(c->S, c->cap_kv, c->H) * 4);
   c->keep_idx.assign(P, nullptr);
@@ -163,6 +163,8 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
     c->drop_idx[p] = (int32_t *)k.take(R * 4);
     c->aux_dst[p] = (int32_t *)k.take(R * 4);
   }
+  c->revived_pos.assign(P, nullptr);
+  for (int p = 0; p < P; ++p) c->revived_pos[p] = (int32_t *)k.take(KV * 4);
   c->rope_table = (float *)k.take((size_t)c->max_pos * c->dh * 4);
   c->kcache = k.take((size_t)L * KV * rb);
   c->vcache = k.take((size_t)L * KV * rb);
@@ -173,7 +175,7 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->d_found = (int32_t *)k.take(KV * 4);
   c->kv_map = (int32_t *)k.take((size_t)L * KV * 4);
   c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
-  c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)64 * (c->S + 1) * 4);
+  c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)16 * 2 * (c->S + 1) * 4);
   c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
   c->capture = with_capture ? k.take((size_t)L * R * rb) : nullptr;
   return k.off;
@@ -396,6 +398,9 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   }
   c->kv_count.assign(L, std::vector<int>(n_seqs, 0));
   c->aux_count.assign(P, std::vector<int>(n_seqs, 0));
+  c->aux_live.assign(P, std::vector<int>(n_seqs, 0));
+  c->dec_revived_cu.assign(P, std::vector<int>(n_seqs + 1, 0));
+  c->last_was_decode = false;
   memset(&c->stats, 0, sizeof(c->stats));
   c->stats.n_layers = L;
 
@@ -434,7 +439,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     char *kc = c->kcache + (size_t)l * c->cap_kv * rb;
     char *vc = c->vcache + (size_t)l * c->cap_kv * rb;
     int32_t *kvp = c->kv_pos + (size_t)l * c->cap_kv;
-    float *sc = c->scores + (size_t)l * c->cap_rows;
+    float *sc = c->scores + (size_t)l * c->cap_kv;
     int seg_max = 0;
     for (int s = 0; s < n_seqs; ++s) {
       const int ns = c->seg_cu[g][s + 1] - c->seg_cu[g][s];
@@ -492,7 +497,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
             launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
       TIMED(LAZY_K_COMPACT, 0, 8.0 * n_keep,
             launch_move_i32(st, pos, c->keep_idx[p], c->pos_seg[g + 1], nullptr, n_keep));
-      for (int s = 0; s < n_seqs; ++s) c->aux_count[p][s] = cu_drop[p][s + 1] - cu_drop[p][s];
+      for (int s = 0; s < n_seqs; ++s)
+        c->aux_count[p][s] = c->aux_live[p][s] = cu_drop[p][s + 1] - cu_drop[p][s];
       c->stats.aux_rows[l] = n_drop;
       char *t = x; x = x2; x2 = t;
       ++g;
@@ -584,7 +590,7 @@ int lazy_get_scores(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, float
   if (h_count) *h_count = b - a;
   cudaStream_t st = (cudaStream_t)stream;
   if (d_scores)
-    LAZY_CUDA_OK(cudaMemcpyAsync(d_scores, c->scores + (size_t)layer * c->cap_rows + a, (size_t)(b - a) * 4,
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_scores, c->scores + (size_t)layer * c->cap_kv + a, (size_t)(b - a) * 4,
                                  cudaMemcpyDeviceToDevice, st));
   LAZY_CUDA_OK(cudaStreamSynchronize(st));
   return LAZY_OK;
@@ -623,25 +629,77 @@ int lazy_get_kv(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t *
   return LAZY_OK;
 }
 
+// Live entries of a region of position tags (tag >= 0), as global rows, uploaded to d_list.
+static int live_rows(lazy_ctx *c, cudaStream_t st, const int32_t *tags, int row0, int count,
+                     int32_t *d_list, int *n_live, bool want_tag_value, std::vector<int32_t> *vals) {
+  std::vector<int32_t> h((size_t)count);
+  if (count) {
+    LAZY_CUDA_OK(cudaMemcpyAsync(h.data(), tags + row0, (size_t)count * 4, cudaMemcpyDeviceToHost, st));
+    LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  }
+  std::vector<int32_t> rows;
+  for (int i = 0; i < count; ++i)
+    if (h[i] >= 0) {
+      rows.push_back(row0 + i);
+      if (want_tag_value && vals) vals->push_back(h[i]);
+    }
+  *n_live = (int)rows.size();
+  if (d_list && !rows.empty()) {
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_list, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice, st));
+    LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  }
+  (void)c;
+  return LAZY_OK;
+}
+
 int lazy_get_aux(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t *d_pos, void *d_hidden,
                  int32_t *h_count) {
   if (!c || layer < 0 || layer >= c->L || seq < 0) return LAZY_E_BADARG;
   if (!c->have_prefill) return LAZY_E_STATE;
   if (seq >= c->n_seqs) return LAZY_E_BADARG;
-  const int p = layer + 1 <= c->L ? c->point_at[layer + 1] : -1;
+  const int p = c->point_at[layer + 1];
   if (p < 0) {
     if (h_count) *h_count = 0;
     return LAZY_OK;
   }
-  const int cnt = c->aux_count[p][seq];
-  const size_t rb = c->row_bytes();
-  const size_t row0 = (size_t)p * c->cap_kv + c->seq_base[seq];
-  if (h_count) *h_count = cnt;
   cudaStream_t st = (cudaStream_t)stream;
-  if (d_pos) LAZY_CUDA_OK(cudaMemcpyAsync(d_pos, c->aux_pos + row0, (size_t)cnt * 4, cudaMemcpyDeviceToDevice, st));
+  DevStatus *status = dev_status_ptr();
+  if (!status) return LAZY_E_CUDA;
+  const size_t rb = c->row_bytes();
+  const int32_t *ap = c->aux_pos + (size_t)p * c->cap_kv;
+  int n_live = 0;
+  // entries revived during decode stay in place with tag -1: hand out the live ones only
+  LAZY_TRY(live_rows(c, st, ap, c->seq_base[seq], c->aux_count[p][seq], c->d_found, &n_live, false, nullptr));
+  if (h_count) *h_count = n_live;
+  if (d_pos) LAZY_TRY(launch_move_i32(st, ap, c->d_found, d_pos, nullptr, n_live));
   if (d_hidden)
-    LAZY_CUDA_OK(cudaMemcpyAsync(d_hidden, c->aux_rows + row0 * rb, (size_t)cnt * rb, cudaMemcpyDeviceToDevice, st));
+    LAZY_TRY(launch_move_rows(st, c->aux_rows + (size_t)p * c->cap_kv * rb, c->d_found, d_hidden, nullptr,
+                              n_live, (int)rb, c->cap_kv, n_live > 0 ? n_live : 1, status));
   LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  return LAZY_OK;
+}
+
+int lazy_get_revived(lazy_ctx *c, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
+                     int32_t *h_count) {
+  if (!c || layer_entered < 0 || layer_entered > c->L || seq < 0) return LAZY_E_BADARG;
+  if (!c->have_prefill) return LAZY_E_STATE;
+  if (seq >= c->n_seqs) return LAZY_E_BADARG;
+  const int p = c->point_at[layer_entered];
+  if (p < 0) return LAZY_E_BADARG;
+  if (!c->last_was_decode) {  // prefill revives nothing
+    if (h_count) *h_count = 0;
+    return LAZY_OK;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const int a = c->dec_revived_cu[p][seq], b = c->dec_revived_cu[p][seq + 1];
+  std::vector<int32_t> vals;
+  int n_live = 0;
+  LAZY_TRY(live_rows(c, st, c->revived_pos[p], a, b - a, nullptr, &n_live, true, &vals));
+  if (h_count) *h_count = n_live;
+  if (d_pos && n_live) {
+    LAZY_CUDA_OK(cudaMemcpyAsync(d_pos, vals.data(), vals.size() * 4, cudaMemcpyHostToDevice, st));
+    LAZY_CUDA_OK(cudaStreamSynchronize(st));
+  }
   return LAZY_OK;
 }
 

@@ -47,6 +47,8 @@ struct lazy_ctx {
   // decode-only buffers
   int32_t *kv_map;   // [L, cap_kv]: cache row of (sequence base + position), -1 if absent
   int32_t *aux_map;  // [P, cap_kv]: Aux row of (sequence base + position), -1 if absent
+  std::vector<int32_t *> revived_pos;  // [P] x [cap_kv]: per in-flight row after a boundary, its
+                                       // position if it came from the Aux Cache, else -1
   int32_t *dec_i32;  // integer scratch of the decode step
   float *dec_f32;
 
@@ -61,7 +63,11 @@ struct lazy_ctx {
   std::vector<int> seq_base;               // [n_seqs] first cache row of the sequence's region
   std::vector<std::vector<int>> seg_cu;    // [P+1][n_seqs+1] packed row offsets per segment
   std::vector<std::vector<int>> kv_count;  // [L][n_seqs]
-  std::vector<std::vector<int>> aux_count; // [P][n_seqs]
+  std::vector<std::vector<int>> aux_count; // [P][n_seqs] rows appended (retired entries included)
+  std::vector<std::vector<int>> aux_live;  // [P][n_seqs] entries currently held
+  std::vector<std::vector<int>> dec_revived_cu;  // [P][n_seqs+1] in-flight rows after each boundary
+  int dec_tag = 0;                         // tag of the latest selection mark
+  bool last_was_decode = false;
   std::map<std::pair<int, int>, std::pair<const int32_t *, int>> forced;  // (point, seq) -> list
   lazy_stats stats;
 

@@ -20,7 +20,9 @@ namespace {
 template <typename T>
 __global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *__restrict__ k,
                                     int ldkv, const int32_t *__restrict__ cu_q,
-                                    const int32_t *__restrict__ kv_base, int n_total, int head_dim,
+                                    const int32_t *__restrict__ kv_base,
+                                    const int32_t *__restrict__ key_rows,
+                                    const int32_t *__restrict__ q_rows, int n_total, int head_dim,
                                     float *__restrict__ logits) {
   constexpr int V = Elem<T>::kPerVec;
   const int seq = blockIdx.z, h = blockIdx.y;
@@ -37,7 +39,8 @@ __global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *_
   float qf[V];
   {
     Vec16<T> qv;
-    qv.load(q + (size_t)(q_start + n - 1) * ldq + h * head_dim + sub * V);
+    const size_t qrow = q_rows ? (size_t)q_rows[seq] : (size_t)(q_start + n - 1);
+    qv.load(q + qrow * ldq + h * head_dim + sub * V);
     qv.unpack(qf);
     const float scale = rsqrtf((float)head_dim);
 #pragma unroll
@@ -51,7 +54,8 @@ __global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *_
     float dot = 0.f;
     if (j < j_end) {
       Vec16<T> kv;
-      kv.load(k + (kb + j) * ldkv + h * head_dim + sub * V);
+      const size_t krow = key_rows ? (size_t)key_rows[q_start + j] : kb + j;
+      kv.load(k + krow * ldkv + h * head_dim + sub * V);
       float kf[V];
       kv.unpack(kf);
 #pragma unroll
@@ -227,6 +231,14 @@ size_t score_scratch_floats(int n_seqs, int n_total, int n_heads) {
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                  const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
                  int n_heads, int head_dim, float *scratch, float *scores) {
+  return launch_score_ex(st, dtype, q, ldq, k, ldkv, cu_q, kv_base, nullptr, nullptr, n_seqs, n_total,
+                         max_len, n_heads, head_dim, scratch, scores);
+}
+
+int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
+                    const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
+                    const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,
+                    int head_dim, float *scratch, float *scores) {
   if (n_total == 0 || n_seqs == 0) return LAZY_OK;
   const int V = dtype == LAZY_F32 ? 4 : 8;
   const int lpk = head_dim / V;
@@ -238,10 +250,12 @@ int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void 
   dim3 grid(cdiv(max_len, keys_per_block), n_heads, n_seqs);
   if (dtype == LAZY_F32)
     score_logits_kernel<float><<<grid, threads, 0, st>>>((const float *)q, ldq, (const float *)k, ldkv,
-                                                         cu_q, kv_base, n_total, head_dim, logits);
+                                                         cu_q, kv_base, key_rows, q_rows, n_total, head_dim,
+                                                         logits);
   else
     score_logits_kernel<bf16><<<grid, threads, 0, st>>>((const bf16 *)q, ldq, (const bf16 *)k, ldkv,
-                                                        cu_q, kv_base, n_total, head_dim, logits);
+                                                        cu_q, kv_base, key_rows, q_rows, n_total, head_dim,
+                                                        logits);
   LAZY_COUNT_LAUNCH();
   score_stats_kernel<<<dim3(n_heads, n_seqs), 256, 0, st>>>(logits, cu_q, n_total, n_heads, stats);
   LAZY_COUNT_LAUNCH();
