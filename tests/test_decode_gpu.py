@@ -1,0 +1,160 @@
+"""Decode step with dynamic re-selection and Aux-Cache revival, against the CPU oracle.
+
+The oracle runs freely; the GPU step is handed the oracle's selected sets at every boundary
+(`lazy_set_forced_keep`), so that logits, revived positions, cache membership and Aux-Cache contents
+are comparable token for token; a second group of tests lets the GPU select by itself.
+Tolerances as in the prefill tests: 2e-2 (bf16) / 1e-4 (fp32) per tensor, indices bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import lazyllm_oracle as O
+from paper_2407_14057_b200 import binding as B
+from paper_2407_14057_b200 import build, synth
+from helpers import rel_err, to_np, weights_to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    B.lib()
+
+
+def _to_cuda(W):
+    out = {k: v.cuda() for k, v in W.items() if k != "layers"}
+    out["layers"] = [{k: v.cuda() for k, v in lw.items()} for lw in W["layers"]]
+    return out
+
+
+def _setup(shape, schedule, lengths, dtype, seed, max_new):
+    bf16 = dtype == torch.bfloat16
+    W = synth.make_weights(shape, seed, bf16=bf16)
+    synth.perturb_gains(W, seed + 50)
+    Wn = weights_to_np(W)
+    ids, cu = synth.make_varlen_batch(shape.vocab, lengths, seed + 1)
+    eng = B.LazyPrefill(shape, _to_cuda(W), schedule, dtype, max_seqs=len(lengths),
+                        max_prompt_tokens=sum(lengths), max_new_tokens=max_new)
+    return Wn, ids, cu, eng
+
+
+def _check_state(eng, states, shape, schedule, tol):
+    """Cache membership, Aux contents and the revival invariant, sequence by sequence."""
+    boundaries = {e - 1 for e, _ in schedule}
+    for s, st in enumerate(states):
+        for l in range(shape.n_layers):
+            kpos, kk, vv = eng.lazy_get_kv(l, s)
+            kpos = to_np(kpos)
+            assert sorted(kpos.tolist()) == sorted(st.layers[l].kv.keys())
+            assert len(set(kpos.tolist())) == len(kpos)              # each token computed once per layer
+            kr, vr = st.layers[l].rows(kpos)
+            assert rel_err(to_np(kk), kr.reshape(len(kpos), -1)) < tol
+            assert rel_err(to_np(vv), vr.reshape(len(kpos), -1)) < tol
+            apos, ahid = eng.lazy_get_aux(l, s)
+            apos = to_np(apos)
+            assert sorted(apos.tolist()) == sorted(st.layers[l].aux.keys())
+            if l not in boundaries:
+                assert len(apos) == 0
+            if len(apos):
+                ref = np.stack([st.layers[l].aux[int(p)] for p in apos])
+                assert rel_err(to_np(ahid), ref) < tol
+
+
+def run_decode_case(shape, schedule, lengths, dtype, seed, steps, forced=True):
+    tol = 1e-4 if dtype == torch.float32 else 2e-2
+    Wn, ids, cu, eng = _setup(shape, schedule, lengths, dtype, seed, max_new=steps)
+    S = len(lengths)
+    logits = torch.empty((S, shape.vocab), dtype=torch.float32, device="cuda")
+    nxt = torch.empty(S, dtype=torch.int32, device="cuda")
+    states = [O.prefill(shape, Wn, to_np(ids)[cu[s]:cu[s + 1]], schedule) for s in range(S)]
+    if forced:
+        for s in range(S):
+            for e, _ in schedule:
+                eng.lazy_set_forced_keep(e, s, torch.tensor(states[s].kept_pos[e], dtype=torch.int32).cuda())
+    eng.lazy_prefill_run(ids.cuda(), cu, logits)
+    eng.lazy_sync_status()
+    for s in range(S):
+        assert rel_err(to_np(logits[s]), states[s].logits) < tol
+    tok = [O.greedy(st.logits) for st in states]
+    revived_total = 0
+    for step in range(steps):
+        ref_logits = [O.decode_step(shape, Wn, states[s], tok[s]) for s in range(S)]
+        if forced:
+            for s in range(S):
+                for e, _ in schedule:
+                    eng.lazy_set_forced_keep(e, s, torch.tensor(states[s].kept_pos[e], dtype=torch.int32).cuda())
+        eng.lazy_decode_step(torch.tensor(tok, dtype=torch.int32).cuda(), logits, nxt)
+        eng.lazy_sync_status()
+        for s in range(S):
+            assert rel_err(to_np(logits[s]), ref_logits[s]) < tol, (step, s)
+            for e, _ in schedule:
+                assert np.array_equal(to_np(eng.lazy_get_kept(e, s)), states[s].kept_pos[e]), (step, s, e)
+                got = sorted(to_np(eng.lazy_get_revived(e, s)).tolist())
+                assert got == sorted(states[s].revived_pos[e].tolist()), (step, s, e)
+                revived_total += len(got)
+            for l in range(shape.n_layers):
+                sc = to_np(eng.lazy_get_scores(l, s))
+                assert sc.shape == states[s].scores[l].shape
+                assert np.max(np.abs(sc - states[s].scores[l])) < 1e-3
+            if dtype == torch.float32:
+                assert int(nxt[s]) == O.greedy(ref_logits[s])
+        _check_state(eng, states, shape, schedule, tol)
+        tok = [O.greedy(l) for l in ref_logits]
+    stats = eng.lazy_get_stats()
+    assert stats.kernel_launches > 0
+    eng.close()
+    return revived_total
+
+
+def test_decode_fp32_tiny_forced_replay():
+    shape = synth.TINY.with_layers(4)
+    rv = run_decode_case(shape, ((1, 7000), (2, 5000), (3, 3000)), [90], torch.float32, seed=1, steps=6)
+    assert rv > 0        # the case exercises revival
+
+
+def test_decode_fp32_free_running_matches_oracle_sets():
+    """fp32 scores differ from the fp64 oracle by ~1e-7: the GPU's own selections coincide."""
+    shape = synth.TINY.with_layers(3)
+    run_decode_case(shape, ((1, 6000), (2, 3000)), [75], torch.float32, seed=2, steps=5, forced=False)
+
+
+def test_decode_fp32_varlen_batch():
+    shape = synth.TINY.with_layers(3)
+    rv = run_decode_case(shape, ((1, 6000), (2, 3000)), [40, 1, 77], torch.float32, seed=3, steps=4)
+    assert rv > 0
+
+
+def test_decode_full_keep_is_standard_kv_cache_decode():
+    shape = synth.TINY
+    rv = run_decode_case(shape, ((1, 10000),), [50], torch.float32, seed=4, steps=3, forced=False)
+    assert rv == 0
+
+
+def test_decode_bf16_small_model():
+    rv = run_decode_case(synth.SMALL, ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16, seed=5, steps=4)
+    assert rv > 0
+
+
+def test_decode_bf16_varlen_batch():
+    run_decode_case(synth.SMALL.with_layers(3), ((1, 6000), (2, 3000)), [130, 65, 200], torch.bfloat16,
+                    seed=6, steps=3)
+
+
+def test_decode_errors():
+    shape = synth.TINY
+    W = _to_cuda(synth.make_weights(shape, 1, bf16=False))
+    eng = B.LazyPrefill(shape, W, synth.SCHEDULE_TINY, torch.float32, 1, 32, max_new_tokens=1)
+    lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+    tok = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_decode_step(tok, lg, None)                # decode before prefill
+    assert e.value.status == -7
+    eng.lazy_prefill_run(synth.make_prompt(shape.vocab, 32, 1).cuda(), [0, 32], lg)
+    eng.lazy_decode_step(tok, lg, None)
+    eng.lazy_sync_status()
+    with pytest.raises(B.LazyError) as e:
+        eng.lazy_decode_step(tok, lg, None)                # caches were sized for one new token
+    assert e.value.status == -3
+    eng.close()
