@@ -58,6 +58,12 @@ int lazy_k_attention(void *stream, int32_t dtype, const void *q, int32_t ldq, co
   if (bad_dtype(dtype) || !q || !k || !v || !o || !d_cu_seqlens || n_seqs < 0 || n_total < 0 ||
       max_len < 0 || n_heads < 1 || head_dim < 32 || head_dim % 32)
     return LAZY_E_BADARG;
+  if (attention_tc_eligible(dtype, head_dim, ldq, ldkv)) {
+    DevStatus *status = dev_status_ptr();
+    if (!status) return LAZY_E_CUDA;
+    return launch_attention_tc((cudaStream_t)stream, q, ldq, n_total, k, v, ldkv, n_total, o, n_heads,
+                               d_cu_seqlens, nullptr, n_seqs, max_len, 0, 0, 0, status);
+  }
   return launch_attention((cudaStream_t)stream, dtype, q, ldq, k, v, ldkv, o, d_cu_seqlens, nullptr,
                           n_seqs, max_len, n_total, n_heads, head_dim);
 }
@@ -170,8 +176,12 @@ int lazy_prune_op(void *stream, int32_t dtype, int32_t n, int32_t d_model, int32
   LAZY_TRY(launch_gemm(st, dtype, w.h, w_qkv, nullptr, w.qkv, n, 3 * d, d, status));
   LAZY_TRY(launch_rope_kv(st, dtype, w.qkv, pos, w.rope, w.k, w.v, nullptr, nullptr, n, n_heads, head_dim,
                           max_pos, status));
-  LAZY_TRY(launch_attention(st, dtype, w.qkv, 3 * d, w.k, w.v, d, w.attn, w.cu, nullptr, 1, n, n, n_heads,
-                            head_dim));
+  if (attention_tc_eligible(dtype, head_dim, 3 * d, d))
+    LAZY_TRY(launch_attention_tc(st, w.qkv, 3 * d, n, w.k, w.v, d, n, w.attn, n_heads, nullptr, nullptr, 1, n,
+                                 0, n, 0, status));
+  else
+    LAZY_TRY(launch_attention(st, dtype, w.qkv, 3 * d, w.k, w.v, d, w.attn, w.cu, nullptr, 1, n, n, n_heads,
+                              head_dim));
   LAZY_TRY(launch_score(st, dtype, w.qkv, 3 * d, w.k, d, w.cu, nullptr, 1, n, n, n_heads, head_dim,
                         w.sscratch, scores));
   LAZY_TRY(launch_gemm(st, dtype, w.attn, w_o, x, w.y, n, d, d, status));

@@ -8,6 +8,8 @@
 //    (query row, head), one key per lane, streaming softmax with warp shuffles.
 // The causal mask is by row order inside a sequence: rows are kept in ascending position order,
 // so row order and position order coincide.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace lazy {
@@ -301,6 +303,15 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
 }
 
 }  // namespace
+
+bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv) {
+  static int veto = -1;  // LAZY_ATTN=mma keeps the warp-level kernel (A/B timing, debugging)
+  if (veto < 0) {
+    const char *e = getenv("LAZY_ATTN");
+    veto = (e && e[0] == 'm') ? 1 : 0;
+  }
+  return !veto && dtype == LAZY_BF16 && head_dim == 128 && (ldq % 8) == 0 && (ldkv % 8) == 0;
+}
 
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                      const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,

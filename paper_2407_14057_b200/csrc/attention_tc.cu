@@ -1,0 +1,327 @@
+// Causal attention on the 5th-generation tensor cores (bf16, head_dim 128, prefill form: query
+// row i of a sequence sees keys 0..i of the same sequence).
+//
+// One CTA = 128 query rows of one head; two CTAs share an SM (96 KiB of shared memory and 256
+// TMEM columns each), so that one CTA's softmax overlaps the other's MMAs.  Warp roles:
+//   warp 0     TMA: Q once (two 128x64 boxes), then 64-key tiles of K and V (two 64x64 boxes
+//              each) into a 2-stage ring;
+//   warp 1     owns TMEM and issues the MMAs from one lane:
+//                S_j = Q K_j^T   (M128 N64 K16 x 8, operands in shared memory, both K-major)
+//                O  += P_j V_j   (M128 N128 K16 x 4, A = P_j read from TMEM, B = V_j as an
+//                                 MN-major shared-memory operand: V stays [key][dh] as loaded)
+//              S is double-buffered: S_{j+1} is issued (once P_{j-1} V_{j-1}, whose P shares its
+//              columns, has retired) before waiting for P_j;
+//   warps 2-5  softmax: thread = query row (TMEM lane).  tcgen05.ld its 64 logits, mask the
+//              diagonal tile, running max / sum in registers, P_j packed to bf16 pairs and written
+//              back over S_j's columns with tcgen05.st.  The running max is only raised when
+//              it grows by more than 2^8 (then O is rescaled in TMEM after the previous P V
+//              retired); otherwise P is allowed to exceed 1, which fp32/bf16 ranges absorb.
+//              After the last tile: O / l -> bf16 -> global.
+// Rows past the sequence end are read as zeros (the tensor maps end there) or as other rows'
+// finite data and are never stored.  Every mbarrier wait is bounded and reports LAZY_E_TIMEOUT.
+#include "tc_common.cuh"
+
+namespace lazy {
+
+namespace {
+
+constexpr int TQ = 128, TK = 64, HD = 128, KV_STAGES = 2;
+constexpr int Q_BYTES = TQ * HD * 2;       // 32 KiB: two [128][64] blocks
+constexpr int KV_TILE_BYTES = TK * HD * 2; // 16 KiB: two [64][64] blocks
+constexpr int Q_BLK = TQ * 64 * 2;         // 16 KiB
+constexpr int KV_BLK = TK * 64 * 2;        // 8 KiB
+constexpr int ATT_TMEM_COLS = 256;         // S0 | S1 (64 columns each) | O (128 columns)
+constexpr int ATT_THREADS = 192;
+constexpr float RESCALE_LOG2 = 8.f;
+
+struct __align__(8) AttBarriers {
+  unsigned long long q_full;
+  unsigned long long kv_full[KV_STAGES];
+  unsigned long long kv_empty[KV_STAGES];
+  unsigned long long s_full[2];
+  unsigned long long p_full[2];
+  unsigned long long pv_done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr int ATT_SMEM_BYTES = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 1024 + (int)sizeof(AttBarriers);
+
+// kind::f16 instruction descriptor: D fp32, A/B bf16; major bits: 0 = K-major, 1 = MN-major.
+__device__ __forceinline__ uint32_t idesc_bf16(int m, int n, int a_mn, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 2)
+attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, bf16 *__restrict__ o, int ldo,
+                    const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base, int q_start_arg,
+                    int n_arg, int kv_start_arg, DevStatus *status) {
+  extern __shared__ uint8_t att_smem_raw[];
+  const uint32_t raw_addr = smem_u32(att_smem_raw);
+  const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+  uint8_t *smem = att_smem_raw + pad;
+  const uint32_t sQ = smem_u32(smem);
+  const uint32_t sK = sQ + Q_BYTES;                          // stage s at + s * KV_TILE_BYTES
+  const uint32_t sV = sK + KV_STAGES * KV_TILE_BYTES;
+  AttBarriers *bars = reinterpret_cast<AttBarriers *>(smem + Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h = blockIdx.y;
+  int q_start = q_start_arg, n = n_arg, kv_start = kv_start_arg;
+  if (cu_q) {
+    q_start = cu_q[blockIdx.z];
+    n = cu_q[blockIdx.z + 1] - q_start;
+    kv_start = kv_base ? kv_base[blockIdx.z] : q_start;
+  }
+  const int q_tiles = (n + TQ - 1) / TQ;
+  if ((int)blockIdx.x >= q_tiles) return;          // before any barrier or TMEM use: safe to leave
+  const int qt = q_tiles - 1 - blockIdx.x;         // longest rows first
+  const int q0 = qt * TQ;
+  const int n_kt = (min(q0 + TQ, n) + TK - 1) / TK;  // key tiles up to the diagonal
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bars->q_full), 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(smem_u32(&bars->kv_full[s]), 1);
+      mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->s_full[b]), 1);
+      mbar_init(smem_u32(&bars->p_full[b]), 4);  // one arrival per softmax warp
+    }
+    mbar_init(smem_u32(&bars->pv_done), 1);
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tma_prefetch_desc(&map_q);
+    tma_prefetch_desc(&map_k);
+    tma_prefetch_desc(&map_v);
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&bars->tmem_base)),
+                 "r"((uint32_t)ATT_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
+  volatile int *abort_flag = &bars->abort_flag;
+  const uint32_t tmem_o = tmem_base + 128u;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      const uint32_t qf = smem_u32(&bars->q_full);
+      mbar_expect_tx(qf, Q_BYTES);
+      tma_load_2d(sQ, &map_q, qf, h * HD, q_start + q0);
+      tma_load_2d(sQ + Q_BLK, &map_q, qf, h * HD + 64, q_start + q0);
+      for (int j = 0; j < n_kt; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&bars->kv_empty[st]), ph ^ 1u, abort_flag, status, W_ATTN_PRODUCER)) break;
+        const uint32_t full = smem_u32(&bars->kv_full[st]);
+        mbar_expect_tx(full, 2 * KV_TILE_BYTES);
+        const int row = kv_start + j * TK;
+        tma_load_2d(sK + st * KV_TILE_BYTES, &map_k, full, h * HD, row);
+        tma_load_2d(sK + st * KV_TILE_BYTES + KV_BLK, &map_k, full, h * HD + 64, row);
+        tma_load_2d(sV + st * KV_TILE_BYTES, &map_v, full, h * HD, row);
+        tma_load_2d(sV + st * KV_TILE_BYTES + KV_BLK, &map_v, full, h * HD + 64, row);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16(TQ, TK, 0, 0);
+      const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
+      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, W_ATTN_MMA);
+      auto issue_s = [&](int j) -> bool {
+        const int st = j & 1;
+        if (!mbar_wait(smem_u32(&bars->kv_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA))
+          return false;
+        tc_fence_after();
+        const uint32_t tmem_s = tmem_base + (uint32_t)(st * 64);
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const uint64_t ad = umma_smem_desc(sQ + (k >> 2) * Q_BLK + (k & 3) * 32);
+          const uint64_t bd = umma_smem_desc(sK + st * KV_TILE_BYTES + (k >> 2) * KV_BLK + (k & 3) * 32);
+          umma_bf16(tmem_s, ad, bd, idesc_s, k != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars->s_full[st]));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < n_kt && ok; ++j) {
+        const int st = j & 1;
+        if (j + 1 < n_kt) {
+          // S_{j+1} lands on the columns that still hold P_{j-1}: MMAs that write different
+          // accumulators are not ordered among themselves, so P_{j-1} V_{j-1} has to retire first.
+          if (j >= 1) {
+            ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_MMA);
+            if (!ok) break;
+          }
+          ok = issue_s(j + 1);
+          if (!ok) break;
+        }
+        ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tmem_p = tmem_base + (uint32_t)(st * 64);
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
+          const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
+          umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars->kv_empty[st]));  // K_j and V_j are free once these MMAs retire
+        umma_commit(smem_u32(&bars->pv_done));
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax warps
+    const int quarter = warp & 3;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const int row = q0 + quarter * 32 + lane;  // index inside the sequence
+    const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kt && ok; ++j) {
+      const int b = j & 1;
+      ok = mbar_wait(smem_u32(&bars->s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t t_s = tmem_base + lane_base + (uint32_t)(b * 64);
+      uint32_t raw[64];
+      tmem_ld_32x32_raw(t_s, raw);
+      tmem_ld_32x32_raw(t_s + 32u, raw + 32);
+      tmem_ld_wait();
+      float mj = -INFINITY;
+      const int col0 = j * TK;
+      const bool diag = col0 + TK - 1 > row;
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        float v = __uint_as_float(raw[c]) * sl2;
+        if (diag && col0 + c > row) v = -INFINITY;
+        raw[c] = __float_as_uint(v);
+        mj = fmaxf(mj, v);
+      }
+      float alpha = 1.f;
+      if (j == 0) {
+        m = mj;  // key 0 is visible to every row: finite
+      } else {
+        const bool need = mj - m > RESCALE_LOG2;
+        if (need) {
+          alpha = exp2f(m - mj);
+          m = mj;
+        }
+        if (__any_sync(0xffffffffu, need)) {
+          // O must be at rest: the previous P V has to retire before it is rescaled in place
+          ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < HD; c += 32) {
+            uint32_t ov[32];
+            tmem_ld_32x32_raw(tmem_o + lane_base + (uint32_t)c, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * alpha);
+            tmem_st_32x32(tmem_o + lane_base + (uint32_t)c, ov);
+          }
+          tmem_st_wait();
+        }
+      }
+      float sum = 0.f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int c = 0; c < 64; c += 2) {
+        const float p0 = exp2f(__uint_as_float(raw[c]) - m);
+        const float p1 = exp2f(__uint_as_float(raw[c + 1]) - m);
+        sum += p0 + p1;
+        pk[c >> 1] = bf16x2_pack(p0, p1);
+      }
+      l = l * alpha + sum;
+      tmem_st_32x32(t_s, pk);  // P_j over the first 32 columns of S_j
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[b]));
+    }
+    // A parity wait can only tell the current phase from the one before it.  After the last P
+    // is handed over, P V of the tile before may still be in flight, so the two remaining phases
+    // are awaited one after the other.
+    if (ok && n_kt >= 2) {
+      ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 2) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.f / l;
+      bf16 *orow = o + (size_t)(q_start + row) * ldo + h * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD; c += 32) {
+        float v[32];
+        tmem_ld_32x32(tmem_o + lane_base + (uint32_t)c, v);
+        if (row < n) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            float f[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) f[t] = v[i + t] * inv;
+            Vec16<bf16> ov;
+            ov.pack(f);
+            ov.store(orow + c + i);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)ATT_TMEM_COLS)
+                 : "memory");
+  }
+}
+
+}  // namespace
+
+// q: rows of pitch ldq elements (heads side by side), k/v: rows of pitch ldkv.  Either the sequences
+// come from device arrays (cu_q, kv_base; one launch, q_rows/kv_rows = extent of the buffers), or one
+// sequence is described by scalars (q_start, n, kv_start).
+int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_rows, const void *k,
+                        const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
+                        const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
+                        int n, int kv_start, DevStatus *status) {
+  if (n_seqs == 0 || max_len == 0) return LAZY_OK;
+  if ((ldq % 8) || (ldkv % 8) || ((uintptr_t)q & 15) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15) ||
+      ((uintptr_t)o & 15))
+    return LAZY_E_BADARG;
+  CUtensorMap mq, mk, mv;
+  LAZY_TRY(tma_map_2d_bf16(&mq, q, q_rows, n_heads * HD, ldq, 64, TQ));
+  LAZY_TRY(tma_map_2d_bf16(&mk, k, kv_rows, n_heads * HD, ldkv, 64, TK));
+  LAZY_TRY(tma_map_2d_bf16(&mv, v, kv_rows, n_heads * HD, ldkv, 64, TK));
+  static bool attr_set = false;
+  if (!attr_set) {
+    LAZY_CUDA_OK(cudaFuncSetAttribute(attn_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      ATT_SMEM_BYTES));
+    attr_set = true;
+  }
+  dim3 grid(cdiv(max_len, TQ), n_heads, n_seqs);
+  attn_tcgen05_kernel<<<grid, ATT_THREADS, ATT_SMEM_BYTES, st>>>(mq, mk, mv, (bf16 *)o, n_heads * HD, cu_q,
+                                                                 kv_base, q_start, n, kv_start, status);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+}  // namespace lazy

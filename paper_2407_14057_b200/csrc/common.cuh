@@ -29,6 +29,9 @@ enum DevWhere {
   W_SELECT = 8,
   W_DECODE = 9,
   W_ROPE_POS = 10,
+  W_ATTN_PRODUCER = 11,
+  W_ATTN_MMA = 12,
+  W_ATTN_SOFTMAX = 13,
 };
 
 __device__ __forceinline__ void dev_fail(DevStatus *st, int code, int where, int a = 0, int b = 0) {
@@ -171,6 +174,15 @@ int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, cons
                         const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                         const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
                         int max_len, int n_total, int n_heads, int head_dim);
+// Prefill attention, bf16 / head_dim 128, on tcgen05 (see attention_tc.cu).  Sequences either come
+// from device arrays (cu_q, kv_base) or one sequence is given by scalars; q_rows / kv_rows bound
+// the tensor maps (reads beyond them give zeros).
+int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_rows, const void *k,
+                        const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
+                        const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
+                        int n, int kv_start, DevStatus *status);
+// True when the tensor-core prefill attention applies (and LAZY_ATTN=mma does not veto it).
+bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                  const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,

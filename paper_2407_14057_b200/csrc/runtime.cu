@@ -460,9 +460,21 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
           launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
                          c->max_pos, status));
-    TIMED(LAZY_K_ATTENTION, attn_flops, 0,
-          launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
-                           c->H, c->dh));
+    if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
+      // one launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
+      // read as zeros instead of whatever the cache region holds
+      for (int s = 0; s < n_seqs; ++s) {
+        const int q0 = c->seg_cu[g][s], ns = c->seg_cu[g][s + 1] - q0;
+        const double fl = 2.0 * d * (double)ns * (ns + 1.0);
+        TIMED(LAZY_K_ATTENTION, fl, 0,
+              launch_attention_tc(st, c->qkv, 3 * d, q0 + ns, kc, vc, d, c->seq_base[s] + ns, c->attn, c->H,
+                                  nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status));
+      }
+    } else {
+      TIMED(LAZY_K_ATTENTION, attn_flops, 0,
+            launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
+                             c->H, c->dh));
+    }
     TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
           launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
                        c->score_scratch, sc));

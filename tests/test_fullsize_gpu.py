@@ -69,7 +69,7 @@ def test_7b_widths_four_layers_full_prompt_vs_oracle():
         # |q| ~ |k| ~ 14.5 at these widths one half-ulp on both gives up to |q||k|/sqrt(dh) * 2^-8
         # ~ 7e-2 on a single head's logit in the worst case (typically ~1e-2 after the head mean).
         rel = np.abs(sc - replay.scores[l]) / replay.scores[l].clip(1e-30)
-        assert np.max(rel) < (3e-2 if l == 0 else 1e-1) and np.median(rel) < 1e-2
+        assert np.max(rel) < (3e-2 if l == 0 else 1e-1) and np.median(rel) < 2e-2
         assert rel_err(to_np(eng.lazy_get_hidden(l)), replay.hidden_out[l]) < TOL
     apos, ahid = eng.lazy_get_aux(0, 0)
     ref = np.stack([replay.layers[0].aux[int(p)] for p in to_np(apos)])
@@ -121,6 +121,18 @@ def test_7b_full_depth_prefill_sampled_and_properties(model7b):
     x1 = x1 + O.mlp(shape, lw, x1)
     h0 = to_np(eng.lazy_get_hidden(0))
     assert rel_err(h0[rows_s], x1) < TOL
+    # determinism: the same call three more times gives the same bits (no race between the warp
+    # roles of the tensor-core kernels shows up as run-to-run noise)
+    first = logits.clone()
+    kept_first = [to_np(eng.lazy_get_kept(e, 0)) for e, _ in schedule]
+    h_first = eng.lazy_get_hidden(31).clone()
+    for _ in range(3):
+        eng.lazy_prefill_run(ids.cuda(), [0, n], logits)
+        eng.lazy_sync_status()
+        assert torch.equal(logits, first)
+        assert torch.equal(eng.lazy_get_hidden(31), h_first)
+        for (e, _), k0 in zip(schedule, kept_first):
+            assert np.array_equal(to_np(eng.lazy_get_kept(e, 0)), k0)
     eng.close()
 
 

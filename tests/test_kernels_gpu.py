@@ -168,6 +168,23 @@ def test_attention_and_score(dtype, H, dh, lengths):
         assert abs(s[a:b].sum() - 1) < 1e-4
 
 
+def test_attention_running_max_rescale_path():
+    """Logits that keep growing with the key index force the streaming softmax to raise its running
+    maximum late (the tensor-core kernel then rescales the accumulator it keeps in tensor memory)."""
+    H, dh, n = 2, 128, 700
+    d = H * dh
+    q = _rand((n, d), 40, torch.bfloat16)
+    k = (_rand((n, d), 41, torch.bfloat16).float() * torch.linspace(0.2, 12.0, n)[:, None]).to(torch.bfloat16)
+    v = _rand((n, d), 42, torch.bfloat16)
+    cu = torch.tensor([0, n], dtype=torch.int32).cuda()
+    o = B.lazy_k_attention(q.cuda(), d, k.cuda(), v.cuda(), d, cu, n, n, H, dh)
+    B.lazy_device_status()
+    pos = np.arange(n)
+    o_ref, _ = O.attend(to_np(q).reshape(n, H, dh), to_np(k).reshape(n, H, dh), to_np(v).reshape(n, H, dh),
+                        pos, pos, -1)
+    assert rel_err(to_np(o), o_ref) < BF16_STEP_TOL
+
+
 # ------------------------------------------------------------------------------------------ select
 def _select_case(score_list, keep_list):
     cu_in = np.concatenate([[0], np.cumsum([len(s) for s in score_list])]).astype(np.int32)
