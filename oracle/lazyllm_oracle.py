@@ -265,6 +265,33 @@ def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]
     return st
 
 
+# --------------------------------------------------------------------------- one layer
+def layer_step(cfg, lw, x, pos, keep_pos: Optional[Sequence[int]] = None):
+    """One decoder layer of the pruned prefill on given inputs (the body of the loop in `prefill`).
+
+    x: [n, d] hidden states entering the layer, pos: [n] their positions (ascending).  If
+    ``keep_pos`` is given, the cut sits after attention: rows whose position is listed go on to the
+    MLP, the others are returned as the layer's Aux rows.  Returns a dict with the Eq. 1 scores, the
+    post-attention hidden states of all rows, the kept positions, the output of the layer for the
+    kept rows and the Aux rows / positions.
+    """
+    x = f64(x)
+    pos = np.asarray(pos).astype(np.int64)
+    q, k, v = _layer_qkv(cfg, lw, x, pos)
+    o, s = attend(q, k, v, pos, pos, -1)
+    y = x + _o_proj(o, lw)
+    if keep_pos is not None:
+        want = set(int(p) for p in keep_pos)
+        keep = np.asarray([r for r in range(len(pos)) if int(pos[r]) in want], dtype=np.int64)
+        drop = np.asarray([r for r in range(len(pos)) if int(pos[r]) not in want], dtype=np.int64)
+    else:
+        keep, drop = np.arange(len(pos)), np.zeros(0, dtype=np.int64)
+    z = y[keep]
+    z = z + mlp(cfg, lw, z)
+    return {"scores": s, "hidden_attn": y, "k": k, "v": v, "pos_out": pos[keep], "hidden_out": z,
+            "aux_rows": y[drop], "aux_pos": pos[drop]}
+
+
 # --------------------------------------------------------------------------- revive
 def revive(st: LazyState, layer: int, positions: Sequence[int], take: bool = False) -> np.ndarray:
     """Hidden states of pruned tokens from the Aux Cache that follows ``layer``.

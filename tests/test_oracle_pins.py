@@ -263,6 +263,22 @@ def test_keep_one_makes_later_attention_the_identity_on_v():
         assert st.scores[l].tolist() == [1.0]
 
 
+def test_layer_step_chain_is_bitwise_the_prefill():
+    """`layer_step` is the loop body of `prefill`: chaining it over the layers, with the kept sets of
+    a prefill run, reproduces that run exactly (so per-layer checks against it mean the same)."""
+    W, ids, pr, full = _pruned_and_full()
+    x = np.asarray(W["tok_embed"], dtype=np.float64)[ids]
+    pos = np.arange(len(ids))
+    for l in range(MINI.n_layers):
+        r = O.layer_step(MINI, W["layers"][l], x, pos, keep_pos=pr.kept_pos.get(l + 1))
+        assert np.array_equal(r["scores"], pr.scores[l])
+        assert np.array_equal(r["hidden_attn"], pr.hidden_after_attn[l])
+        assert np.array_equal(r["hidden_out"], pr.hidden_out[l])
+        assert sorted(pr.layers[l].aux.keys()) == r["aux_pos"].tolist()
+        x, pos = r["hidden_out"], r["pos_out"]
+    assert np.array_equal(O.lm_head(MINI, W, x[-1]), pr.logits)
+
+
 def test_forced_keep_replays_the_same_run():
     W, ids, pr, full = _pruned_and_full()
     again = O.prefill(MINI, W, ids, ((1, 7000), (2, 4000)), forced_keep=dict(pr.kept_pos))
