@@ -3,8 +3,8 @@
 //
 // One CTA = 128 query rows of one head; two CTAs share an SM (96 KiB of shared memory and 256
 // TMEM columns each), so that one CTA's softmax overlaps the other's MMAs.  Warp roles:
-//   warp 0     TMA: Q once (two 128x64 boxes), then 64-key tiles of K and V (two 64x64 boxes
-//              each) into a 2-stage ring;
+//   warp 0     TMA: Q once (two 128x64 boxes), then 64-key tiles of K and of V (two 64x64 boxes
+//              each) into two 2-stage rings with their own barriers (one lane per ring);
 //   warp 1     owns TMEM and issues the MMAs from one lane:
 //                S_j = Q K_j^T   (M128 N64 K16 x 8, operands in shared memory, both K-major)
 //                O  += P_j V_j   (M128 N128 K16 x 4, A = P_j read from TMEM, B = V_j as an
@@ -36,8 +36,10 @@ constexpr float RESCALE_LOG2 = 8.f;
 
 struct __align__(8) AttBarriers {
   unsigned long long q_full;
-  unsigned long long kv_full[KV_STAGES];
-  unsigned long long kv_empty[KV_STAGES];
+  unsigned long long k_full[KV_STAGES];
+  unsigned long long k_empty[KV_STAGES];
+  unsigned long long v_full[KV_STAGES];
+  unsigned long long v_empty[KV_STAGES];
   unsigned long long s_full[2];
   unsigned long long p_full[2];
   unsigned long long pv_done;
@@ -50,6 +52,13 @@ constexpr int ATT_SMEM_BYTES = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 1024 + 
 __device__ __forceinline__ uint32_t idesc_bf16(int m, int n, int a_mn, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// 2^x on the special-function unit; ex2(-inf) = 0.
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 __global__ void __launch_bounds__(ATT_THREADS, 2)
@@ -83,8 +92,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   if (threadIdx.x == 0) {
     mbar_init(smem_u32(&bars->q_full), 1);
     for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(smem_u32(&bars->kv_full[s]), 1);
-      mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+      mbar_init(smem_u32(&bars->k_full[s]), 1);
+      mbar_init(smem_u32(&bars->k_empty[s]), 1);
+      mbar_init(smem_u32(&bars->v_full[s]), 1);
+      mbar_init(smem_u32(&bars->v_empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->s_full[b]), 1);
@@ -112,7 +123,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t tmem_o = tmem_base + 128u;
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
+    // ---------------------------------------------------------------- TMA producers
+    // Lane 0 streams Q and the K tiles, lane 1 the V tiles.  A K stage is free as soon as S_j has
+    // been computed, a V stage once P_j V_j has: K_{j+2} is then in flight long before it is needed.
     if (lane == 0) {
       const uint32_t qf = smem_u32(&bars->q_full);
       mbar_expect_tx(qf, Q_BYTES);
@@ -121,12 +134,21 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       for (int j = 0; j < n_kt; ++j) {
         const int st = j & 1;
         const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&bars->kv_empty[st]), ph ^ 1u, abort_flag, status, W_ATTN_PRODUCER)) break;
-        const uint32_t full = smem_u32(&bars->kv_full[st]);
-        mbar_expect_tx(full, 2 * KV_TILE_BYTES);
+        if (!mbar_wait(smem_u32(&bars->k_empty[st]), ph ^ 1u, abort_flag, status, W_ATTN_PRODUCER)) break;
+        const uint32_t full = smem_u32(&bars->k_full[st]);
+        mbar_expect_tx(full, KV_TILE_BYTES);
         const int row = kv_start + j * TK;
         tma_load_2d(sK + st * KV_TILE_BYTES, &map_k, full, h * HD, row);
         tma_load_2d(sK + st * KV_TILE_BYTES + KV_BLK, &map_k, full, h * HD + 64, row);
+      }
+    } else if (lane == 1) {
+      for (int j = 0; j < n_kt; ++j) {
+        const int st = j & 1;
+        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&bars->v_empty[st]), ph ^ 1u, abort_flag, status, W_ATTN_PRODUCER)) break;
+        const uint32_t full = smem_u32(&bars->v_full[st]);
+        mbar_expect_tx(full, KV_TILE_BYTES);
+        const int row = kv_start + j * TK;
         tma_load_2d(sV + st * KV_TILE_BYTES, &map_v, full, h * HD, row);
         tma_load_2d(sV + st * KV_TILE_BYTES + KV_BLK, &map_v, full, h * HD + 64, row);
       }
@@ -139,7 +161,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, W_ATTN_MMA);
       auto issue_s = [&](int j) -> bool {
         const int st = j & 1;
-        if (!mbar_wait(smem_u32(&bars->kv_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA))
+        if (!mbar_wait(smem_u32(&bars->k_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA))
           return false;
         tc_fence_after();
         const uint32_t tmem_s = tmem_base + (uint32_t)(st * 64);
@@ -149,6 +171,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const uint64_t bd = umma_smem_desc(sK + st * KV_TILE_BYTES + (k >> 2) * KV_BLK + (k & 3) * 32);
           umma_bf16(tmem_s, ad, bd, idesc_s, k != 0 ? 1u : 0u);
         }
+        umma_commit(smem_u32(&bars->k_empty[st]));  // K_j is free once S_j is computed
         umma_commit(smem_u32(&bars->s_full[st]));
         return true;
       };
@@ -167,6 +190,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
         if (!ok) break;
+        ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_p = tmem_base + (uint32_t)(st * 64);
 #pragma unroll
@@ -174,7 +199,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
           umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bars->kv_empty[st]));  // K_j and V_j are free once these MMAs retire
+        umma_commit(smem_u32(&bars->v_empty[st]));  // V_j is free once these MMAs retire
         umma_commit(smem_u32(&bars->pv_done));
       }
     }
@@ -197,23 +222,30 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tmem_ld_32x32_raw(t_s, raw);
       tmem_ld_32x32_raw(t_s + 32u, raw + 32);
       tmem_ld_wait();
-      float mj = -INFINITY;
+      // running maximum on the raw logits (the softmax scale is positive); the mask only matters on
+      // tiles that cross the row's diagonal, so the common tile takes the short path
       const int col0 = j * TK;
-      const bool diag = col0 + TK - 1 > row;
+      if (col0 + TK - 1 > row) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        float v = __uint_as_float(raw[c]) * sl2;
-        if (diag && col0 + c > row) v = -INFINITY;
-        raw[c] = __float_as_uint(v);
-        mj = fmaxf(mj, v);
+        for (int c = 0; c < 64; ++c)
+          if (col0 + c > row) raw[c] = 0xff800000u;  // -inf
       }
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: shorter dependency
+#pragma unroll
+      for (int c = 0; c < 64; c += 4) {
+        mx[0] = fmaxf(mx[0], __uint_as_float(raw[c]));
+        mx[1] = fmaxf(mx[1], __uint_as_float(raw[c + 1]));
+        mx[2] = fmaxf(mx[2], __uint_as_float(raw[c + 2]));
+        mx[3] = fmaxf(mx[3], __uint_as_float(raw[c + 3]));
+      }
+      const float mj = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;  // log2 units
       float alpha = 1.f;
       if (j == 0) {
         m = mj;  // key 0 is visible to every row: finite
       } else {
         const bool need = mj - m > RESCALE_LOG2;
         if (need) {
-          alpha = exp2f(m - mj);
+          alpha = ex2_approx(m - mj);
           m = mj;
         }
         if (__any_sync(0xffffffffu, need)) {
@@ -234,16 +266,24 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tmem_st_wait();
         }
       }
-      float sum = 0.f;
+      // p = 2^(s * scale - m): one FFMA and one ex2 per element
+      float sm[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
+      const float neg_m = -m;
 #pragma unroll
-      for (int c = 0; c < 64; c += 2) {
-        const float p0 = exp2f(__uint_as_float(raw[c]) - m);
-        const float p1 = exp2f(__uint_as_float(raw[c + 1]) - m);
-        sum += p0 + p1;
+      for (int c = 0; c < 64; c += 4) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
+        const float p2 = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
+        const float p3 = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
+        sm[0] += p0;
+        sm[1] += p1;
+        sm[2] += p2;
+        sm[3] += p3;
         pk[c >> 1] = bf16x2_pack(p0, p1);
+        pk[(c >> 1) + 1] = bf16x2_pack(p2, p3);
       }
-      l = l * alpha + sum;
+      l = l * alpha + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
       tmem_st_32x32(t_s, pk);  // P_j over the first 32 columns of S_j
       tmem_st_wait();
       tc_fence_before();
