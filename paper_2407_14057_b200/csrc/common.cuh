@@ -160,6 +160,13 @@ int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const 
                 int M, int N, int K, DevStatus *status);
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
                        void *C, int M, int F, int K, DevStatus *status);
+// QKV projection with the rotary embedding and the K/V cache write in its epilogue (bf16,
+// head_dim 128, d_model a multiple of 256): qkv [M, 3d] receives the rotated q (its k and v thirds
+// are left untouched), rotated k and v go to cache rows kv_row[r] (or r) with their position tag.
+bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
+int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
+                         const float *table, void *kcache, void *vcache, int32_t *kv_pos,
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
 int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
                      const void *R, void *C, int M, int N, int K, int swiglu);
 // Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows

@@ -39,7 +39,19 @@ struct __align__(8) GemmBarriers {
 constexpr int GEMM_SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align slack*/ +
                                 (int)sizeof(GemmBarriers);
 
-enum { EPI_PLAIN = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2 };
+enum { EPI_PLAIN = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_QKV_ROPE = 3 };
+
+// Extra operands of the QKV epilogue: the rotary embedding is applied to the fp32 accumulators and
+// the rotated k, and v, go straight to the layer's cache rows (head_dim 128: one 256-column tile is
+// two whole heads of q, k or v, and a thread holds its row's full heads).
+struct RopeArgs {
+  const int32_t *pos;     // [M] original positions
+  const float2 *table;    // [max_pos][64] (cos, sin)
+  bf16 *kcache, *vcache;  // [rows, d_model]
+  int32_t *kv_pos;        // position tag per cache row (may be NULL)
+  const int32_t *kv_row;  // cache row of GEMM row r (NULL: r)
+  int d_model, max_pos;
+};
 
 // C is [M, ldc]; for EPI_SWIGLU the accumulator's columns [0,128) are gate features and
 // [128,256) the matching up features, and C receives 128 columns per tile.
@@ -48,7 +60,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
                          const __grid_constant__ CUtensorMap map_b0,
                          const __grid_constant__ CUtensorMap map_b1, const bf16 *__restrict__ R,
-                         bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status) {
+                         bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
+                         const RopeArgs rope) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -171,6 +184,69 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       bf16 *crow = C + (size_t)row * ldc;
       const bf16 *rrow = (EPI == EPI_RESIDUAL) ? R + (size_t)row * ldc : nullptr;
+      if (EPI == EPI_QKV_ROPE) {
+        // section of the fused projection this tile belongs to: 0 = q, 1 = k, 2 = v
+        const int sect = n0 / rope.d_model;
+        const int col_in = n0 - sect * rope.d_model;
+        int p = 0;
+        size_t krow = 0;
+        if (row < M) {
+          p = rope.pos[row];
+          if (p < 0 || p >= rope.max_pos) {
+            dev_fail(status, LAZY_E_CAPACITY, W_ROPE_POS, row, p);
+            p = 0;
+          }
+          krow = rope.kv_row ? (size_t)rope.kv_row[row] : (size_t)row;
+        }
+        bf16 *dst = sect == 0 ? crow + n0
+                              : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_model + col_in;
+        if (sect == 2) {
+#pragma unroll 1
+          for (int c = 0; c < BN; c += 32) {
+            float v[32];
+            tmem_ld_32x32(taddr + (uint32_t)c, v);
+            if (row < M) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                Vec16<bf16> o;
+                o.pack(v + j);
+                o.store(dst + c + j);
+              }
+            }
+          }
+        } else {
+          const float2 *tab = rope.table + (size_t)p * 64;
+#pragma unroll 1
+          for (int hc = 0; hc < BN; hc += 128) {  // the two heads of the tile
+#pragma unroll 1
+            for (int o = 0; o < 64; o += 32) {    // pairs (i, i + 64), 32 at a time
+              float lo[32], hi[32];
+              tmem_ld_32x32(taddr + (uint32_t)(hc + o), lo);
+              tmem_ld_32x32(taddr + (uint32_t)(hc + o + 64), hi);
+              if (row < M) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                  const float4 cs = *reinterpret_cast<const float4 *>(tab + o + i);  // two (cos, sin)
+                  const float a0 = lo[i], b0 = hi[i], a1 = lo[i + 1], b1 = hi[i + 1];
+                  lo[i] = a0 * cs.x - b0 * cs.y;
+                  hi[i] = b0 * cs.x + a0 * cs.y;
+                  lo[i + 1] = a1 * cs.z - b1 * cs.w;
+                  hi[i + 1] = b1 * cs.z + a1 * cs.w;
+                }
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  Vec16<bf16> ol, oh;
+                  ol.pack(lo + j);
+                  oh.pack(hi + j);
+                  ol.store(dst + hc + o + j);
+                  oh.store(dst + hc + o + 64 + j);
+                }
+              }
+            }
+          }
+          if (sect == 1 && col_in == 0 && row < M && rope.kv_pos) rope.kv_pos[krow] = p;
+        }
+      } else {
 #pragma unroll 1
       for (int c = 0; c < TILE_N_OUT; c += 32) {
         float v[32];
@@ -204,6 +280,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           }
         }
       }
+      }  // epilogue kinds
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[acc]));
@@ -229,7 +306,7 @@ int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_row
 
 template <int EPI>
 int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C,
-              int M, int N, int K, DevStatus *status) {
+              int M, int N, int K, DevStatus *status, const RopeArgs &rope = RopeArgs()) {
   // TMA needs 16-byte aligned bases and row pitches; the epilogue stores 8 columns at a time.
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
@@ -248,7 +325,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
     attr_set = true;
   }
   kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N,
-                                                  status);
+                                                  status, rope);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
@@ -261,6 +338,26 @@ int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const 
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, B, nullptr, R, C, M, N, K, 0);
   if (R) return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status);
   return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status);
+}
+
+bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {
+  return dtype == LAZY_BF16 && head_dim == 128 && d_model % BN == 0;
+}
+
+int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
+                         const float *table, void *kcache, void *vcache, int32_t *kv_pos,
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status) {
+  if (M == 0) return LAZY_OK;
+  RopeArgs r;
+  r.pos = pos;
+  r.table = (const float2 *)table;
+  r.kcache = (bf16 *)kcache;
+  r.vcache = (bf16 *)vcache;
+  r.kv_pos = kv_pos;
+  r.kv_row = kv_row;
+  r.d_model = d_model;
+  r.max_pos = max_pos;
+  return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, 3 * d_model, d_model, status, r);
 }
 
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,

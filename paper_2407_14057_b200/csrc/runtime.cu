@@ -455,11 +455,18 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       attn_flops += 2.0 * d * ns * (ns + 1.0);
     }
     TIMED(LAZY_K_RMSNORM, 0, 2.0 * n * rb, launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
-    TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
-          launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
-    TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
-          launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
-                         c->max_pos, status));
+    if (gemm_qkv_rope_eligible(dt, d, c->dh)) {
+      // rotary embedding and the K/V cache write ride in the projection's epilogue
+      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
+            launch_gemm_qkv_rope(st, c->h, c->w_qkv[l], c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n,
+                                 d, c->max_pos, status));
+    } else {
+      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
+            launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
+      TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
+            launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
+                           c->max_pos, status));
+    }
     if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
       // one launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
       // read as zeros instead of whatever the cache region holds
