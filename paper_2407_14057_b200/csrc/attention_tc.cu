@@ -54,6 +54,19 @@ __device__ __forceinline__ uint32_t idesc_bf16(int m, int n, int a_mn, int b_mn)
          ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+}  // namespace
+
+// Optional by-product: the last row's softmax numerators, for the Eq. 1 score.
+// p[(seq*H + h)*max_tiles*64 + j] receives 2^(s - m_tile) for key j of the sequence,
+// mtile[(seq*H + h)*max_tiles + t] the reference exponent used in tile t, stats[(seq*H + h)*2 ..] the
+// final (m, 1/l).
+struct AttnScoreOut {
+  float *p, *mtile, *stats;
+  int max_tiles, seq_id;
+};
+
+namespace {
+
 // 2^x on the special-function unit; ex2(-inf) = 0.
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -65,7 +78,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, bf16 *__restrict__ o, int ldo,
                     const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base, int q_start_arg,
-                    int n_arg, int kv_start_arg, DevStatus *status) {
+                    int n_arg, int kv_start_arg, DevStatus *status, const AttnScoreOut sc) {
   extern __shared__ uint8_t att_smem_raw[];
   const uint32_t raw_addr = smem_u32(att_smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -211,6 +224,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
     float m = -INFINITY, l = 0.f;
     bool ok = true;
+    // the thread that owns the sequence's last row also records that row's softmax numerators
+    const bool score_row = sc.p != nullptr && row == n - 1;
+    const bool score_warp = __any_sync(0xffffffffu, score_row);
+    const int seq_id = cu_q ? (int)blockIdx.z : sc.seq_id;
+    // row (seq, h) of P: max_tiles * 64 floats, 16-byte aligned, so whole tiles are stored as float4
+    float *sc_p = score_row ? sc.p + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles * TK : nullptr;
+    float *sc_m = score_row ? sc.mtile + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles : nullptr;
     for (int j = 0; j < n_kt && ok; ++j) {
       const int b = j & 1;
       ok = mbar_wait(smem_u32(&bars->s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
@@ -284,6 +304,21 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         pk[(c >> 1) + 1] = bf16x2_pack(p2, p3);
       }
       l = l * alpha + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
+      if (score_warp) {  // warp-uniform: only the warp that owns the sequence's last row gets here
+        if (score_row) {
+          float4 *dst = reinterpret_cast<float4 *>(sc_p + col0);
+#pragma unroll
+          for (int c = 0; c < 64; c += 4) {
+            float4 pv;
+            pv.x = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
+            pv.y = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
+            pv.z = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
+            pv.w = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
+            dst[c >> 2] = pv;  // keys past the row hold 0 (masked) and land in the row's padding
+          }
+          sc_m[j] = m;
+        }
+      }
       tmem_st_32x32(t_s, pk);  // P_j over the first 32 columns of S_j
       tmem_st_wait();
       tc_fence_before();
@@ -300,6 +335,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (ok) {
       ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
       ok = __all_sync(0xffffffffu, ok);
+    }
+    if (ok && score_row) {
+      float *stt = sc.stats + ((size_t)seq_id * gridDim.y + h) * 2;
+      stt[0] = m;
+      stt[1] = 1.f / l;
     }
     if (ok) {
       tc_fence_after();
@@ -342,7 +382,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_rows, const void *k,
                         const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
                         const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
-                        int n, int kv_start, DevStatus *status) {
+                        int n, int kv_start, DevStatus *status, float *score_scratch, int max_tiles,
+                        int n_seqs_total, int seq_id) {
   if (n_seqs == 0 || max_len == 0) return LAZY_OK;
   if ((ldq % 8) || (ldkv % 8) || ((uintptr_t)q & 15) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15) ||
       ((uintptr_t)o & 15))
@@ -358,8 +399,62 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
     attr_set = true;
   }
   dim3 grid(cdiv(max_len, TQ), n_heads, n_seqs);
+  AttnScoreOut sc = {nullptr, nullptr, nullptr, 0, 0};
+  if (score_scratch) {  // layout: P [S, H, max_tiles*64] | mtile [S, H, max_tiles] | stats [S, H, 2]
+    sc.p = score_scratch;
+    sc.mtile = score_scratch + (size_t)n_seqs_total * n_heads * max_tiles * TK;
+    sc.stats = sc.mtile + (size_t)n_seqs_total * n_heads * max_tiles;
+    sc.max_tiles = max_tiles;
+    sc.seq_id = seq_id;
+  }
   attn_tcgen05_kernel<<<grid, ATT_THREADS, ATT_SMEM_BYTES, st>>>(mq, mk, mv, (bf16 *)o, n_heads * HD, cu_q,
-                                                                 kv_base, q_start, n, kv_start, status);
+                                                                 kv_base, q_start, n, kv_start, status, sc);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+namespace {
+// Eq. 1 from the attention kernel's by-product: s_r = (1/H) sum_h p[h][r] * 2^(m_tile - m_final) / l.
+// Eight lanes share a key row, each summing every eighth head; a fixed shuffle tree adds them up.
+__global__ void score_from_attention_kernel(const float *__restrict__ p, const float *__restrict__ mtile,
+                                            const float *__restrict__ stats, const int32_t *__restrict__ cu_q,
+                                            int n_seqs, int n_total, int n_heads, int max_tiles,
+                                            float *__restrict__ scores) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = t >> 3, part = t & 7;
+  float acc = 0.f;
+  if (r < n_total) {
+    int lo = 0, hi = n_seqs;
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (cu_q[mid] <= r) lo = mid; else hi = mid;
+    }
+    const int j = r - cu_q[lo];
+    const int tile = j / TK;
+#pragma unroll 4
+    for (int h = part; h < n_heads; h += 8) {
+      const size_t sh = (size_t)lo * n_heads + h;
+      acc += p[sh * max_tiles * TK + j] * ex2_approx(mtile[sh * max_tiles + tile] - stats[sh * 2]) * stats[sh * 2 + 1];
+    }
+  }
+  acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+  if (r < n_total && part == 0) scores[r] = acc / (float)n_heads;
+}
+}  // namespace
+
+size_t attn_score_scratch_floats(int n_seqs, int n_heads, int max_tiles) {
+  return (size_t)n_seqs * n_heads * max_tiles * (TK + 1) + (size_t)2 * n_seqs * n_heads;
+}
+
+int launch_score_from_attention(cudaStream_t st, const float *scratch, const int32_t *cu_q, int n_seqs,
+                                int n_total, int n_heads, int max_tiles, float *scores) {
+  if (n_total == 0) return LAZY_OK;
+  const float *mtile = scratch + (size_t)n_seqs * n_heads * max_tiles * TK;
+  const float *stats = mtile + (size_t)n_seqs * n_heads * max_tiles;
+  score_from_attention_kernel<<<cdiv(n_total * 8, 256), 256, 0, st>>>(scratch, mtile, stats, cu_q, n_seqs, n_total,
+                                                                     n_heads, max_tiles, scores);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

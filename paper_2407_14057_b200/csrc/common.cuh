@@ -187,7 +187,14 @@ int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, cons
 int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_rows, const void *k,
                         const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
                         const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
-                        int n, int kv_start, DevStatus *status);
+                        int n, int kv_start, DevStatus *status, float *score_scratch = nullptr,
+                        int max_tiles = 0, int n_seqs_total = 0, int seq_id = 0);
+// With score_scratch (attn_score_scratch_floats floats) the attention kernel also leaves the last
+// row's softmax numerators there; launch_score_from_attention turns them into the Eq. 1 scores.
+// max_tiles = ceil(longest sequence / 64), the same value in both calls.
+size_t attn_score_scratch_floats(int n_seqs, int n_heads, int max_tiles);
+int launch_score_from_attention(cudaStream_t st, const float *scratch, const int32_t *cu_q, int n_seqs,
+                                int n_total, int n_heads, int max_tiles, float *scores);
 // True when the tensor-core prefill attention applies (and LAZY_ATTN=mma does not veto it).
 bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);

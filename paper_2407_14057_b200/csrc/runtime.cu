@@ -154,7 +154,11 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   }
   c->scores = (float *)k.take((size_t)L * KV * 4);
   c->sel_scores = (float *)k.take(R * 4);
-  c->score_scratch = (float *)k.take(score_scratch_floats(c->S, c->cap_kv, c->H) * 4);
+  {
+    size_t a = score_scratch_floats(c->S, c->cap_kv, c->H);
+    size_t b = attn_score_scratch_floats(c->S, c->H, c->cap_rows / 64 + 1);
+    c->score_scratch = (float *)k.take((a > b ? a : b) * 4);
+  }
   c->keep_idx.assign(P, nullptr);
   c->drop_idx.assign(P, nullptr);
   c->aux_dst.assign(P, nullptr);
@@ -467,6 +471,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
             launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
                            c->max_pos, status));
     }
+    bool fused_score = false;
     if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
       // one launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
       // read as zeros instead of whatever the cache region holds
@@ -475,16 +480,22 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
         const double fl = 2.0 * d * (double)ns * (ns + 1.0);
         TIMED(LAZY_K_ATTENTION, fl, 0,
               launch_attention_tc(st, c->qkv, 3 * d, q0 + ns, kc, vc, d, c->seq_base[s] + ns, c->attn, c->H,
-                                  nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status));
+                                  nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status, c->score_scratch,
+                                  cdiv(seg_max, 64), n_seqs, s));
       }
+      // Eq. 1 from the last row's softmax numerators the attention kernel left behind
+      TIMED(LAZY_K_SCORE, 0, 4.0 * c->H * n + 4.0 * n,
+            launch_score_from_attention(st, c->score_scratch, d_cu(g), n_seqs, n, c->H, cdiv(seg_max, 64), sc));
+      fused_score = true;
     } else {
       TIMED(LAZY_K_ATTENTION, attn_flops, 0,
             launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
                              c->H, c->dh));
     }
-    TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
-          launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
-                       c->score_scratch, sc));
+    if (!fused_score)
+      TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
+            launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
+                         c->score_scratch, sc));
     TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status));
 
     const int p = c->point_at[l + 1];
