@@ -1,23 +1,15 @@
 // bf16 GEMM on the 5th-generation tensor cores: C[M,N] = A[M,K] * B[N,K]^T with fp32
 // accumulation in tensor memory (TMEM).
 //
-// One persistent CTA per SM.  Work is counted in 128x256 "half tiles"; every CTA takes an equal,
-// contiguous share of them and runs two vertically adjacent halves as ONE 256x256 tile wherever it
-// can: the two halves share the B tile, so a k-slice costs 64 KiB of shared memory per 2 x 4 MMAs
-// instead of 48 KiB per 4.  Three such stages keep ~3000 tensor-pipe cycles of operands in flight,
-// which is what the L2 -> shared-memory latency under load asks for (a 48 KiB / 4-stage ring of
-// single halves covered 2000 and left the tensor pipe idle a fifth of the time).  A half without
-// a partner (odd count, ragged last rows, or the end of a CTA's share) runs alone, so row padding
-// and wave quantisation stay those of 128-row tiles.  Warp roles:
-//   warp 0      TMA producer: K-slices of A (one or two 128x64 boxes) and B (2 boxes of 128x64)
-//               into the 3-stage ring of 128-byte-swizzled tiles, completion on "full" mbarriers;
-//   warp 1      owns TMEM (512 columns = one 128x256 fp32 accumulator per half) and issues
+// One persistent CTA per SM walks 128x256 output tiles.  Warp roles:
+//   warp 0      TMA producer: K-slices of A (128x64) and B (2 boxes of 128x64) into a 4-stage
+//               ring of 128-byte-swizzled shared-memory tiles, completion on "full" mbarriers;
+//   warp 1      owns TMEM (512 columns = two 128x256 fp32 accumulators) and issues
 //               tcgen05.mma (M128 N256 K16) from one lane; tcgen05.commit releases ring stages
-//               ("empty" barriers) and publishes the finished tile ("tmem full");
-//   warps 2-9   epilogue, four warps per half: tcgen05.ld their 32-lane quarter of the
-//               accumulator, apply the epilogue (plain / + residual / SiLU(gate)*up / RoPE + cache
-//               write), convert to bf16, 16-byte stores.  The producer keeps prefetching the next
-//               tile's first stages meanwhile.
+//               ("empty" barriers) and publishes finished accumulators ("tmem full");
+//   warps 2-5   epilogue: tcgen05.ld their 32-lane quarter of the accumulator, apply the
+//               epilogue (plain / + residual / SiLU(gate)*up), convert to bf16, 16-byte stores.
+// The second accumulator lets the epilogue of tile i overlap the MMAs of tile i+1.
 // Ragged M, N, K rely on TMA zero fill for loads and on predicated stores.
 // Every mbarrier wait is bounded (wall-clock limit); on expiry the kernel records
 // LAZY_E_TIMEOUT in the status word, every role leaves its loop, TMEM is released and the CTA
@@ -28,41 +20,21 @@ namespace lazy {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 3, UMMA_K = 16;
-constexpr int A_HALF_BYTES = BM * BK * 2;        // 16 KiB: the A rows of one half
-constexpr int A_STAGE_BYTES = 2 * A_HALF_BYTES;  // room for both halves
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB
 constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KiB
 constexpr int B_HALF_BYTES = B_STAGE_BYTES / 2;  // one 128-row TMA box
-constexpr int TMEM_COLS = 512;                   // accumulator of half h at columns h * 256
-constexpr int GEMM_THREADS = 320;                // TMA warp, MMA warp, 2 x 4 epilogue warps
+constexpr int NUM_ACC = 2;
+constexpr int TMEM_COLS = 512;
+constexpr int GEMM_THREADS = 192;
 
 struct __align__(8) GemmBarriers {
   unsigned long long full[STAGES];
   unsigned long long empty[STAGES];
-  unsigned long long tmem_full;
-  unsigned long long tmem_empty;
+  unsigned long long tmem_full[NUM_ACC];
+  unsigned long long tmem_empty[NUM_ACC];
   uint32_t tmem_base;
   int abort_flag;
-};
-
-// The CTA's share of half tiles, walked in the same order by every role.  Half u = (column tile
-// u / m_halves, row half u % m_halves); halves 2i and 2i+1 of a column tile pair up.
-struct TileWalk {
-  int u, u_end, m_halves;
-  __device__ TileWalk(int total, int m_halves_) : m_halves(m_halves_) {
-    u = (int)((long long)blockIdx.x * total / gridDim.x);
-    u_end = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
-  }
-  // Next tile: first row, column-tile index, number of halves (1 or 2).  False when done.
-  __device__ bool next(int &m0, int &n_idx, int &halves) {
-    if (u >= u_end) return false;
-    n_idx = u / m_halves;
-    const int mh = u - n_idx * m_halves;
-    m0 = mh * BM;
-    halves = ((mh & 1) == 0 && mh + 1 < m_halves && u + 1 < u_end) ? 2 : 1;
-    u += halves;
-    return true;
-  }
 };
 constexpr int GEMM_SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align slack*/ +
                                 (int)sizeof(GemmBarriers);
@@ -101,9 +73,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Output tiles: columns per tile as seen by the caller.
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
-  const int m_halves = (M + BM - 1) / BM;
+  const int m_tiles = (M + BM - 1) / BM;
   const int n_tiles = (N + TILE_N_OUT - 1) / TILE_N_OUT;
-  const int total_halves = m_halves * n_tiles;
+  const int num_tiles = m_tiles * n_tiles;
   const int num_kb = (K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
@@ -111,8 +83,10 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
-    mbar_init(smem_u32(&bars->tmem_full), 1);
-    mbar_init(smem_u32(&bars->tmem_empty), 8);  // one arrival per epilogue warp
+    for (int a = 0; a < NUM_ACC; ++a) {
+      mbar_init(smem_u32(&bars->tmem_full[a]), 1);
+      mbar_init(smem_u32(&bars->tmem_empty[a]), 4);  // one arrival per epilogue warp
+    }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     tma_prefetch_desc(&map_a);
@@ -138,18 +112,15 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      TileWalk walk(total_halves, m_halves);
-      int m0, n_idx, halves;
-      while (ok && walk.next(m0, n_idx, halves)) {
-        const int n0 = n_idx * TILE_N_OUT;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % m_tiles) * BM;
+        const int n0 = (tile / m_tiles) * TILE_N_OUT;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status, W_GEMM_PRODUCER);
           if (!ok) break;
           const uint32_t full = smem_u32(&bars->full[stage]);
-          mbar_expect_tx(full, halves * A_HALF_BYTES + B_STAGE_BYTES);
-          const uint32_t adst = smem_u32(smem_a + stage * A_STAGE_BYTES);
-          tma_load_2d(adst, &map_a, full, kb * BK, m0);
-          if (halves == 2) tma_load_2d(adst + A_HALF_BYTES, &map_a, full, kb * BK, m0 + BM);
+          mbar_expect_tx(full, A_STAGE_BYTES + B_STAGE_BYTES);
+          tma_load_2d(smem_u32(smem_a + stage * A_STAGE_BYTES), &map_a, full, kb * BK, m0);
           const uint32_t bdst = smem_u32(smem_b + stage * B_STAGE_BYTES);
           if (EPI == EPI_SWIGLU) {
             tma_load_2d(bdst, &map_b0, full, kb * BK, n0);
@@ -168,15 +139,15 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       const uint32_t idesc = umma_idesc_bf16(BM, BN);
       int stage = 0;
       uint32_t phase = 0;
-      uint32_t tile_phase = 0;
+      int local = 0;
       bool ok = true;
-      TileWalk walk(total_halves, m_halves);
-      int m0, n_idx, halves;
-      while (ok && walk.next(m0, n_idx, halves)) {
-        // the accumulators are single-buffered: the previous tile has to be drained first
-        ok = mbar_wait(smem_u32(&bars->tmem_empty), tile_phase ^ 1u, abort_flag, status, W_GEMM_MMA_TMEM);
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        ok = mbar_wait(smem_u32(&bars->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status, W_GEMM_MMA_TMEM);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status, W_GEMM_MMA_FULL);
           if (!ok) break;
@@ -185,38 +156,32 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           const uint32_t b_addr = smem_u32(smem_b + stage * B_STAGE_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t adesc = umma_smem_desc(a_addr + k * UMMA_K * 2);
             const uint64_t bdesc = umma_smem_desc(b_addr + k * UMMA_K * 2);
-            const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-            umma_bf16(tmem_base, umma_smem_desc(a_addr + k * UMMA_K * 2), bdesc, idesc, accum);
-            if (halves == 2)
-              umma_bf16(tmem_base + (uint32_t)BN, umma_smem_desc(a_addr + A_HALF_BYTES + k * UMMA_K * 2), bdesc,
-                        idesc, accum);
+            umma_bf16(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit(smem_u32(&bars->empty[stage]));  // stage reusable once these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(smem_u32(&bars->tmem_full));
-        tile_phase ^= 1u;
+        if (ok) umma_commit(smem_u32(&bars->tmem_full[acc]));
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    const int quarter = warp & 3;        // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
-    const int half = (warp - 2) >> 2;    // which accumulator / which 128 rows of the tile
-    uint32_t tile_phase = 0;
+    const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
+    int local = 0;
     bool ok = true;
-    TileWalk walk(total_halves, m_halves);
-    int m0_tile, n_idx, halves;
-    while (ok && walk.next(m0_tile, n_idx, halves)) {
-      const int n0 = n_idx * TILE_N_OUT;
-      ok = mbar_wait(smem_u32(&bars->tmem_full), tile_phase, abort_flag, status, W_GEMM_EPILOGUE);
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+      const int acc = local & 1;
+      const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+      const int m0 = (tile % m_tiles) * BM;
+      const int n0 = (tile / m_tiles) * TILE_N_OUT;
+      ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      tile_phase ^= 1u;
       tc_fence_after();
-      if (half < halves) {
-      const int row = m0_tile + half * BM + quarter * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(half * BN);
+      const int row = m0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       bf16 *crow = C + (size_t)row * ldc;
       const bf16 *rrow = (EPI == EPI_RESIDUAL) ? R + (size_t)row * ldc : nullptr;
       if (EPI == EPI_QKV_ROPE) {
@@ -316,10 +281,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
         }
       }
       }  // epilogue kinds
-      }  // this warp's half is part of the tile
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty));
+      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[acc]));
     }
   }
 
@@ -352,9 +316,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   LAZY_TRY(make_map(&mb0, B0, N, K, BN / 2));
   LAZY_TRY(make_map(&mb1, B1, N, K, BN / 2));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
-  // one CTA per SM, but never more CTAs than pairs of half tiles (a CTA with one half is fine)
-  const int halves = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
-  const int grid = halves < sm_count() ? halves : sm_count();
+  const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
+  const int grid = tiles < sm_count() ? tiles : sm_count();
   auto kfn = gemm_bf16_tcgen05_kernel<EPI>;
   static bool attr_set = false;
   if (!attr_set) {
