@@ -179,7 +179,9 @@ int lazy_get_stats(lazy_ctx *ctx, lazy_stats *out);
  * CUDA events on the caller's stream; lazy_get_kernel_times synchronises the stream and returns,
  * per kind of step, the summed event time of the latest run together with the ALGORITHMIC work of
  * those launches (floating-point operations for the tensor-core steps, bytes that must move for
- * the memory-bound ones).  Event creation happens inside lazy_set_kernel_timing. */
+ * the memory-bound ones).  Event creation happens inside lazy_set_kernel_timing.  `on`: 0 = off,
+ * 1 = every kind, otherwise a bit set shifted left by one ((1 << LAZY_K_x) << 1 per wanted kind), so
+ * that a single kernel family can be timed without the events of all the small kernels around it. */
 enum {
   LAZY_K_GEMM_QKV = 0, LAZY_K_GEMM_O, LAZY_K_GEMM_GATE_UP, LAZY_K_GEMM_DOWN, LAZY_K_ATTENTION,
   LAZY_K_SCORE, LAZY_K_SELECT, LAZY_K_COMPACT, LAZY_K_RMSNORM, LAZY_K_ROPE_KV, LAZY_K_EMBED,

@@ -291,8 +291,12 @@ class LazyPrefill:
         _check("lazy_get_stats", lib().lazy_get_stats(self.ctx, C.byref(s)))
         return s
 
-    def lazy_set_kernel_timing(self, on: bool) -> None:
-        _check("lazy_set_kernel_timing", lib().lazy_set_kernel_timing(self.ctx, 1 if on else 0))
+    def lazy_set_kernel_timing(self, on, kinds: Optional[Sequence[str]] = None) -> None:
+        """on: bool; kinds: optional names from KERNEL_KINDS to time only those."""
+        arg = 1 if on else 0
+        if on and kinds:
+            arg = sum(1 << KERNEL_KINDS.index(k) for k in kinds) << 1
+        _check("lazy_set_kernel_timing", lib().lazy_set_kernel_timing(self.ctx, arg))
 
     def lazy_get_kernel_times(self) -> Dict[str, Dict[str, float]]:
         t = lazy_kernel_times()

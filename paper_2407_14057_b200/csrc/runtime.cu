@@ -214,7 +214,7 @@ lazy_ctx::~lazy_ctx() {
   for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
 }
 int lazy_ctx::time_begin(cudaStream_t st, int kind, double flops, double bytes) {
-  if (!timing_on) return -1;
+  if (!timing_on || !((timing_mask >> kind) & 1u)) return -1;
   k_flops[kind] += flops;
   k_bytes[kind] += bytes;
   const int slot = (int)ev_kind.size();
@@ -742,6 +742,7 @@ int lazy_get_stats(lazy_ctx *c, lazy_stats *out) {
 int lazy_set_kernel_timing(lazy_ctx *c, int32_t on) {
   if (!c) return LAZY_E_BADARG;
   c->timing_on = on != 0;
+  c->timing_mask = on == 1 ? 0xffffffffu : (uint32_t)on >> 1;  // 1 = every kind, else (kind bits << 1)
   if (on) {  // create the events now so that the timed run itself creates none
     while (c->ev_pool.size() < 2048) {
       cudaEvent_t e;

@@ -73,6 +73,7 @@ struct lazy_ctx {
 
   // ---- optional per-kernel event timing
   bool timing_on = false;
+  uint32_t timing_mask = 0xffffffffu;  // kinds that get an event pair
   std::vector<cudaEvent_t> ev_pool;  // pairs: 2*i start, 2*i+1 stop
   std::vector<int> ev_kind;          // kind of each used pair
   double k_flops[LAZY_N_KERNEL_KINDS], k_bytes[LAZY_N_KERNEL_KINDS];
