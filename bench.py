@@ -26,6 +26,24 @@ WORKLOAD = ("llama2-7b-shape prefill (32 layers, d=4096, 32x128 heads, ffn 11008
             "3376-token prompt, keep 100/70/50/30% entering layers 0/8/16/24")
 
 
+# DRAM traffic of the dominant kernel from the committed ncu capture (profiles/
+# gemm_bf16_tcgen05_2layer_3376.md): mean of dram__bytes_read.sum + dram__bytes_write.sum over the four
+# GEMM launches of one layer.  Only valid for the kernel source it was taken on.
+NCU_GEMM_TRAFFIC_BYTES = 193.4e6
+NCU_GEMM_SOURCE_SHA16 = "cefa092589e64b8c"
+
+
+def _gemm_traffic():
+    import hashlib
+    src = os.path.join(ROOT, "paper_2407_14057_b200", "csrc", "gemm_tcgen05.cu")
+    try:
+        with open(src, "rb") as f:
+            cur = hashlib.sha256(f.read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return NCU_GEMM_TRAFFIC_BYTES if cur == NCU_GEMM_SOURCE_SHA16 else None
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -313,7 +331,8 @@ def run_gpu(args):
         "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel (QKV, O, gate/up+SwiGLU, down)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_kind": f"sustained bf16, {peaks['source']}", "launches_per_step": g_launch,
-                     "ms_per_step": g_ms, "traffic": None},
+                     "ms_per_step": g_ms, "algorithmic_bytes_per_launch": None,
+                     "traffic": _gemm_traffic()},
         "kernels": breakdown,
     }
     if not args.no_cpu:
