@@ -331,7 +331,7 @@ def run_gpu(args):
         "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel (QKV, O, gate/up+SwiGLU, down)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_kind": f"sustained bf16, {peaks['source']}", "launches_per_step": g_launch,
-                     "ms_per_step": g_ms, "algorithmic_bytes_per_launch": None,
+                     "ms_per_step": g_ms, "algorithmic_flops_per_launch": g_fl / max(g_launch, 1),
                      "traffic": _gemm_traffic()},
         "kernels": breakdown,
     }
