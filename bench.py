@@ -186,6 +186,24 @@ def run_reference(args):
     print(json.dumps(out), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ replicas
+def max_over_ranks(ms: float, world: int, device: str) -> float:
+    """Replicas only: no collective touches the data path; the one reduction is this MAX of the
+    per-rank step times, so that the whole job is charged with its slowest replica."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_replica: int, world: int, ms: float) -> float:
+    """Aggregate throughput of `world` independent replicas that each process their own prompt."""
+    return world * tokens_per_replica / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------ GPU leg
 def run_gpu(args):
     import torch
@@ -249,11 +267,7 @@ def run_gpu(args):
         barrier()
         engine.lazy_sync_status()
         engine.lazy_set_kernel_timing(False)
-        ms = e0.elapsed_time(e1) / steps
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1) / steps, world, "cuda")
         return ms, per_kind
 
     sampler = ClockSampler(local)
@@ -285,10 +299,7 @@ def run_gpu(args):
         e2e_step()
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     eng.lazy_sync_status()
 
     if rank != 0:
@@ -313,7 +324,7 @@ def run_gpu(args):
         if v["bytes"] > 0:
             ent["gbs"] = round(v["bytes"] / ksteps / (ms * 1e-3) / 1e9, 1)
         breakdown[k] = ent
-    value = world * n / (ms_pruned * 1e-3)
+    value = whole_job_value(n, world, ms_pruned)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_pruned, "higher_is_better": True, "scaling": "weak",
