@@ -356,6 +356,54 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Timing side of the single-pruning-layer study (Section 4.4): one cut, swept over its location
+    and the fraction kept, plus the "static pruning" point (one early cut) and the progressive
+    schedule.  Prints one JSON object; accuracy needs the datasets and is out of scope."""
+    import torch
+    from paper_2407_14057_b200 import binding as B
+    from paper_2407_14057_b200 import build, synth
+    torch.cuda.set_device(0)
+    build.build()
+    B.lib()
+    shape, n = synth.LLAMA7B, args.prompt
+    W = synth.make_weights(shape, 2, bf16=True, device="cuda")
+    ids = synth.make_prompt(shape.vocab, n, 100).cuda()
+    logits = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+
+    def ttft(schedule):
+        eng = B.LazyPrefill(shape, W, schedule, torch.bfloat16, 1, n)
+        for _ in range(3):
+            eng.lazy_prefill_run(ids, [0, n], logits)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            eng.lazy_prefill_run(ids, [0, n], logits)
+        e1.record()
+        torch.cuda.synchronize()
+        eng.lazy_sync_status()
+        st = eng.lazy_get_stats()
+        rows = [st.rows_computed[l] for l in range(shape.n_layers)]
+        eng.close()
+        return e0.elapsed_time(e1) / args.steps, 100.0 * sum(rows) / (n * shape.n_layers)
+
+    base, _ = ttft(())
+    out = {"workload": f"llama2-7b shape, {n}-token prompt, bf16, 1 GPU", "ttft_ms_full_keep": round(base, 3),
+           "single_cut": [], "schedules": {}}
+    for layer in (4, 8, 12, 16, 20, 24, 28):
+        for keep in (9000, 7000, 5000, 3000, 1000):
+            ms, pct = ttft(((layer, keep),))
+            out["single_cut"].append({"layer_entered": layer, "keep_pct": keep // 100, "ttft_ms": round(ms, 3),
+                                      "speedup": round(base / ms, 3), "token_layers_computed_pct": round(pct, 2)})
+    for name, sched in (("progressive 100/70/50/30 @ 0/8/16/24", synth.SCHEDULE_7B),
+                        ("static: one cut entering layer 2, keep 50%", ((2, 5000),))):
+        ms, pct = ttft(sched)
+        out["schedules"][name] = {"ttft_ms": round(ms, 3), "speedup": round(base / ms, 3),
+                                  "token_layers_computed_pct": round(pct, 2)}
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -365,8 +413,12 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="reduced depth (profiling captures only)")
     ap.add_argument("--prompt", type=int, default=N_PROMPT)
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--sweep", action="store_true",
+                    help="single-cut location x keep-fraction TTFT surface instead of the bench line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
