@@ -9,8 +9,8 @@
 //                S_j = Q K_j^T   (M128 N64 K16 x 8, operands in shared memory, both K-major)
 //                O  += P_j V_j   (M128 N128 K16 x 4, A = P_j read from TMEM, B = V_j as an
 //                                 MN-major shared-memory operand: V stays [key][dh] as loaded)
-//              S is double-buffered: S_{j+1} is issued (after P_{j-1} V_{j-1}, whose P shares its
-//              columns: same issuing thread, in-order tensor pipe) before waiting for P_j;
+//              S is double-buffered: S_{j+1} is issued (once P_{j-1} V_{j-1}, whose P shares its
+//              columns, has retired) before waiting for P_j;
 //   warps 2-5  softmax: thread = query row (TMEM lane).  tcgen05.ld its 64 logits, mask the
 //              diagonal tile, running max / sum in registers, P_j packed to bf16 pairs and written
 //              back over S_j's columns with tcgen05.st.  The running max is only raised when
@@ -192,9 +192,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       for (int j = 0; j < n_kt && ok; ++j) {
         const int st = j & 1;
         if (j + 1 < n_kt) {
-          // S_{j+1} lands on the columns that still hold P_{j-1}.  P_{j-1} V_{j-1} was issued before it
-          // by this same thread and the tensor pipe executes one thread's MMAs in issue order, so the
-          // overwrite cannot overtake the read.
+          // S_{j+1} lands on the columns that still hold P_{j-1}: MMAs that write different
+          // accumulators are not ordered among themselves, so P_{j-1} V_{j-1} has to retire first.
+          if (j >= 1) {
+            ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_MMA);
+            if (!ok) break;
+          }
           ok = issue_s(j + 1);
           if (!ok) break;
         }
