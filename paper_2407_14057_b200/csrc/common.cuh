@@ -167,6 +167,10 @@ bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
+// Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.
+bool gemv_small_m_eligible(int dtype, int M, int K);
+int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
+                        void *C, int M, int N, int K, int swiglu);
 int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
                      const void *R, void *C, int M, int N, int K, int swiglu);
 // Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows

@@ -336,6 +336,7 @@ int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const 
                 int M, int N, int K, DevStatus *status) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, B, nullptr, R, C, M, N, K, 0);
+  if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, B, nullptr, R, C, M, N, K, 0);
   if (R) return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status);
   return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status);
 }
@@ -364,6 +365,7 @@ int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg
                        void *C, int M, int F, int K, DevStatus *status) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
+  if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, Bg, Bu, nullptr, C, M, F, K, 1);
   return launch_tc<EPI_SWIGLU>(st, A, Bg, Bu, nullptr, C, M, F, K, status);
 }
 

@@ -1,0 +1,108 @@
+// Skinny GEMM for decode: C[M,N] = A[M,K] * B[N,K]^T with M <= 4 rows (bf16 storage, fp32
+// accumulation).  At these sizes the step is pure weight streaming, so the kernel is laid out for
+// HBM: every warp owns output columns, reads each weight row exactly once with 16-byte loads
+// (several in flight per lane), keeps the few activation rows in shared memory, and reduces with
+// shuffles.  Same epilogues as the tensor-core GEMM: plain, + residual, SiLU(gate) * up.
+#include "common.cuh"
+
+namespace lazy {
+
+namespace {
+
+constexpr int GV_MAX_M = 4;
+constexpr int GV_THREADS = 256;
+
+template <int M_ROWS, bool SWIGLU>
+__global__ void __launch_bounds__(GV_THREADS)
+gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, const bf16 *__restrict__ B1,
+                    const bf16 *__restrict__ R, bf16 *__restrict__ C, int N, int K) {
+  extern __shared__ uint4 gv_smem[];  // [M_ROWS][K/8] activation rows as 16-byte vectors
+  const int kvec = K >> 3;
+  for (int i = threadIdx.x; i < M_ROWS * kvec; i += GV_THREADS)
+    gv_smem[i] = reinterpret_cast<const uint4 *>(A)[i];
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps_total = gridDim.x * (GV_THREADS / 32);
+  for (int n = blockIdx.x * (GV_THREADS / 32) + warp; n < N; n += warps_total) {
+    const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n * K);
+    const uint4 *w1 = SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n * K) : nullptr;
+    float acc0[M_ROWS], acc1[M_ROWS];
+#pragma unroll
+    for (int m = 0; m < M_ROWS; ++m) acc0[m] = acc1[m] = 0.f;
+#pragma unroll 4
+    for (int v = lane; v < kvec; v += 32) {
+      Vec16<bf16> wv;
+      wv.raw = w0[v];
+      float wf[8], uf[8];
+      wv.unpack(wf);
+      if (SWIGLU) {
+        Vec16<bf16> uv;
+        uv.raw = w1[v];
+        uv.unpack(uf);
+      }
+#pragma unroll
+      for (int m = 0; m < M_ROWS; ++m) {
+        Vec16<bf16> av;
+        av.raw = gv_smem[m * kvec + v];
+        float af[8];
+        av.unpack(af);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          acc0[m] = fmaf(af[i], wf[i], acc0[m]);
+          if (SWIGLU) acc1[m] = fmaf(af[i], uf[i], acc1[m]);
+        }
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < M_ROWS; ++m) {
+      float g = warp_sum(acc0[m]);
+      float u = SWIGLU ? warp_sum(acc1[m]) : 0.f;
+      if (lane == 0) {
+        float out = g;
+        if (SWIGLU) out = g / (1.f + __expf(-g)) * u;
+        else if (R) out += __bfloat162float(R[(size_t)m * N + n]);
+        C[(size_t)m * N + n] = __float2bfloat16_rn(out);
+      }
+    }
+  }
+}
+
+template <int M_ROWS, bool SWIGLU>
+int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C, int N,
+               int K) {
+  const size_t smem = (size_t)M_ROWS * K * 2;
+  auto kfn = gemv_small_m_kernel<M_ROWS, SWIGLU>;
+  LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  int blocks = cdiv(N, GV_THREADS / 32);
+  const int cap = sm_count() * 4;
+  if (blocks > cap) blocks = cap;
+  kfn<<<blocks, GV_THREADS, smem, st>>>((const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R,
+                                       (bf16 *)C, N, K);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+}  // namespace
+
+bool gemv_small_m_eligible(int dtype, int M, int K) {
+  return dtype == LAZY_BF16 && M >= 1 && M <= GV_MAX_M && (K % 8) == 0 && (size_t)M * K * 2 <= 200 * 1024;
+}
+
+int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
+                        void *C, int M, int N, int K, int swiglu) {
+  if (((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15)) return LAZY_E_BADARG;
+#define GV_CASE(m)                                                                      \
+  case m:                                                                               \
+    return swiglu ? launch_one<m, true>(st, A, B0, B1, nullptr, C, N, K)                \
+                  : launch_one<m, false>(st, A, B0, nullptr, R, C, N, K);
+  switch (M) {
+    GV_CASE(1)
+    GV_CASE(2)
+    GV_CASE(3)
+    GV_CASE(4)
+    default: return LAZY_E_BADARG;
+  }
+#undef GV_CASE
+}
+
+}  // namespace lazy

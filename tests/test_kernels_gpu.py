@@ -93,6 +93,24 @@ def test_gemm_fp32(M, N, K):
     assert rel_err(to_np(out), ref) < F32_TOL
 
 
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5])
+def test_gemm_bf16_few_rows_weight_streaming_kernel(M):
+    """M <= 4 takes the weight-streaming kernel, M = 5 the tensor-core one: same answers."""
+    N, K = 4096, 11008
+    A = _rand((M, K), 16, torch.bfloat16)
+    Bm = _rand((N, K), 17, torch.bfloat16, 0.02)
+    R = _rand((M, N), 18, torch.bfloat16)
+    out = B.lazy_k_gemm(A.cuda(), Bm.cuda(), R.cuda())
+    B.lazy_device_status()
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(R))
+    assert rel_err(to_np(out), ref) < BF16_STEP_TOL
+    g = B.lazy_k_gemm_swiglu(A.cuda(), Bm[:1024].contiguous().cuda(), Bm[1024:2048].contiguous().cuda())
+    B.lazy_device_status()
+    a = O.f64(to_np(A))
+    ref = O.silu(a @ O.f64(to_np(Bm[:1024])).T) * (a @ O.f64(to_np(Bm[1024:2048])).T)
+    assert rel_err(to_np(g), ref) < BF16_STEP_TOL
+
+
 @pytest.mark.parametrize("dtype,M,F,K", [(torch.bfloat16, 300, 1408, 512), (torch.bfloat16, 128, 128, 64),
                                          (torch.bfloat16, 77, 688, 256), (torch.bfloat16, 500, 11008, 4096),
                                          (torch.float32, 70, 688, 256)])
