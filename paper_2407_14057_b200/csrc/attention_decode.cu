@@ -1,0 +1,201 @@
+// Attention for a handful of query rows over long key lists (decode: the new token, plus at most
+// a few revived rows).  With one to eight query rows there is nothing for the tensor cores to chew
+// on: the step is a read of the selected K and V rows, so the keys are split across many CTAs
+// (256 keys each), every CTA produces a partial softmax (max, sum, unnormalised output) and a small
+// second kernel merges the partials.  The row of the new token also leaves its logits and final
+// softmax statistics behind, from which the Eq. 1 score is averaged without reading K again.
+// bf16, head_dim 128.  Keys come through a list of cache rows (ascending positions); query row r
+// sees the first q_kvlen[r] entries of its sequence's list.
+#include "common.cuh"
+
+namespace lazy {
+
+namespace {
+
+constexpr int DK_SPLIT = 256;   // keys per CTA
+constexpr int DK_THREADS = 128; // 4 warps; thread t owns output column t
+constexpr int DK_HD = 128;
+constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float ex2f_fast(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ int seq_of_row(const int32_t *cu, int n_seqs, int r) {
+  int lo = 0, hi = n_seqs;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= r) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// grid (n_splits, H, M).  part_o [M, H, n_splits, 128] fp32, part_ml [M, H, n_splits, 2] (max in log2
+// units, sum).  logits (score rows only): [H, n_ctx_total] natural-log units.
+__global__ void __launch_bounds__(DK_THREADS)
+attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
+                           const bf16 *__restrict__ v, int ldkv, const int32_t *__restrict__ cu_x,
+                           const int32_t *__restrict__ cu_ctx, const int32_t *__restrict__ ctx_rows,
+                           const int32_t *__restrict__ q_kvlen, const int32_t *__restrict__ score_row,
+                           int n_seqs, int n_ctx_total, float *__restrict__ part_o,
+                           float *__restrict__ part_ml, float *__restrict__ logits) {
+  __shared__ float sl[DK_SPLIT];
+  __shared__ float red[DK_THREADS / 32];
+  const int split = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
+  const int n_splits = gridDim.x, H = gridDim.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int s = seq_of_row(cu_x, n_seqs, r);
+  const int c0 = cu_ctx[s];
+  const int vis = q_kvlen[r];
+  const int k0 = split * DK_SPLIT;
+  const int cnt = min(DK_SPLIT, vis - k0);
+  const size_t pidx = ((size_t)r * H + h) * n_splits + split;
+  if (cnt <= 0) {  // nothing visible in this split: an empty partial
+    if (threadIdx.x == 0) {
+      part_ml[pidx * 2] = -INFINITY;
+      part_ml[pidx * 2 + 1] = 0.f;
+    }
+    return;
+  }
+  const int32_t *rows = ctx_rows + c0 + k0;
+  // ---- logits: 16 lanes per key (16 bytes each), two keys per warp instruction
+  const int sub = lane & 15, kslot = lane >> 4;
+  float qf[8];
+  {
+    Vec16<bf16> qv;
+    qv.load(q + (size_t)r * ldq + h * DK_HD + sub * 8);
+    qv.unpack(qf);
+    const float sc = rsqrtf((float)DK_HD) * LOG2E;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qf[i] *= sc;
+  }
+  const bool is_score = score_row[s] == r;
+  for (int j0 = warp * 2; j0 < cnt; j0 += (DK_THREADS / 32) * 2) {
+    const int j = j0 + kslot;
+    float dot = 0.f;
+    if (j < cnt) {
+      Vec16<bf16> kv;
+      kv.load(k + (size_t)rows[j] * ldkv + h * DK_HD + sub * 8);
+      float kf[8];
+      kv.unpack(kf);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) dot = fmaf(qf[i], kf[i], dot);
+    }
+    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+    dot += __shfl_xor_sync(0xffffffffu, dot, 8);
+    if (j < cnt && sub == 0) {
+      sl[j] = dot;
+      if (is_score) logits[(size_t)h * n_ctx_total + c0 + k0 + j] = dot * LN2;
+    }
+  }
+  __syncthreads();
+  // ---- partial softmax over the split
+  float m = -INFINITY;
+  for (int j = threadIdx.x; j < cnt; j += DK_THREADS) m = fmaxf(m, sl[j]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  __syncthreads();
+  float sum = 0.f;
+  for (int j = threadIdx.x; j < cnt; j += DK_THREADS) {
+    const float p = ex2f_fast(sl[j] - m);
+    sl[j] = p;
+    sum += p;
+  }
+  sum = warp_sum(sum);
+  if (lane == 0) red[warp] = sum;
+  __syncthreads();
+  sum = (red[0] + red[1]) + (red[2] + red[3]);
+  // ---- unnormalised output: thread t accumulates column t over the split's keys
+  const bf16 *vcol = v + h * DK_HD + threadIdx.x;
+  float acc = 0.f;
+  int j = 0;
+  for (; j + 8 <= cnt; j += 8) {
+    float vv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) vv[i] = __bfloat162float(vcol[(size_t)rows[j + i] * ldkv]);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc = fmaf(sl[j + i], vv[i], acc);
+  }
+  for (; j < cnt; ++j) acc = fmaf(sl[j], __bfloat162float(vcol[(size_t)rows[j] * ldkv]), acc);
+  part_o[pidx * DK_HD + threadIdx.x] = acc;
+  if (threadIdx.x == 0) {
+    part_ml[pidx * 2] = m;
+    part_ml[pidx * 2 + 1] = sum;
+  }
+}
+
+// grid (H, M): merges the splits of one (row, head).  Thread t finishes output column t.  For a score
+// row the final (max, 1/sum) pair goes to stats[(seq*H + h)*2], max in natural-log units.
+__global__ void __launch_bounds__(DK_THREADS)
+attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
+                           int n_splits, const int32_t *__restrict__ cu_x,
+                           const int32_t *__restrict__ score_row, int n_seqs, bf16 *__restrict__ o,
+                           int ldo, float *__restrict__ stats) {
+  const int h = blockIdx.x, r = blockIdx.y, H = gridDim.x;
+  const size_t base = ((size_t)r * H + h) * n_splits;
+  float m = -INFINITY;
+  for (int i = 0; i < n_splits; ++i) m = fmaxf(m, part_ml[(base + i) * 2]);
+  float l = 0.f, acc = 0.f;
+  for (int i = 0; i < n_splits; ++i) {
+    const float li = part_ml[(base + i) * 2 + 1];
+    if (li <= 0.f) continue;  // empty split: its output slot was never written
+    const float w = ex2f_fast(part_ml[(base + i) * 2] - m);
+    l = fmaf(li, w, l);
+    acc = fmaf(part_o[(base + i) * DK_HD + threadIdx.x], w, acc);
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  o[(size_t)r * ldo + h * DK_HD + threadIdx.x] = __float2bfloat16(acc * inv);
+  if (threadIdx.x == 0) {
+    const int s = seq_of_row(cu_x, n_seqs, r);
+    if (score_row[s] == r) {
+      stats[((size_t)s * H + h) * 2] = m * LN2;
+      stats[((size_t)s * H + h) * 2 + 1] = inv;
+    }
+  }
+}
+
+}  // namespace
+
+bool attention_decode_eligible(int dtype, int head_dim, int n_rows) {
+  return dtype == LAZY_BF16 && head_dim == DK_HD && n_rows >= 1 && n_rows <= 8;
+}
+
+size_t attention_decode_scratch_floats(int n_rows, int n_heads, int max_ctx) {
+  const size_t n_splits = (size_t)cdiv(max_ctx > 0 ? max_ctx : 1, DK_SPLIT);
+  return (size_t)n_rows * n_heads * n_splits * (DK_HD + 2);
+}
+
+// q/o: [n_rows, ld] bf16 with head h at columns h*128; k/v: cache rows addressed through ctx_rows.
+// cu_x [n_seqs+1] query rows per sequence, cu_ctx [n_seqs+1] key-list offsets, q_kvlen [n_rows] visible
+// keys per row, score_row [n_seqs] the row whose probabilities feed Eq. 1.  logits [H, n_ctx_total] and
+// stats [n_seqs, H, 2] are outputs for launch_score_mean.  part: attention_decode_scratch_floats().
+int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void *k, const void *v,
+                            int ldkv, void *o, int ldo, const int32_t *cu_x, const int32_t *cu_ctx,
+                            const int32_t *ctx_rows, const int32_t *q_kvlen, const int32_t *score_row,
+                            int n_seqs, int n_rows, int n_ctx_total, int max_ctx, int n_heads,
+                            float *part, float *logits, float *stats) {
+  if (n_rows == 0) return LAZY_OK;
+  if (!q || !k || !v || !o || !cu_x || !cu_ctx || !ctx_rows || !q_kvlen || !score_row || !part ||
+      !logits || !stats)
+    return LAZY_E_BADARG;
+  if (n_rows > 8 || n_seqs < 1 || n_heads < 1 || max_ctx < 1) return LAZY_E_BADARG;
+  const int n_splits = cdiv(max_ctx, DK_SPLIT);
+  float *part_o = part;
+  float *part_ml = part + (size_t)n_rows * n_heads * n_splits * DK_HD;
+  attn_decode_partial_kernel<<<dim3(n_splits, n_heads, n_rows), DK_THREADS, 0, st>>>(
+      (const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v, ldkv, cu_x, cu_ctx, ctx_rows, q_kvlen,
+      score_row, n_seqs, n_ctx_total, part_o, part_ml, logits);
+  LAZY_COUNT_LAUNCH();
+  attn_decode_combine_kernel<<<dim3(n_heads, n_rows), DK_THREADS, 0, st>>>(
+      part_o, part_ml, n_splits, cu_x, score_row, n_seqs, (bf16 *)o, ldo, stats);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+}  // namespace lazy

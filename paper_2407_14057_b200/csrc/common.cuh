@@ -207,6 +207,17 @@ int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void 
                  int n_heads, int head_dim, float *scratch, float *scores);
 // General form (decode): sequence s scores the key LIST key_rows[cu_q[s] .. cu_q[s+1]) (cache rows)
 // with the query in row q_rows[s].
+int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, const int32_t *cu_q,
+                      int n_seqs, int n_total, int n_heads, float *scores);
+// Split-key attention for one to eight query rows over key lists (decode); leaves the score row's
+// logits and softmax statistics for launch_score_mean.
+bool attention_decode_eligible(int dtype, int head_dim, int n_rows);
+size_t attention_decode_scratch_floats(int n_rows, int n_heads, int max_ctx);
+int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void *k, const void *v,
+                            int ldkv, void *o, int ldo, const int32_t *cu_x, const int32_t *cu_ctx,
+                            const int32_t *ctx_rows, const int32_t *q_kvlen, const int32_t *score_row,
+                            int n_seqs, int n_rows, int n_ctx_total, int max_ctx, int n_heads,
+                            float *part, float *logits, float *stats);
 int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                     const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
                     const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,

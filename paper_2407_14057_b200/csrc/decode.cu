@@ -346,12 +346,22 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     KLAUNCH_OK();
     kvlen_kernel<<<cdiv(M, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), xpos, ctx_pos, S, M, q_kvlen);
     KLAUNCH_OK();
-    LAZY_TRY(launch_attention_ex(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), nullptr,
-                                 dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh));
     int max_ctx = 0;
     for (int s = 0; s < S; ++s) max_ctx = ctx_n[s] > max_ctx ? ctx_n[s] : max_ctx;
-    LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
-                             n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
+    // the MLP activation buffer is idle during attention: it holds the split partials
+    if (attention_decode_eligible(dt, c->dh, M) &&
+        attention_decode_scratch_floats(M, c->H, max_ctx) * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
+      float *logits = c->score_scratch, *stats = c->score_scratch + (size_t)c->H * n_ctx;
+      LAZY_TRY(launch_attention_decode(st, c->qkv, 3 * d, kc, vc, d, c->attn, d, dtab(T_CU_X), dtab(T_CU_CTX),
+                                       ctx_rows, q_kvlen, dtab(T_QROW), S, M, n_ctx, max_ctx, c->H,
+                                       (float *)c->act, logits, stats));
+      LAZY_TRY(launch_score_mean(st, logits, stats, dtab(T_CU_CTX), S, n_ctx, c->H, sc));
+    } else {
+      LAZY_TRY(launch_attention_ex(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), nullptr,
+                                   dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh));
+      LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
+                               n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
+    }
     LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status));
 
     const int pt = c->point_at[l + 1];

@@ -265,6 +265,18 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
   return launch_ok();
 }
 
+// Eq. 1 mean over heads from logits [H, n_total] and per-(sequence, head) (max, 1/sum) pairs that
+// another kernel already produced.
+int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, const int32_t *cu_q,
+                      int n_seqs, int n_total, int n_heads, float *scores) {
+  if (n_total == 0) return LAZY_OK;
+  if (!logits || !stats || !cu_q || !scores) return LAZY_E_BADARG;
+  score_mean_kernel<<<cdiv(n_total, 256), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
+                                                        scores);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
                   const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
                   DevStatus *status) {
