@@ -1,7 +1,7 @@
 // Attention for a handful of query rows over long key lists (decode: the new token, plus at most
 // a few revived rows).  With one to eight query rows there is nothing for the tensor cores to chew
 // on: the step is a read of the selected K and V rows, so the keys are split across many CTAs
-// (256 keys each), every CTA produces a partial softmax (max, sum, unnormalised output) and a small
+// (64 keys each), every CTA produces a partial softmax (max, sum, unnormalised output) and a small
 // second kernel merges the partials.  The row of the new token also leaves its logits and final
 // softmax statistics behind, from which the Eq. 1 score is averaged without reading K again.
 // bf16, head_dim 128.  Keys come through a list of cache rows (ascending positions); query row r
@@ -12,9 +12,10 @@ namespace lazy {
 
 namespace {
 
-constexpr int DK_SPLIT = 256;   // keys per CTA
+constexpr int DK_SPLIT = 64;    // keys per CTA
 constexpr int DK_THREADS = 128; // 4 warps; thread t owns output column t
 constexpr int DK_HD = 128;
+static_assert(DK_SPLIT == 64 && DK_THREADS == 128 && DK_HD == 128, "the partial kernel maps 4 warps x 16 keys and 8 groups x 8 keys");
 constexpr float LOG2E = 1.4426950408889634f, LN2 = 0.6931471805599453f;
 
 __device__ __forceinline__ float ex2f_fast(float x) {
@@ -34,6 +35,8 @@ __device__ __forceinline__ int seq_of_row(const int32_t *cu, int n_seqs, int r) 
 
 // grid (n_splits, H, M).  part_o [M, H, n_splits, 128] fp32, part_ml [M, H, n_splits, 2] (max in log2
 // units, sum).  logits (score rows only): [H, n_ctx_total] natural-log units.
+// Every load of a phase is issued before the first use, so one CTA keeps 8 x 16 bytes per thread in
+// flight; 64 keys per CTA put a few thousand CTAs on the machine at a 4096-token context.
 __global__ void __launch_bounds__(DK_THREADS)
 attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
                            const bf16 *__restrict__ v, int ldkv, const int32_t *__restrict__ cu_x,
@@ -41,8 +44,9 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
                            const int32_t *__restrict__ q_kvlen, const int32_t *__restrict__ score_row,
                            int n_seqs, int n_ctx_total, float *__restrict__ part_o,
                            float *__restrict__ part_ml, float *__restrict__ logits) {
+  __shared__ int32_t srow[DK_SPLIT];
   __shared__ float sl[DK_SPLIT];
-  __shared__ float red[DK_THREADS / 32];
+  __shared__ float so[DK_THREADS / 16][DK_HD];
   const int split = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
   const int n_splits = gridDim.x, H = gridDim.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -59,9 +63,11 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
     }
     return;
   }
-  const int32_t *rows = ctx_rows + c0 + k0;
-  // ---- logits: 16 lanes per key (16 bytes each), two keys per warp instruction
-  const int sub = lane & 15, kslot = lane >> 4;
+  if (threadIdx.x < DK_SPLIT) {
+    srow[threadIdx.x] = threadIdx.x < cnt ? ctx_rows[c0 + k0 + threadIdx.x] : -1;
+    sl[threadIdx.x] = -INFINITY;
+  }
+  const int sub = lane & 15, half = lane >> 4;
   float qf[8];
   {
     Vec16<bf16> qv;
@@ -72,58 +78,67 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
     for (int i = 0; i < 8; ++i) qf[i] *= sc;
   }
   const bool is_score = score_row[s] == r;
-  for (int j0 = warp * 2; j0 < cnt; j0 += (DK_THREADS / 32) * 2) {
-    const int j = j0 + kslot;
-    float dot = 0.f;
-    if (j < cnt) {
-      Vec16<bf16> kv;
-      kv.load(k + (size_t)rows[j] * ldkv + h * DK_HD + sub * 8);
-      float kf[8];
-      kv.unpack(kf);
+  __syncthreads();
+  // ---- logits: 16 lanes per key; warp w owns keys w*16 .. w*16+15, two per instruction
+  {
+    Vec16<bf16> kv[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) dot = fmaf(qf[i], kf[i], dot);
+    for (int i = 0; i < 8; ++i) {
+      const int row = srow[warp * 16 + i * 2 + half];
+      if (row >= 0) kv[i].load(k + (size_t)row * ldkv + h * DK_HD + sub * 8);
+      else kv[i].raw = make_uint4(0, 0, 0, 0);
     }
-    dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 4);
-    dot += __shfl_xor_sync(0xffffffffu, dot, 8);
-    if (j < cnt && sub == 0) {
-      sl[j] = dot;
-      if (is_score) logits[(size_t)h * n_ctx_total + c0 + k0 + j] = dot * LN2;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float kf[8], dot = 0.f;
+      kv[i].unpack(kf);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) dot = fmaf(qf[e], kf[e], dot);
+      dot += __shfl_xor_sync(0xffffffffu, dot, 1);
+      dot += __shfl_xor_sync(0xffffffffu, dot, 2);
+      dot += __shfl_xor_sync(0xffffffffu, dot, 4);
+      dot += __shfl_xor_sync(0xffffffffu, dot, 8);
+      const int j = warp * 16 + i * 2 + half;
+      if (sub == 0 && j < cnt) {
+        sl[j] = dot;
+        if (is_score) logits[(size_t)h * n_ctx_total + c0 + k0 + j] = dot * LN2;
+      }
     }
   }
   __syncthreads();
-  // ---- partial softmax over the split
-  float m = -INFINITY;
-  for (int j = threadIdx.x; j < cnt; j += DK_THREADS) m = fmaxf(m, sl[j]);
-  m = warp_max(m);
-  if (lane == 0) red[warp] = m;
-  __syncthreads();
-  m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-  __syncthreads();
-  float sum = 0.f;
-  for (int j = threadIdx.x; j < cnt; j += DK_THREADS) {
-    const float p = ex2f_fast(sl[j] - m);
-    sl[j] = p;
-    sum += p;
-  }
-  sum = warp_sum(sum);
-  if (lane == 0) red[warp] = sum;
-  __syncthreads();
-  sum = (red[0] + red[1]) + (red[2] + red[3]);
-  // ---- unnormalised output: thread t accumulates column t over the split's keys
-  const bf16 *vcol = v + h * DK_HD + threadIdx.x;
-  float acc = 0.f;
-  int j = 0;
-  for (; j + 8 <= cnt; j += 8) {
-    float vv[8];
+  // ---- partial softmax over the split (every warp computes the same max and sum)
+  const float l0 = sl[lane], l1 = sl[lane + 32];
+  const float m = warp_max(fmaxf(l0, l1));
+  const float sum = warp_sum(ex2f_fast(l0 - m) + ex2f_fast(l1 - m));  // ex2(-inf) = 0 past the tail
+  // ---- unnormalised output: group g (16 lanes) takes keys g*8 .. g*8+7, lane takes 8 columns
+  const int g = threadIdx.x >> 4;
+  float acc[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) vv[i] = __bfloat162float(vcol[(size_t)rows[j + i] * ldkv]);
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  {
+    Vec16<bf16> vv[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc = fmaf(sl[j + i], vv[i], acc);
+    for (int i = 0; i < 8; ++i) {
+      const int row = srow[g * 8 + i];
+      if (row >= 0) vv[i].load(v + (size_t)row * ldkv + h * DK_HD + sub * 8);
+      else vv[i].raw = make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float p = ex2f_fast(sl[g * 8 + i] - m);
+      float vf[8];
+      vv[i].unpack(vf);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = fmaf(p, vf[e], acc[e]);
+    }
   }
-  for (; j < cnt; ++j) acc = fmaf(sl[j], __bfloat162float(vcol[(size_t)rows[j] * ldkv]), acc);
-  part_o[pidx * DK_HD + threadIdx.x] = acc;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) so[g][sub * 8 + e] = acc[e];
+  __syncthreads();
+  float o = 0.f;
+#pragma unroll
+  for (int gg = 0; gg < DK_THREADS / 16; ++gg) o += so[gg][threadIdx.x];
+  part_o[pidx * DK_HD + threadIdx.x] = o;
   if (threadIdx.x == 0) {
     part_ml[pidx * 2] = m;
     part_ml[pidx * 2 + 1] = sum;

@@ -54,47 +54,41 @@ __global__ void map_build_kernel(const int32_t *tags, int32_t *map, int base, in
   }
 }
 
-// In-flight rows: cache row they append to, and the position -> row map entry.
-__global__ void dec_rows_kernel(const int32_t *cu_x, const int32_t *seq_base, const int32_t *append_at,
-                                const int32_t *xpos, int n_seqs, int m, int32_t *kv_row_new,
-                                int32_t *kv_map) {
-  int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= m) return;
-  const int s = seq_of(cu_x, n_seqs, r);
-  const int row = append_at[s] + (r - cu_x[s]);
-  kv_row_new[r] = row;
-  kv_map[seq_base[s] + xpos[r]] = row;
-}
-
-// Context list -> cache rows of this layer.
-__global__ void ctx_lookup_kernel(const int32_t *cu_ctx, const int32_t *seq_base, const int32_t *ctx_pos,
-                                  const int32_t *kv_map, int n_seqs, int n, int32_t *ctx_rows,
-                                  DevStatus *status) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const int s = seq_of(cu_ctx, n_seqs, i);
-  int row = kv_map[seq_base[s] + ctx_pos[i]];
-  if (row < 0) {  // a selected token without K/V here would break the subset property
-    dev_fail(status, LAZY_E_STATE, W_DECODE, i, ctx_pos[i]);
-    row = seq_base[s];
+// Per-layer bookkeeping in one launch.  Thread i < m (in-flight rows): the cache row it appends to, its
+// position -> row map entry, and the number of context entries it may see (those with position <= its
+// own).  Thread i < n (context list): the cache row of this layer holding that position.  A position
+// that is in flight gets its row from xmap (the row is being appended by this very step), so no thread
+// depends on a map entry another thread of this launch writes.
+__global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, const int32_t *seq_base,
+                                   const int32_t *append_at, const int32_t *xpos, const int32_t *ctx_pos,
+                                   const int32_t *xmap, int n_seqs, int m, int n, int32_t *kv_row_new,
+                                   int32_t *kv_map, int32_t *q_kvlen, int32_t *ctx_rows, DevStatus *status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    const int s = seq_of(cu_ctx, n_seqs, i);
+    const int p = ctx_pos[i];
+    const int xr = xmap[seq_base[s] + p];
+    int row = xr >= 0 ? append_at[s] + (xr - cu_x[s]) : kv_map[seq_base[s] + p];
+    if (row < 0) {  // a selected token without K/V here would break the subset property
+      dev_fail(status, LAZY_E_STATE, W_DECODE, i, p);
+      row = seq_base[s];
+    }
+    ctx_rows[i] = row;
   }
-  ctx_rows[i] = row;
-}
-
-// Keys visible to an in-flight row = context entries with position <= its own.
-__global__ void kvlen_kernel(const int32_t *cu_x, const int32_t *cu_ctx, const int32_t *xpos,
-                             const int32_t *ctx_pos, int n_seqs, int m, int32_t *q_kvlen) {
-  int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= m) return;
-  const int s = seq_of(cu_x, n_seqs, r);
-  const int32_t *list = ctx_pos + cu_ctx[s];
-  int lo = 0, hi = cu_ctx[s + 1] - cu_ctx[s];  // first index with list[idx] > pos
-  const int p = xpos[r];
-  while (lo < hi) {
-    int mid = (lo + hi) >> 1;
-    if (list[mid] <= p) lo = mid + 1; else hi = mid;
+  if (i < m) {
+    const int s = seq_of(cu_x, n_seqs, i);
+    const int row = append_at[s] + (i - cu_x[s]);
+    const int p = xpos[i];
+    kv_row_new[i] = row;
+    kv_map[seq_base[s] + p] = row;
+    const int32_t *list = ctx_pos + cu_ctx[s];
+    int lo = 0, hi = cu_ctx[s + 1] - cu_ctx[s];  // first index with list[idx] > p
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (list[mid] <= p) lo = mid + 1; else hi = mid;
+    }
+    q_kvlen[i] = lo;
   }
-  q_kvlen[r] = lo;
 }
 
 // xmap[base + pos] = row (or -1 to clear) for the in-flight rows.
@@ -335,17 +329,16 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
 
     LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
     LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status));
-    dec_rows_kernel<<<cdiv(M, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_BASE), dtab(T_APPEND), xpos, S, M,
-                                                  kv_row_new, kvm);
-    KLAUNCH_OK();
+    {
+      const int n_thr = M > n_ctx ? M : n_ctx;
+      dec_prepare_kernel<<<cdiv(n_thr, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), dtab(T_BASE),
+                                                           dtab(T_APPEND), xpos, ctx_pos, xmap, S, M, n_ctx,
+                                                           kv_row_new, kvm, q_kvlen, ctx_rows, status);
+      KLAUNCH_OK();
+    }
     LAZY_TRY(launch_rope_kv(st, dt, c->qkv, xpos, c->rope_table, kc, vc, kvp, kv_row_new, M, c->H, c->dh,
                             c->max_pos, status));
     for (int s = 0; s < S; ++s) c->kv_count[l][s] += m_of[s];
-    ctx_lookup_kernel<<<cdiv(n_ctx, 256), 256, 0, st>>>(dtab(T_CU_CTX), dtab(T_BASE), ctx_pos, kvm, S, n_ctx,
-                                                        ctx_rows, status);
-    KLAUNCH_OK();
-    kvlen_kernel<<<cdiv(M, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), xpos, ctx_pos, S, M, q_kvlen);
-    KLAUNCH_OK();
     int max_ctx = 0;
     for (int s = 0; s < S; ++s) max_ctx = ctx_n[s] > max_ctx ? ctx_n[s] : max_ctx;
     // the MLP activation buffer is idle during attention: it holds the split partials

@@ -12,6 +12,14 @@ namespace {
 constexpr int GV_MAX_M = 4;
 constexpr int GV_THREADS = 256;
 
+// Weights are read once: keep them out of L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+
 template <int M_ROWS, bool SWIGLU>
 __global__ void __launch_bounds__(GV_THREADS)
 gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, const bf16 *__restrict__ B1,
@@ -29,27 +37,42 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
     float acc0[M_ROWS], acc1[M_ROWS];
 #pragma unroll
     for (int m = 0; m < M_ROWS; ++m) acc0[m] = acc1[m] = 0.f;
-#pragma unroll 4
-    for (int v = lane; v < kvec; v += 32) {
-      Vec16<bf16> wv;
-      wv.raw = w0[v];
-      float wf[8], uf[8];
-      wv.unpack(wf);
-      if (SWIGLU) {
-        Vec16<bf16> uv;
-        uv.raw = w1[v];
-        uv.unpack(uf);
+    // U weight vectors per lane are requested before the first is used: 8 x 16 bytes in flight
+    constexpr int U = SWIGLU ? 4 : 8;
+    for (int v0 = lane; v0 < kvec; v0 += 32 * U) {
+      uint4 wr[U], ur[SWIGLU ? U : 1];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int v = v0 + 32 * u;
+        if (v < kvec) {
+          wr[u] = ld_stream(w0 + v);
+          if (SWIGLU) ur[u] = ld_stream(w1 + v);
+        }
       }
 #pragma unroll
-      for (int m = 0; m < M_ROWS; ++m) {
-        Vec16<bf16> av;
-        av.raw = gv_smem[m * kvec + v];
-        float af[8];
-        av.unpack(af);
+      for (int u = 0; u < U; ++u) {
+        const int v = v0 + 32 * u;
+        if (v >= kvec) break;
+        Vec16<bf16> wv;
+        wv.raw = wr[u];
+        float wf[8], uf[8];
+        wv.unpack(wf);
+        if (SWIGLU) {
+          Vec16<bf16> uv;
+          uv.raw = ur[u];
+          uv.unpack(uf);
+        }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          acc0[m] = fmaf(af[i], wf[i], acc0[m]);
-          if (SWIGLU) acc1[m] = fmaf(af[i], uf[i], acc1[m]);
+        for (int m = 0; m < M_ROWS; ++m) {
+          Vec16<bf16> av;
+          av.raw = gv_smem[m * kvec + v];
+          float af[8];
+          av.unpack(af);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            acc0[m] = fmaf(af[i], wf[i], acc0[m]);
+            if (SWIGLU) acc1[m] = fmaf(af[i], uf[i], acc1[m]);
+          }
         }
       }
     }
