@@ -147,25 +147,56 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
 
 // grid (H, M): merges the splits of one (row, head).  Thread t finishes output column t.  For a score
 // row the final (max, 1/sum) pair goes to stats[(seq*H + h)*2], max in natural-log units.
+constexpr int DK_MAX_SPLITS = 2048;  // 131072 keys
 __global__ void __launch_bounds__(DK_THREADS)
 attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                            int n_splits, const int32_t *__restrict__ cu_x,
                            const int32_t *__restrict__ score_row, int n_seqs, bf16 *__restrict__ o,
                            int ldo, float *__restrict__ stats) {
+  __shared__ float sw[DK_MAX_SPLITS];  // weight of each split: 2^(m_i - m), 0 for an empty one
+  __shared__ float red[DK_THREADS / 32];
   const int h = blockIdx.x, r = blockIdx.y, H = gridDim.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t base = ((size_t)r * H + h) * n_splits;
+  const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + base;
   float m = -INFINITY;
-  for (int i = 0; i < n_splits; ++i) m = fmaxf(m, part_ml[(base + i) * 2]);
-  float l = 0.f, acc = 0.f;
-  for (int i = 0; i < n_splits; ++i) {
-    const float li = part_ml[(base + i) * 2 + 1];
-    if (li <= 0.f) continue;  // empty split: its output slot was never written
-    const float w = ex2f_fast(part_ml[(base + i) * 2] - m);
-    l = fmaf(li, w, l);
-    acc = fmaf(part_o[(base + i) * DK_HD + threadIdx.x], w, acc);
+  for (int i = threadIdx.x; i < n_splits; i += DK_THREADS) m = fmaxf(m, ml[i].x);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  __syncthreads();
+  float l = 0.f;
+  for (int i = threadIdx.x; i < n_splits; i += DK_THREADS) {
+    const float2 v = ml[i];
+    const float w = v.y > 0.f ? ex2f_fast(v.x - m) : 0.f;
+    sw[i] = w;
+    l = fmaf(v.y, w, l);
+  }
+  l = warp_sum(l);
+  if (lane == 0) red[warp] = l;
+  __syncthreads();
+  l = (red[0] + red[1]) + (red[2] + red[3]);
+  const float *po = part_o + base * DK_HD + threadIdx.x;
+  float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+  int i = 0;
+  for (; i + 4 <= n_splits; i += 4) {  // an empty split never wrote its slot: do not touch it
+    const float w0 = sw[i], w1 = sw[i + 1], w2 = sw[i + 2], w3 = sw[i + 3];
+    const float v0 = w0 > 0.f ? po[(size_t)i * DK_HD] : 0.f;
+    const float v1 = w1 > 0.f ? po[(size_t)(i + 1) * DK_HD] : 0.f;
+    const float v2 = w2 > 0.f ? po[(size_t)(i + 2) * DK_HD] : 0.f;
+    const float v3 = w3 > 0.f ? po[(size_t)(i + 3) * DK_HD] : 0.f;
+    acc0 = fmaf(v0, w0, acc0);
+    acc1 = fmaf(v1, w1, acc1);
+    acc2 = fmaf(v2, w2, acc2);
+    acc3 = fmaf(v3, w3, acc3);
+  }
+  for (; i < n_splits; ++i) {
+    const float w = sw[i];
+    if (w > 0.f) acc0 = fmaf(po[(size_t)i * DK_HD], w, acc0);
   }
   const float inv = l > 0.f ? 1.f / l : 0.f;
-  o[(size_t)r * ldo + h * DK_HD + threadIdx.x] = __float2bfloat16(acc * inv);
+  o[(size_t)r * ldo + h * DK_HD + threadIdx.x] = __float2bfloat16(((acc0 + acc1) + (acc2 + acc3)) * inv);
   if (threadIdx.x == 0) {
     const int s = seq_of_row(cu_x, n_seqs, r);
     if (score_row[s] == r) {
@@ -177,8 +208,9 @@ attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__rest
 
 }  // namespace
 
-bool attention_decode_eligible(int dtype, int head_dim, int n_rows) {
-  return dtype == LAZY_BF16 && head_dim == DK_HD && n_rows >= 1 && n_rows <= 8;
+bool attention_decode_eligible(int dtype, int head_dim, int n_rows, int max_ctx) {
+  return dtype == LAZY_BF16 && head_dim == DK_HD && n_rows >= 1 && n_rows <= 8 &&
+         max_ctx <= DK_MAX_SPLITS * DK_SPLIT;
 }
 
 size_t attention_decode_scratch_floats(int n_rows, int n_heads, int max_ctx) {
@@ -201,6 +233,7 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
     return LAZY_E_BADARG;
   if (n_rows > 8 || n_seqs < 1 || n_heads < 1 || max_ctx < 1) return LAZY_E_BADARG;
   const int n_splits = cdiv(max_ctx, DK_SPLIT);
+  if (n_splits > DK_MAX_SPLITS) return LAZY_E_CAPACITY;
   float *part_o = part;
   float *part_ml = part + (size_t)n_rows * n_heads * n_splits * DK_HD;
   attn_decode_partial_kernel<<<dim3(n_splits, n_heads, n_rows), DK_THREADS, 0, st>>>(

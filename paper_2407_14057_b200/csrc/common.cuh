@@ -167,10 +167,12 @@ bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
-// Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.
+// Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
+// rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).
 bool gemv_small_m_eligible(int dtype, int M, int K);
 int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
-                        void *C, int M, int N, int K, int swiglu);
+                        void *C, int M, int N, int K, int swiglu, const void *gain = nullptr,
+                        float eps = 0.f, int c_f32 = 0);
 int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
                      const void *R, void *C, int M, int N, int K, int swiglu);
 // Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows
@@ -211,7 +213,7 @@ int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, 
                       int n_seqs, int n_total, int n_heads, float *scores);
 // Split-key attention for one to eight query rows over key lists (decode); leaves the score row's
 // logits and softmax statistics for launch_score_mean.
-bool attention_decode_eligible(int dtype, int head_dim, int n_rows);
+bool attention_decode_eligible(int dtype, int head_dim, int n_rows, int max_ctx);
 size_t attention_decode_scratch_floats(int n_rows, int n_heads, int max_ctx);
 int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void *k, const void *v,
                             int ldkv, void *o, int ldo, const int32_t *cu_x, const int32_t *cu_ctx,

@@ -83,6 +83,7 @@ __global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, c
     kv_map[seq_base[s] + p] = row;
     const int32_t *list = ctx_pos + cu_ctx[s];
     int lo = 0, hi = cu_ctx[s + 1] - cu_ctx[s];  // first index with list[idx] > p
+    if (hi > 0 && list[hi - 1] <= p) lo = hi;    // the new token sees the whole list
     while (lo < hi) {
       const int mid = (lo + hi) >> 1;
       if (list[mid] <= p) lo = mid + 1; else hi = mid;
@@ -327,8 +328,14 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     LAZY_TRY(upload(T_QROW));
     c->stats.rows_computed[l] = M;
 
-    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
-    LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status));
+    // one to four rows: the weight-streaming kernel normalises its input rows itself
+    if (gemv_small_m_eligible(dt, M, d)) {
+      LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, 3 * d, d, 0, c->g_attn[l],
+                                   c->cfg.rms_eps, 0));
+    } else {
+      LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
+      LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status));
+    }
     {
       const int n_thr = M > n_ctx ? M : n_ctx;
       dec_prepare_kernel<<<cdiv(n_thr, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), dtab(T_BASE),
@@ -342,7 +349,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     int max_ctx = 0;
     for (int s = 0; s < S; ++s) max_ctx = ctx_n[s] > max_ctx ? ctx_n[s] : max_ctx;
     // the MLP activation buffer is idle during attention: it holds the split partials
-    if (attention_decode_eligible(dt, c->dh, M) &&
+    if (attention_decode_eligible(dt, c->dh, M, max_ctx) &&
         attention_decode_scratch_floats(M, c->H, max_ctx) * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
       float *logits = c->score_scratch, *stats = c->score_scratch + (size_t)c->H * n_ctx;
       LAZY_TRY(launch_attention_decode(st, c->qkv, 3 * d, kc, vc, d, c->attn, d, dtab(T_CU_X), dtab(T_CU_CTX),
@@ -454,8 +461,13 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
       KLAUNCH_OK();
       c->stats.revived[l + 1] = revived_total;
     }
-    LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
-    LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status));
+    if (gemv_small_m_eligible(dt, M, d)) {
+      LAZY_TRY(launch_gemv_small_m(st, x, c->w_gate[l], c->w_up[l], nullptr, c->act, M, c->F, d, 1, c->g_mlp[l],
+                                   c->cfg.rms_eps, 0));
+    } else {
+      LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
+      LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status));
+    }
     LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status));
   }
   for (int s = 0; s < S; ++s) tab(T_LAST)[s] = tab(T_CU_X)[s + 1] - 1;

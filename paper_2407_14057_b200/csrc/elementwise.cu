@@ -188,7 +188,7 @@ int launch_rope_table(cudaStream_t st, float *table, int max_pos, int head_dim, 
 }
 
 // ---- RoPE + KV-cache write ---------------------------------------------------------------------------
-// One CTA per row of qkv = [q | k | v].  Pairs (i, i + dh/2) of every q and k head are rotated by
+// gridDim.y CTAs per row of qkv = [q | k | v].  Pairs (i, i + dh/2) of every q and k head are rotated by
 // the row's ORIGINAL position; q goes back in place, k and v go to the layer's cache rows.
 template <typename T>
 __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ pos,
@@ -210,7 +210,8 @@ __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ 
   const float2 *tab = table + (size_t)p * half;
   const int vec_per_half = half / V;
   const int pairs = n_heads * vec_per_half;  // vector pairs per q (and per k)
-  for (int t = threadIdx.x; t < 2 * pairs; t += blockDim.x) {
+  const int tid = blockIdx.y * blockDim.x + threadIdx.x, tstep = gridDim.y * blockDim.x;
+  for (int t = tid; t < 2 * pairs; t += tstep) {
     const int which = t / pairs;  // 0 = q, 1 = k
     const int u = t - which * pairs;
     const int h = u / vec_per_half;
@@ -241,20 +242,21 @@ __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ 
   }
   const uint4 *vs = reinterpret_cast<const uint4 *>(row + 2 * d);
   uint4 *vd = reinterpret_cast<uint4 *>(vcache + krow * d);
-  for (int i = threadIdx.x; i < d / V; i += blockDim.x) vd[i] = vs[i];
-  if (threadIdx.x == 0 && kv_pos) kv_pos[krow] = p;
+  for (int i = tid; i < d / V; i += tstep) vd[i] = vs[i];
+  if (tid == 0 && kv_pos) kv_pos[krow] = p;
 }
 
 int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, const float *table,
                    void *kcache, void *vcache, int32_t *kv_pos, const int32_t *kv_row, int n,
                    int n_heads, int head_dim, int max_pos, DevStatus *status) {
   if (n == 0) return LAZY_OK;
+  const dim3 grid(n, n <= 16 ? 8 : 1);  // a handful of rows (decode): spread each over several CTAs
   if (dtype == LAZY_F32)
-    rope_kv_kernel<float><<<n, 128, 0, st>>>((float *)qkv, pos, (const float2 *)table,
+    rope_kv_kernel<float><<<grid, 128, 0, st>>>((float *)qkv, pos, (const float2 *)table,
                                              (float *)kcache, (float *)vcache, kv_pos, kv_row,
                                              n_heads, head_dim, max_pos, status);
   else
-    rope_kv_kernel<bf16><<<n, 128, 0, st>>>((bf16 *)qkv, pos, (const float2 *)table, (bf16 *)kcache,
+    rope_kv_kernel<bf16><<<grid, 128, 0, st>>>((bf16 *)qkv, pos, (const float2 *)table, (bf16 *)kcache,
                                             (bf16 *)vcache, kv_pos, kv_row, n_heads, head_dim,
                                             max_pos, status);
   LAZY_COUNT_LAUNCH();
@@ -345,6 +347,14 @@ __global__ void lm_head_kernel(const T *__restrict__ h, const T *__restrict__ w,
 int launch_lm_head(cudaStream_t st, int dtype, const void *h, const void *w, float *logits,
                    int n_rows, int d, int vocab) {
   if (n_rows == 0) return LAZY_OK;
+  if (gemv_small_m_eligible(dtype, 4, d)) {  // up to four rows per pass over the matrix
+    for (int s0 = 0; s0 < n_rows; s0 += 4) {
+      const int m = n_rows - s0 < 4 ? n_rows - s0 : 4;
+      LAZY_TRY(launch_gemv_small_m(st, (const bf16 *)h + (size_t)s0 * d, w, nullptr, nullptr,
+                                   logits + (size_t)s0 * vocab, m, vocab, d, 0, nullptr, 0.f, 1));
+    }
+    return LAZY_OK;
+  }
   constexpr int SC = 4;
   size_t smem = (size_t)SC * d * sizeof(float);
   int blocks = sm_count() * 2;
@@ -362,35 +372,54 @@ int launch_lm_head(cudaStream_t st, int dtype, const void *h, const void *w, flo
 }
 
 // ---- greedy argmax (ties -> lowest id) ----------------------------------------------------------------------
-__global__ void argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int vocab) {
+constexpr int ARGMAX_THREADS = 1024;
+__global__ void __launch_bounds__(ARGMAX_THREADS)
+argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, int vocab) {
   const float *row = logits + (size_t)blockIdx.x * vocab;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int i = threadIdx.x; i < vocab; i += blockDim.x) {
-    float v = row[i];
+  auto take = [&](float v, int i) {
     if (v > best || (v == best && i < bi)) { best = v; bi = i; }
-  }
-  __shared__ float sv[256];
-  __shared__ int si[256];
-  sv[threadIdx.x] = best;
-  si[threadIdx.x] = bi;
-  __syncthreads();
-  for (int o = blockDim.x / 2; o > 0; o >>= 1) {
-    if (threadIdx.x < o) {
-      float v = sv[threadIdx.x + o];
-      int i = si[threadIdx.x + o];
-      if (v > sv[threadIdx.x] || (v == sv[threadIdx.x] && i < si[threadIdx.x])) {
-        sv[threadIdx.x] = v;
-        si[threadIdx.x] = i;
-      }
+  };
+  if ((((uintptr_t)row) & 15) == 0) {
+    const int nv = vocab >> 2;
+    for (int i = threadIdx.x; i < nv; i += ARGMAX_THREADS) {
+      const float4 v = reinterpret_cast<const float4 *>(row)[i];
+      take(v.x, 4 * i); take(v.y, 4 * i + 1); take(v.z, 4 * i + 2); take(v.w, 4 * i + 3);
     }
-    __syncthreads();
+    for (int i = 4 * nv + threadIdx.x; i < vocab; i += ARGMAX_THREADS) take(row[i], i);
+  } else {
+    for (int i = threadIdx.x; i < vocab; i += ARGMAX_THREADS) take(row[i], i);
   }
-  if (threadIdx.x == 0) out[blockIdx.x] = si[0] == 0x7fffffff ? 0 : si[0];
+  // warp, then CTA: larger value wins, equal values go to the lower id
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float v = __shfl_xor_sync(0xffffffffu, best, o);
+    const int i = __shfl_xor_sync(0xffffffffu, bi, o);
+    take(v, i);
+  }
+  __shared__ float sv[ARGMAX_THREADS / 32];
+  __shared__ int si[ARGMAX_THREADS / 32];
+  if ((threadIdx.x & 31) == 0) {
+    sv[threadIdx.x >> 5] = best;
+    si[threadIdx.x >> 5] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    best = sv[threadIdx.x];
+    bi = si[threadIdx.x];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float v = __shfl_xor_sync(0xffffffffu, best, o);
+      const int i = __shfl_xor_sync(0xffffffffu, bi, o);
+      take(v, i);
+    }
+    if (threadIdx.x == 0) out[blockIdx.x] = bi == 0x7fffffff ? 0 : bi;
+  }
 }
 int launch_argmax(cudaStream_t st, const float *logits, int32_t *out, int n_rows, int vocab) {
   if (n_rows == 0) return LAZY_OK;
-  argmax_kernel<<<n_rows, 256, 0, st>>>(logits, out, vocab);
+  argmax_kernel<<<n_rows, ARGMAX_THREADS, 0, st>>>(logits, out, vocab);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

@@ -23,13 +23,53 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
 template <int M_ROWS, bool SWIGLU>
 __global__ void __launch_bounds__(GV_THREADS)
 gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, const bf16 *__restrict__ B1,
-                    const bf16 *__restrict__ R, bf16 *__restrict__ C, int N, int K) {
+                    const bf16 *__restrict__ R, void *__restrict__ C, int N, int K,
+                    const bf16 *__restrict__ gain, float eps, int c_f32) {
   extern __shared__ uint4 gv_smem[];  // [M_ROWS][K/8] activation rows as 16-byte vectors
+  __shared__ float gv_red[M_ROWS][GV_THREADS / 32];
   const int kvec = K >> 3;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int i = threadIdx.x; i < M_ROWS * kvec; i += GV_THREADS)
     gv_smem[i] = reinterpret_cast<const uint4 *>(A)[i];
   __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (gain) {  // RMSNorm of the rows on the way in: a = bf16(x * rsqrt(mean(x^2) + eps) * gain)
+    float ss[M_ROWS];
+#pragma unroll
+    for (int m = 0; m < M_ROWS; ++m) {
+      ss[m] = 0.f;
+      for (int v = threadIdx.x; v < kvec; v += GV_THREADS) {
+        Vec16<bf16> xv;
+        xv.raw = gv_smem[m * kvec + v];
+        float f[8];
+        xv.unpack(f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss[m] = fmaf(f[i], f[i], ss[m]);
+      }
+      ss[m] = warp_sum(ss[m]);
+      if (lane == 0) gv_red[m][warp] = ss[m];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < M_ROWS; ++m) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < GV_THREADS / 32; ++w) tot += gv_red[m][w];
+      const float scale = rsqrtf(tot / (float)K + eps);
+      for (int v = threadIdx.x; v < kvec; v += GV_THREADS) {
+        Vec16<bf16> xv, gv;
+        xv.raw = gv_smem[m * kvec + v];
+        gv.raw = reinterpret_cast<const uint4 *>(gain)[v];
+        float f[8], gf[8];
+        xv.unpack(f);
+        gv.unpack(gf);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = f[i] * scale * gf[i];
+        xv.pack(f);
+        gv_smem[m * kvec + v] = xv.raw;
+      }
+    }
+    __syncthreads();
+  }
   const int warps_total = gridDim.x * (GV_THREADS / 32);
   for (int n = blockIdx.x * (GV_THREADS / 32) + warp; n < N; n += warps_total) {
     const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n * K);
@@ -84,7 +124,8 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
         float out = g;
         if (SWIGLU) out = g / (1.f + __expf(-g)) * u;
         else if (R) out += __bfloat162float(R[(size_t)m * N + n]);
-        C[(size_t)m * N + n] = __float2bfloat16_rn(out);
+        if (c_f32) reinterpret_cast<float *>(C)[(size_t)m * N + n] = out;
+        else reinterpret_cast<bf16 *>(C)[(size_t)m * N + n] = __float2bfloat16_rn(out);
       }
     }
   }
@@ -92,15 +133,15 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
 
 template <int M_ROWS, bool SWIGLU>
 int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C, int N,
-               int K) {
+               int K, const void *gain, float eps, int c_f32) {
   const size_t smem = (size_t)M_ROWS * K * 2;
   auto kfn = gemv_small_m_kernel<M_ROWS, SWIGLU>;
   LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int blocks = cdiv(N, GV_THREADS / 32);
   const int cap = sm_count() * 4;
   if (blocks > cap) blocks = cap;
-  kfn<<<blocks, GV_THREADS, smem, st>>>((const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R,
-                                       (bf16 *)C, N, K);
+  kfn<<<blocks, GV_THREADS, smem, st>>>((const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R, C,
+                                       N, K, (const bf16 *)gain, eps, c_f32);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
@@ -111,13 +152,16 @@ bool gemv_small_m_eligible(int dtype, int M, int K) {
   return dtype == LAZY_BF16 && M >= 1 && M <= GV_MAX_M && (K % 8) == 0 && (size_t)M * K * 2 <= 200 * 1024;
 }
 
+// gain != NULL: the rows of A are RMS-normalised (gain, eps) before the product, with the rounding a
+// separate normalisation kernel writing bf16 would have had.  c_f32: C holds fp32 instead of bf16.
 int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
-                        void *C, int M, int N, int K, int swiglu) {
-  if (((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15)) return LAZY_E_BADARG;
-#define GV_CASE(m)                                                                      \
-  case m:                                                                               \
-    return swiglu ? launch_one<m, true>(st, A, B0, B1, nullptr, C, N, K)                \
-                  : launch_one<m, false>(st, A, B0, nullptr, R, C, N, K);
+                        void *C, int M, int N, int K, int swiglu, const void *gain, float eps, int c_f32) {
+  if (((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) || ((uintptr_t)gain & 15))
+    return LAZY_E_BADARG;
+#define GV_CASE(m)                                                                            \
+  case m:                                                                                     \
+    return swiglu ? launch_one<m, true>(st, A, B0, B1, nullptr, C, N, K, gain, eps, c_f32)    \
+                  : launch_one<m, false>(st, A, B0, nullptr, R, C, N, K, gain, eps, c_f32);
   switch (M) {
     GV_CASE(1)
     GV_CASE(2)

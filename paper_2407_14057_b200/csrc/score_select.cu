@@ -95,21 +95,27 @@ __global__ void score_stats_kernel(const float *__restrict__ logits, const int32
   }
 }
 
+// 8 lanes per key, each over a slice of the heads.
 __global__ void score_mean_kernel(const float *__restrict__ logits, const float *__restrict__ stats,
                                   const int32_t *__restrict__ cu_q, int n_seqs, int n_total,
                                   int n_heads, float *__restrict__ scores) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= n_total) return;
-  int lo = 0, hi = n_seqs;
-  while (hi - lo > 1) {
-    int mid = (lo + hi) >> 1;
-    if (cu_q[mid] <= r) lo = mid; else hi = mid;
-  }
-  const float *st = stats + (size_t)lo * n_heads * 2;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  const int r = t >> 3, sub = t & 7;
   float acc = 0.f;
-  for (int h = 0; h < n_heads; ++h)
-    acc += __expf(logits[(size_t)h * n_total + r] - st[2 * h]) * st[2 * h + 1];
-  scores[r] = acc / (float)n_heads;
+  if (r < n_total) {
+    int lo = 0, hi = n_seqs;
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (cu_q[mid] <= r) lo = mid; else hi = mid;
+    }
+    const float *st = stats + (size_t)lo * n_heads * 2;
+    for (int h = sub; h < n_heads; h += 8)
+      acc += __expf(logits[(size_t)h * n_total + r] - st[2 * h]) * st[2 * h + 1];
+  }
+  acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+  acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+  if (r < n_total && sub == 0) scores[r] = acc / (float)n_heads;
 }
 
 // ------------------------------------------------------------------------------------------ select
@@ -259,7 +265,7 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
   LAZY_COUNT_LAUNCH();
   score_stats_kernel<<<dim3(n_heads, n_seqs), 256, 0, st>>>(logits, cu_q, n_total, n_heads, stats);
   LAZY_COUNT_LAUNCH();
-  score_mean_kernel<<<cdiv(n_total, 256), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
+  score_mean_kernel<<<cdiv(n_total, 32), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
                                                         scores);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
@@ -271,7 +277,7 @@ int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, 
                       int n_seqs, int n_total, int n_heads, float *scores) {
   if (n_total == 0) return LAZY_OK;
   if (!logits || !stats || !cu_q || !scores) return LAZY_E_BADARG;
-  score_mean_kernel<<<cdiv(n_total, 256), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
+  score_mean_kernel<<<cdiv(n_total, 32), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
                                                         scores);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
