@@ -291,6 +291,15 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
   }
   if (n_ctx > KV) return LAZY_E_CAPACITY;
   LAZY_TRY(upload(T_CU_X));
+  // Where each layer's cache appends this step is known up front (one table per layer, one copy); the
+  // score row only moves when the in-flight set changes.
+  std::vector<int32_t> h_append((size_t)L * W, 0);
+  for (int l = 0; l < L; ++l)
+    for (int s = 0; s < S; ++s) h_append[(size_t)l * W + s] = c->seq_base[s] + c->kv_count[l][s];
+  int32_t *d_append = tabs + (size_t)2 * T_N * W;
+  LAZY_CUDA_OK(cudaMemcpyAsync(d_append, h_append.data(), h_append.size() * 4, cudaMemcpyHostToDevice, st));
+  for (int s = 0; s < S; ++s) tab(T_QROW)[s] = tab(T_CU_X)[s + 1] - 1;  // the new token: largest position
+  LAZY_TRY(upload(T_QROW));
   LAZY_TRY(upload(T_CU_CTX));
   LAZY_TRY(upload(T_BASE));
   LAZY_TRY(upload(T_P));
@@ -318,14 +327,10 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     float *sc = c->scores + (size_t)l * KV;
     int max_m = 0;
     for (int s = 0; s < S; ++s) {
-      tab(T_APPEND)[s] = c->seq_base[s] + c->kv_count[l][s];
-      tab(T_QROW)[s] = tab(T_CU_X)[s + 1] - 1;  // the new token has the largest position in flight
       if (c->kv_count[l][s] + m_of[s] > c->prompt_len[s] + c->cfg.max_new_tokens) return LAZY_E_CAPACITY;
       if (m_of[s] > max_m) max_m = m_of[s];
     }
     if (M > c->cap_rows) return LAZY_E_CAPACITY;
-    LAZY_TRY(upload(T_APPEND));
-    LAZY_TRY(upload(T_QROW));
     c->stats.rows_computed[l] = M;
 
     // one to four rows: the weight-streaming kernel normalises its input rows itself
@@ -339,7 +344,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     {
       const int n_thr = M > n_ctx ? M : n_ctx;
       dec_prepare_kernel<<<cdiv(n_thr, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), dtab(T_BASE),
-                                                           dtab(T_APPEND), xpos, ctx_pos, xmap, S, M, n_ctx,
+                                                           d_append + (size_t)l * W, xpos, ctx_pos, xmap, S, M, n_ctx,
                                                            kv_row_new, kvm, q_kvlen, ctx_rows, status);
       KLAUNCH_OK();
     }
@@ -457,6 +462,8 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
       LAZY_CUDA_OK(cudaMemcpyAsync(c->revived_pos[pt], revived, (size_t)m_new * 4, cudaMemcpyDeviceToDevice, st));
       M = m_new;
       LAZY_TRY(upload(T_CU_X));
+      for (int s = 0; s < S; ++s) tab(T_QROW)[s] = tab(T_CU_X)[s + 1] - 1;
+      LAZY_TRY(upload(T_QROW));
       xmap_kernel<<<cdiv(M, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_BASE), xpos, S, M, xmap, 1);
       KLAUNCH_OK();
       c->stats.revived[l + 1] = revived_total;

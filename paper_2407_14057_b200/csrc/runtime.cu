@@ -179,7 +179,7 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->d_found = (int32_t *)k.take(KV * 4);
   c->kv_map = (int32_t *)k.take((size_t)L * KV * 4);
   c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
-  c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)16 * 2 * (c->S + 1) * 4);
+  c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)(16 * 2 + L) * (c->S + 1) * 4);
   c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
   c->capture = with_capture ? k.take((size_t)L * R * rb) : nullptr;
   return k.off;
