@@ -23,7 +23,10 @@ int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const 
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, B, nullptr, R, C, M, N, K, 0);
-  return launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status);
+  gemm_force_single(impl == 2);
+  const int rc = launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status);
+  gemm_force_single(0);
+  return rc;
 }
 
 int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
@@ -34,7 +37,10 @@ int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A,
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  return launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status);
+  gemm_force_single(impl == 2);
+  const int rc = launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status);
+  gemm_force_single(0);
+  return rc;
 }
 
 int lazy_k_rope_kv(void *stream, int32_t dtype, void *qkv, const int32_t *pos, float *rope_table,

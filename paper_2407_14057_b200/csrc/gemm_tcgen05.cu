@@ -14,11 +14,13 @@
 // Every mbarrier wait is bounded (wall-clock limit); on expiry the kernel records
 // LAZY_E_TIMEOUT in the status word, every role leaves its loop, TMEM is released and the CTA
 // exits.  No cluster launch, no multicast.
-#include "tc_common.cuh"
+#include "gemm_epilogue.cuh"
 
 namespace lazy {
 
 namespace {
+
+static_assert(GEMM_ACC_N == 256, "tile width");
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_STAGE_BYTES = BM * BK * 2;       // 16 KiB
@@ -38,20 +40,6 @@ struct __align__(8) GemmBarriers {
 };
 constexpr int GEMM_SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align slack*/ +
                                 (int)sizeof(GemmBarriers);
-
-enum { EPI_PLAIN = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_QKV_ROPE = 3 };
-
-// Extra operands of the QKV epilogue: the rotary embedding is applied to the fp32 accumulators and
-// the rotated k, and v, go straight to the layer's cache rows (head_dim 128: one 256-column tile is
-// two whole heads of q, k or v, and a thread holds its row's full heads).
-struct RopeArgs {
-  const int32_t *pos;     // [M] original positions
-  const float2 *table;    // [max_pos][64] (cos, sin)
-  bf16 *kcache, *vcache;  // [rows, d_model]
-  int32_t *kv_pos;        // position tag per cache row (may be NULL)
-  const int32_t *kv_row;  // cache row of GEMM row r (NULL: r)
-  int d_model, max_pos;
-};
 
 // C is [M, ldc]; for EPI_SWIGLU the accumulator's columns [0,128) are gate features and
 // [128,256) the matching up features, and C receives 128 columns per tile.
@@ -182,105 +170,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-      bf16 *crow = C + (size_t)row * ldc;
-      const bf16 *rrow = (EPI == EPI_RESIDUAL) ? R + (size_t)row * ldc : nullptr;
-      if (EPI == EPI_QKV_ROPE) {
-        // section of the fused projection this tile belongs to: 0 = q, 1 = k, 2 = v
-        const int sect = n0 / rope.d_model;
-        const int col_in = n0 - sect * rope.d_model;
-        int p = 0;
-        size_t krow = 0;
-        if (row < M) {
-          p = rope.pos[row];
-          if (p < 0 || p >= rope.max_pos) {
-            dev_fail(status, LAZY_E_CAPACITY, W_ROPE_POS, row, p);
-            p = 0;
-          }
-          krow = rope.kv_row ? (size_t)rope.kv_row[row] : (size_t)row;
-        }
-        bf16 *dst = sect == 0 ? crow + n0
-                              : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_model + col_in;
-        if (sect == 2) {
-#pragma unroll 1
-          for (int c = 0; c < BN; c += 32) {
-            float v[32];
-            tmem_ld_32x32(taddr + (uint32_t)c, v);
-            if (row < M) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                Vec16<bf16> o;
-                o.pack(v + j);
-                o.store(dst + c + j);
-              }
-            }
-          }
-        } else {
-          const float2 *tab = rope.table + (size_t)p * 64;
-#pragma unroll 1
-          for (int hc = 0; hc < BN; hc += 128) {  // the two heads of the tile
-#pragma unroll 1
-            for (int o = 0; o < 64; o += 32) {    // pairs (i, i + 64), 32 at a time
-              float lo[32], hi[32];
-              tmem_ld_32x32(taddr + (uint32_t)(hc + o), lo);
-              tmem_ld_32x32(taddr + (uint32_t)(hc + o + 64), hi);
-              if (row < M) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                  const float4 cs = *reinterpret_cast<const float4 *>(tab + o + i);  // two (cos, sin)
-                  const float a0 = lo[i], b0 = hi[i], a1 = lo[i + 1], b1 = hi[i + 1];
-                  lo[i] = a0 * cs.x - b0 * cs.y;
-                  hi[i] = b0 * cs.x + a0 * cs.y;
-                  lo[i + 1] = a1 * cs.z - b1 * cs.w;
-                  hi[i + 1] = b1 * cs.z + a1 * cs.w;
-                }
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  Vec16<bf16> ol, oh;
-                  ol.pack(lo + j);
-                  oh.pack(hi + j);
-                  ol.store(dst + hc + o + j);
-                  oh.store(dst + hc + o + 64 + j);
-                }
-              }
-            }
-          }
-          if (sect == 1 && col_in == 0 && row < M && rope.kv_pos) rope.kv_pos[krow] = p;
-        }
-      } else {
-#pragma unroll 1
-      for (int c = 0; c < TILE_N_OUT; c += 32) {
-        float v[32];
-        tmem_ld_32x32(taddr + (uint32_t)c, v);
-        if (EPI == EPI_SWIGLU) {
-          float u[32];
-          tmem_ld_32x32(taddr + (uint32_t)(BN / 2 + c), u);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
-        }
-        if (row < M) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            const int col = n0 + c + j;
-            if (col < N) {  // N is a multiple of 8: a vector is entirely inside or outside
-              float f[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) f[i] = v[j + i];
-              if (EPI == EPI_RESIDUAL) {
-                Vec16<bf16> rv;
-                rv.load(rrow + col);
-                float rf[8];
-                rv.unpack(rf);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) f[i] += rf[i];
-              }
-              Vec16<bf16> o;
-              o.pack(f);
-              o.store(crow + col);
-            }
-          }
-        }
-      }
-      }  // epilogue kinds
+      gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[acc]));
@@ -304,6 +194,17 @@ int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_row
   return tma_map_2d_bf16(map, base, rows, cols, cols, BK, box_rows);
 }
 
+// More than one row tile: the CTA-pair kernel, unless LAZY_GEMM=single asks for this one (A/B timing).
+int g_force_single = 0;
+bool gemm_pair_enabled() {
+  static int on = -1;
+  if (on < 0) {
+    const char *e = getenv("LAZY_GEMM");
+    on = (e && strcmp(e, "single") == 0) ? 0 : 1;
+  }
+  return on == 1 && !g_force_single;
+}
+
 template <int EPI>
 int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C,
               int M, int N, int K, DevStatus *status, const RopeArgs &rope = RopeArgs()) {
@@ -311,6 +212,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
+  if (M > BM && gemm_pair_enabled()) return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope);
   CUtensorMap ma, mb0, mb1;
   LAZY_TRY(make_map(&ma, A, M, K, BM));
   LAZY_TRY(make_map(&mb0, B0, N, K, BN / 2));
@@ -331,6 +233,9 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
 }
 
 }  // namespace
+
+// Cross-check switch of the context-free entry points: the next launches use one CTA per tile.
+void gemm_force_single(int on) { g_force_single = on; }
 
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
                 int M, int N, int K, DevStatus *status) {

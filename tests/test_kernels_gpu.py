@@ -93,6 +93,32 @@ def test_gemm_fp32(M, N, K):
     assert rel_err(to_np(out), ref) < F32_TOL
 
 
+@pytest.mark.parametrize("M,N,K", [(129, 256, 64), (256, 512, 128), (300, 1376, 688), (513, 4096, 4096),
+                                   (3376, 768, 4096), (1013, 4096, 11008)])
+def test_gemm_bf16_cta_pair_kernel_against_one_cta_kernel_and_oracle(M, N, K):
+    """Above 128 rows the CTA-pair kernel (256x256 tiles over two SMs) is the production path; impl=2
+    forces one CTA per 128x256 tile.  Both accumulate a tile's K range in the same order in fp32, so they
+    agree to the last bit, and both match the fp64 product."""
+    A = _rand((M, K), 21, torch.bfloat16).cuda()
+    Bm = _rand((N, K), 22, torch.bfloat16, 0.05).cuda()
+    R = _rand((M, N), 23, torch.bfloat16).cuda()
+    pair = B.lazy_k_gemm(A, Bm, R)
+    one = B.lazy_k_gemm(A, Bm, R, impl=2)
+    B.lazy_device_status()
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(R))
+    assert rel_err(to_np(pair), ref) < BF16_STEP_TOL
+    assert rel_err(to_np(one), ref) < BF16_STEP_TOL
+    assert torch.equal(pair, one)
+    F = min(N, 1408)
+    g_pair = B.lazy_k_gemm_swiglu(A, Bm[:F // 2].contiguous(), Bm[F // 2:F].contiguous())
+    g_one = B.lazy_k_gemm_swiglu(A, Bm[:F // 2].contiguous(), Bm[F // 2:F].contiguous(), impl=2)
+    B.lazy_device_status()
+    a = O.f64(to_np(A))
+    ref = O.silu(a @ O.f64(to_np(Bm[:F // 2])).T) * (a @ O.f64(to_np(Bm[F // 2:F])).T)
+    assert rel_err(to_np(g_pair), ref) < BF16_STEP_TOL
+    assert torch.equal(g_pair, g_one)
+
+
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 5])
 def test_gemm_bf16_few_rows_weight_streaming_kernel(M):
     """M <= 4 takes the weight-streaming kernel, M = 5 the tensor-core one: same answers."""
