@@ -239,9 +239,22 @@ int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, vo
  * tensor cores with one CTA per tile at every M > 4 (cross-check and timing of the pair kernel). */
 int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B,
                 const void *R, void *C, int32_t M, int32_t N, int32_t K);
+/* The same product with a device scratch of lazy_k_gemm_scratch_bytes() bytes that the bf16
+ * tensor-core kernels use to split the last, partial wave of output tiles along K (partial sums and
+ * arrival counters).  The scratch must be zero before its first use, is left zero by every call,
+ * and must not be shared by calls running at the same time.  Results do not depend on it being
+ * given (the parts of a tile are added in a fixed order).  The paper has no counterpart: this is
+ * scheduling of the dense products of Section 3.2's layers.  NULL scratch = lazy_k_gemm. */
+size_t lazy_k_gemm_scratch_bytes(void);
+int lazy_k_gemm_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B,
+                   const void *R, void *C, int32_t M, int32_t N, int32_t K, void *d_scratch,
+                   size_t scratch_bytes);
 /* C[M,F] = silu(A Bg^T) * (A Bu^T), Bg, Bu [F, K] (SwiGLU, first half of the MLP). */
 int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
                        const void *Bu, void *C, int32_t M, int32_t F, int32_t K);
+int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
+                          const void *Bu, void *C, int32_t M, int32_t F, int32_t K, void *d_scratch,
+                          size_t scratch_bytes);
 /* In-place RoPE of q and k inside qkv [n, 3*H*dh] by positions pos[n]; rotated k and v are
  * also written to kcache / vcache [n, H*dh].  rope_table: device fp32[max_pos*head_dim] scratch
  * that the call fills first. */

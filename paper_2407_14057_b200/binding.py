@@ -96,6 +96,9 @@ _SIGNATURES = {
     "lazy_k_rmsnorm": (_I, [_P, _I, _P, _P, _P, _I, _I, _F]),
     "lazy_k_gemm": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
     "lazy_k_gemm_swiglu": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
+    "lazy_k_gemm_scratch_bytes": (_Z, []),
+    "lazy_k_gemm_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
+    "lazy_k_gemm_swiglu_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
     "lazy_k_rope_kv": (_I, [_P, _I, _P, _P, _P, _P, _P, _I, _I, _I, _I, _F]),
     "lazy_k_attention": (_I, [_P, _I, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _I]),
     "lazy_k_score_scratch_floats": (_Z, [_I, _I, _I]),
@@ -320,23 +323,37 @@ def lazy_k_rmsnorm(x: torch.Tensor, g: torch.Tensor, eps: float) -> torch.Tensor
     return y
 
 
+def lazy_k_gemm_scratch(device="cuda") -> torch.Tensor:
+    """Zeroed scratch for the `scratch=` argument of lazy_k_gemm / lazy_k_gemm_swiglu."""
+    return torch.zeros(lib().lazy_k_gemm_scratch_bytes(), dtype=torch.uint8, device=device)
+
+
 def lazy_k_gemm(A: torch.Tensor, B: torch.Tensor, R: Optional[torch.Tensor] = None, impl: int = 0,
-                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                out: Optional[torch.Tensor] = None, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
     M, K = A.shape
     N = B.shape[0]
     Cm = out if out is not None else torch.empty((M, N), dtype=A.dtype, device=A.device)
-    _check("lazy_k_gemm", lib().lazy_k_gemm(_stream(), dtype_code(A.dtype), impl, _ptr(A), _ptr(B), _ptr(R),
-                                            _ptr(Cm), M, N, K))
+    if scratch is None:
+        _check("lazy_k_gemm", lib().lazy_k_gemm(_stream(), dtype_code(A.dtype), impl, _ptr(A), _ptr(B), _ptr(R),
+                                                _ptr(Cm), M, N, K))
+    else:
+        _check("lazy_k_gemm_ws", lib().lazy_k_gemm_ws(_stream(), dtype_code(A.dtype), impl, _ptr(A), _ptr(B),
+                                                      _ptr(R), _ptr(Cm), M, N, K, _ptr(scratch), scratch.numel()))
     return Cm
 
 
 def lazy_k_gemm_swiglu(A: torch.Tensor, Bg: torch.Tensor, Bu: torch.Tensor, impl: int = 0,
-                       out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                       out: Optional[torch.Tensor] = None, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:
     M, K = A.shape
     F = Bg.shape[0]
     Cm = out if out is not None else torch.empty((M, F), dtype=A.dtype, device=A.device)
-    _check("lazy_k_gemm_swiglu", lib().lazy_k_gemm_swiglu(_stream(), dtype_code(A.dtype), impl, _ptr(A),
-                                                          _ptr(Bg), _ptr(Bu), _ptr(Cm), M, F, K))
+    if scratch is None:
+        _check("lazy_k_gemm_swiglu", lib().lazy_k_gemm_swiglu(_stream(), dtype_code(A.dtype), impl, _ptr(A),
+                                                              _ptr(Bg), _ptr(Bu), _ptr(Cm), M, F, K))
+    else:
+        _check("lazy_k_gemm_swiglu_ws",
+               lib().lazy_k_gemm_swiglu_ws(_stream(), dtype_code(A.dtype), impl, _ptr(A), _ptr(Bg), _ptr(Bu),
+                                           _ptr(Cm), M, F, K, _ptr(scratch), scratch.numel()))
     return Cm
 
 

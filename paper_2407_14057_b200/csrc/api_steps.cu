@@ -15,8 +15,15 @@ int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, vo
   return launch_rmsnorm((cudaStream_t)stream, dtype, x, g, y, n, d, eps);
 }
 
+size_t lazy_k_gemm_scratch_bytes(void) { return gemm_scratch_bytes(); }
+
 int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B, const void *R,
                 void *C, int32_t M, int32_t N, int32_t K) {
+  return lazy_k_gemm_ws(stream, dtype, impl, A, B, R, C, M, N, K, nullptr, 0);
+}
+
+int lazy_k_gemm_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B, const void *R,
+                   void *C, int32_t M, int32_t N, int32_t K, void *d_scratch, size_t scratch_bytes) {
   if (bad_dtype(dtype) || M < 0 || N < 1 || K < 1 || N % 8 || K % 8) return LAZY_E_BADARG;
   if (M == 0) return LAZY_OK;  // nothing to compute; an empty matrix may have no address
   if (!A || !B || !C) return LAZY_E_BADARG;
@@ -24,13 +31,19 @@ int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const 
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, B, nullptr, R, C, M, N, K, 0);
   gemm_force_single(impl == 2);
-  const int rc = launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status);
+  const int rc = launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status, d_scratch, scratch_bytes);
   gemm_force_single(0);
   return rc;
 }
 
 int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
                        const void *Bu, void *C, int32_t M, int32_t F, int32_t K) {
+  return lazy_k_gemm_swiglu_ws(stream, dtype, impl, A, Bg, Bu, C, M, F, K, nullptr, 0);
+}
+
+int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
+                          const void *Bu, void *C, int32_t M, int32_t F, int32_t K, void *d_scratch,
+                          size_t scratch_bytes) {
   if (bad_dtype(dtype) || M < 0 || F < 1 || K < 1 || F % 8 || K % 8) return LAZY_E_BADARG;
   if (M == 0) return LAZY_OK;
   if (!A || !Bg || !Bu || !C) return LAZY_E_BADARG;
@@ -38,7 +51,8 @@ int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A,
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
   gemm_force_single(impl == 2);
-  const int rc = launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status);
+  const int rc = launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status, d_scratch,
+                                    scratch_bytes);
   gemm_force_single(0);
   return rc;
 }

@@ -32,6 +32,7 @@ enum DevWhere {
   W_ATTN_PRODUCER = 11,
   W_ATTN_MMA = 12,
   W_ATTN_SOFTMAX = 13,
+  W_GEMM_TAIL = 14,
 };
 
 __device__ __forceinline__ void dev_fail(DevStatus *st, int code, int where, int a = 0, int b = 0) {
@@ -156,17 +157,22 @@ int launch_rope_table(cudaStream_t st, float *table, int max_pos, int head_dim, 
 int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, const float *table,
                    void *kcache, void *vcache, int32_t *kv_pos, const int32_t *kv_row, int n,
                    int n_heads, int head_dim, int max_pos, DevStatus *status);
+// scratch (gemm_scratch_bytes() bytes, zeroed once, private to the stream) lets the tensor-core kernels
+// split the last partial wave of tiles along K; without it they run a plain tile loop.
+size_t gemm_scratch_bytes();
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
-                int M, int N, int K, DevStatus *status);
+                int M, int N, int K, DevStatus *status, void *scratch = nullptr, size_t scratch_bytes = 0);
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
-                       void *C, int M, int F, int K, DevStatus *status);
+                       void *C, int M, int F, int K, DevStatus *status, void *scratch = nullptr,
+                       size_t scratch_bytes = 0);
 // QKV projection with the rotary embedding and the K/V cache write in its epilogue (bf16,
 // head_dim 128, d_model a multiple of 256): qkv [M, 3d] receives the rotated q (its k and v thirds
 // are left untouched), rotated k and v go to cache rows kv_row[r] (or r) with their position tag.
 bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
-                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
+                         void *scratch = nullptr, size_t scratch_bytes = 0);
 void gemm_force_single(int on);
 // Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
 // rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).

@@ -339,7 +339,8 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
                                    c->cfg.rms_eps, 0));
     } else {
       LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
-      LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status));
+      LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status, c->gemm_scratch,
+                           c->gemm_scratch_bytes));
     }
     {
       const int n_thr = M > n_ctx ? M : n_ctx;
@@ -367,7 +368,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
       LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
                                n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
     }
-    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status));
+    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status, c->gemm_scratch, c->gemm_scratch_bytes));
 
     const int pt = c->point_at[l + 1];
     if (pt >= 0) {
@@ -473,9 +474,11 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
                                    c->cfg.rms_eps, 0));
     } else {
       LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
-      LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status));
+      LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status, c->gemm_scratch,
+                                  c->gemm_scratch_bytes));
     }
-    LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status));
+    LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status, c->gemm_scratch,
+                         c->gemm_scratch_bytes));
   }
   for (int s = 0; s < S; ++s) tab(T_LAST)[s] = tab(T_CU_X)[s + 1] - 1;
   LAZY_TRY(upload(T_LAST));

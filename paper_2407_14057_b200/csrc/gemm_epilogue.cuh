@@ -21,14 +21,149 @@ struct RopeArgs {
   int d_model, max_pos;
 };
 
+// ---- the last, partial wave ------------------------------------------------------------------------------
+// num_tiles is rarely a multiple of the number of persistent units (CTAs, or CTA pairs), so a plain
+// tile loop ends with a wave in which most units idle for a whole tile time.  Instead the K loops of the
+// last (num_tiles - first_tail) tiles are laid end to end and cut into tail_units equal ranges, one per
+// unit.  A range touches at most two tiles: the end of one (a DUMP: the fp32 partial accumulator goes to
+// the unit's slot of `partials`) and the start of the next (the FINISH part: it waits for the dumps of the
+// units after it that cover the same tile, adds them in unit order - deterministic - and runs the normal
+// epilogue).  A dump never waits, and every unit dumps before it finishes, so no wait is circular; all
+// units are resident at once (persistent grid), and the wait is time-bounded anyway.
+constexpr int GEMM_TAIL_MIN_KB = 8;               // shortest K range (in 64-wide slices) worth a part
+constexpr int GEMM_SLOT_FLOATS = 128 * GEMM_ACC_N;  // one CTA's accumulator
+
+struct GemmTail {
+  float *partials;   // [CTAs][128][256] fp32
+  unsigned *flags;   // [tail tiles x ranks] dump arrivals (one per epilogue warp); zero between launches
+  unsigned *done;    // [tail tiles x ranks] finisher warps through; the last one re-zeroes both
+  int first_tail;    // tiles [first_tail, num_tiles) are split along K; num_tiles: nothing is
+  int tail_units;    // units that share them
+};
+
+// Scratch layout: 2 x GEMM_TAIL_MAX_CTAS counters (2 KiB), then one accumulator slot per persistent CTA.
+constexpr int GEMM_TAIL_MAX_CTAS = 160;
+constexpr size_t GEMM_TAIL_COUNTER_BYTES = 2048;
+static_assert(2 * GEMM_TAIL_MAX_CTAS * sizeof(unsigned) <= GEMM_TAIL_COUNTER_BYTES, "counter block");
+inline size_t gemm_tail_scratch_bytes(int ctas) {
+  return GEMM_TAIL_COUNTER_BYTES + (size_t)ctas * GEMM_SLOT_FLOATS * 4;
+}
+
+struct GemmWork {
+  int tile, kb0, kb1;
+  int mode;      // 0: whole tile, 1: dump, 2: finish
+  int tail_idx;  // index among the tail tiles
+};
+
+__device__ __forceinline__ int gemm_tail_start(int u, int tail_units, int total_kb) {
+  return (int)(((long long)u * total_kb) / tail_units);
+}
+
+// i-th work item of unit u of `units`; false when the unit has no more.
+__device__ __forceinline__ bool gemm_work_item(int i, int u, int units, int num_tiles, int num_kb,
+                                               const GemmTail &t, GemmWork &w) {
+  const int n_whole = u < t.first_tail ? (t.first_tail - u + units - 1) / units : 0;
+  if (i < n_whole) {
+    w.tile = u + i * units;
+    w.kb0 = 0;
+    w.kb1 = num_kb;
+    w.mode = 0;
+    w.tail_idx = 0;
+    return true;
+  }
+  if (t.first_tail >= num_tiles || u >= t.tail_units) return false;
+  const int total = (num_tiles - t.first_tail) * num_kb;
+  const int s = gemm_tail_start(u, t.tail_units, total), e = gemm_tail_start(u + 1, t.tail_units, total);
+  const int t0 = s / num_kb;
+  const int e0 = min(e, (t0 + 1) * num_kb);
+  int a, b, tt;
+  if (i == n_whole) {
+    a = s; b = e0; tt = t0;
+  } else if (i == n_whole + 1) {
+    a = e0; b = e; tt = t0 + 1;
+  } else {
+    return false;
+  }
+  if (b <= a) return false;
+  w.tile = t.first_tail + tt;
+  w.kb0 = a - tt * num_kb;
+  w.kb1 = b - tt * num_kb;
+  w.mode = w.kb0 != 0 ? 1 : (w.kb1 == num_kb ? 0 : 2);
+  w.tail_idx = tt;
+  return true;
+}
+
+// Units after u whose range starts inside tail tile tt: each holds one dump for it.
+__device__ __forceinline__ int gemm_tail_dumps(int u, int tt, int num_tiles, int num_kb, const GemmTail &t) {
+  const int total = (num_tiles - t.first_tail) * num_kb;
+  int n = 0;
+  for (int v = u + 1; v < t.tail_units && gemm_tail_start(v, t.tail_units, total) < (tt + 1) * num_kb; ++v) ++n;
+  return n;
+}
+
+// v[0..32) += the same 32 columns of n partial accumulators, SLOT_STEP slots apart.
+template <int SLOT_STEP>
+__device__ __forceinline__ void gemm_add_partials(float (&v)[32], const float *part_row, int n, int col) {
+  for (int d = 0; d < n; ++d) {
+    const float4 *q = reinterpret_cast<const float4 *>(part_row + (size_t)d * SLOT_STEP * GEMM_SLOT_FLOATS + col);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float4 x = __ldcg(q + j);  // written by other SMs during this launch: read at L2
+      v[4 * j] += x.x;
+      v[4 * j + 1] += x.y;
+      v[4 * j + 2] += x.z;
+      v[4 * j + 3] += x.w;
+    }
+  }
+}
+
+// Dump of one accumulator row (a thread's 256 fp32 columns) to its slot.
+__device__ __forceinline__ void gemm_dump_row(uint32_t taddr, float *slot_row) {
+#pragma unroll 1
+  for (int c = 0; c < GEMM_ACC_N; c += 32) {
+    float v[32];
+    tmem_ld_32x32(taddr + (uint32_t)c, v);
+    float4 *q = reinterpret_cast<float4 *>(slot_row + c);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+  }
+}
+
+// Warp-level, bounded wait until *flag >= target.  False (and the abort flag set) on expiry.
+__device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned target, volatile int *abort_flag,
+                                               DevStatus *status) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) {
+    const unsigned long long t0 = global_timer_ns();
+    uint32_t spins = 0;
+    for (;;) {
+      unsigned v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+      if (v >= target) break;
+      if ((++spins & 63u) == 0) {
+        if (*abort_flag) { ok = 0; break; }
+        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+          *abort_flag = 1;
+          dev_fail(status, LAZY_E_TIMEOUT, W_GEMM_TAIL, (int)blockIdx.x, (int)v);
+          ok = 0;
+          break;
+        }
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
 // One thread, one row.  taddr: TMEM address of the row's first accumulator column (lane field set);
-// row: global output row; n0: first output column of the tile as the caller sees it.  C is [M, ldc];
+// row: global output row; n0: first output column of the tile as the caller sees it; part_row / n_parts:
+// this row in the first of n_parts partial accumulators to add first (finish part of a split tile).  C is [M, ldc];
 // for EPI_SWIGLU accumulator columns [0,128) are gate features, [128,256) the matching up features and C
 // receives 128 columns per tile.
-template <int EPI>
+template <int EPI, int SLOT_STEP = 1>
 __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n0, int M, int N, int ldc,
                                                   const bf16 *__restrict__ R, bf16 *__restrict__ C,
-                                                  const RopeArgs &rope, DevStatus *status) {
+                                                  const RopeArgs &rope, DevStatus *status,
+                                                  const float *part_row = nullptr, int n_parts = 0) {
   constexpr int BN = GEMM_ACC_N;
   constexpr int TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   bf16 *crow = C + (size_t)row * ldc;
@@ -54,6 +189,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       for (int c = 0; c < BN; c += 32) {
         float v[32];
         tmem_ld_32x32(taddr + (uint32_t)c, v);
+        gemm_add_partials<SLOT_STEP>(v, part_row, n_parts, c);
         if (row < M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
@@ -72,6 +208,8 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
           float lo[32], hi[32];
           tmem_ld_32x32(taddr + (uint32_t)(hc + o), lo);
           tmem_ld_32x32(taddr + (uint32_t)(hc + o + 64), hi);
+          gemm_add_partials<SLOT_STEP>(lo, part_row, n_parts, hc + o);
+          gemm_add_partials<SLOT_STEP>(hi, part_row, n_parts, hc + o + 64);
           if (row < M) {
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
@@ -100,9 +238,11 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
   for (int c = 0; c < TILE_N; c += 32) {
     float v[32];
     tmem_ld_32x32(taddr + (uint32_t)c, v);
+    gemm_add_partials<SLOT_STEP>(v, part_row, n_parts, c);
     if (EPI == EPI_SWIGLU) {
       float u[32];
       tmem_ld_32x32(taddr + (uint32_t)(BN / 2 + c), u);
+      gemm_add_partials<SLOT_STEP>(u, part_row, n_parts, BN / 2 + c);
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
     }
@@ -132,9 +272,34 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
   }  // epilogue kinds
 }
 
+// Splits the last partial wave along K when that pays: `units` persistent units, `cta_per_unit` CTAs each.
+// scratch NULL or too small, a whole number of waves, or a nearly full last wave: plain tile loop.
+inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, void *scratch, size_t scratch_bytes) {
+  GemmTail t = {};
+  t.first_tail = num_tiles;
+  t.tail_units = 0;
+  if (!scratch || units * cta_per_unit > GEMM_TAIL_MAX_CTAS ||
+      scratch_bytes < gemm_tail_scratch_bytes(units * cta_per_unit))
+    return t;
+  const int first = (num_tiles / units) * units, rem = num_tiles - first;
+  if (rem == 0) return t;
+  // idle unit-time of the last wave, in K slices, must outweigh the dump and fix-up traffic
+  if ((long long)(units - rem) * num_kb < 16ll * units) return t;
+  long long tu = (long long)rem * num_kb / GEMM_TAIL_MIN_KB;
+  if (tu > units) tu = units;
+  if (tu <= rem) return t;
+  t.flags = (unsigned *)scratch;
+  t.done = t.flags + GEMM_TAIL_MAX_CTAS;
+  t.partials = (float *)((char *)scratch + GEMM_TAIL_COUNTER_BYTES);
+  t.first_tail = first;
+  t.tail_units = (int)tu;
+  return t;
+}
+
 // The same GEMM on CTA pairs (256x256 tiles, cta_group::2); epi is one of the EPI_* values.
 int launch_gemm_pair(int epi, cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
-                     void *C, int M, int N, int K, DevStatus *status, const RopeArgs &rope);
+                     void *C, int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
+                     size_t scratch_bytes);
 // Clusters of two CTAs of that kernel the device can hold at once (-1: query failed).
 int gemm_pair_max_clusters();
 

@@ -49,7 +49,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
                          const __grid_constant__ CUtensorMap map_b0,
                          const __grid_constant__ CUtensorMap map_b1, const bf16 *__restrict__ R,
                          bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
-                         const RopeArgs rope) {
+                         const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -100,10 +100,11 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile % m_tiles) * BM;
-        const int n0 = (tile / m_tiles) * TILE_N_OUT;
-        for (int kb = 0; kb < num_kb; ++kb) {
+      GemmWork w;
+      for (int it = 0; ok && gemm_work_item(it, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++it) {
+        const int m0 = (w.tile % m_tiles) * BM;
+        const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status, W_GEMM_PRODUCER);
           if (!ok) break;
           const uint32_t full = smem_u32(&bars->full[stage]);
@@ -129,14 +130,15 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+      GemmWork w;
+      for (; ok && gemm_work_item(local, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++local) {
         const int acc = local & 1;
         const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
         ok = mbar_wait(smem_u32(&bars->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status, W_GEMM_MMA_TMEM);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status, W_GEMM_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
@@ -146,7 +148,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t adesc = umma_smem_desc(a_addr + k * UMMA_K * 2);
             const uint64_t bdesc = umma_smem_desc(b_addr + k * UMMA_K * 2);
-            umma_bf16(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16(tmem_d, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(smem_u32(&bars->empty[stage]));  // stage reusable once these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -159,18 +161,44 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
     int local = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+    GemmWork w;
+    for (; ok && gemm_work_item(local, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-      const int m0 = (tile % m_tiles) * BM;
-      const int n0 = (tile / m_tiles) * TILE_N_OUT;
+      const int m0 = (w.tile % m_tiles) * BM;
+      const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-      gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
+      const int row_in_tile = quarter * 32 + lane;
+      if (w.mode == 1) {  // partial accumulator of a split tile: to this CTA's slot, then tell the finisher
+        gemm_dump_row(taddr, tail.partials + ((size_t)blockIdx.x * BM + row_in_tile) * BN);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(tail.flags + w.tail_idx, 1u);
+        }
+      } else {
+        int n_parts = 0;
+        if (w.mode == 2) {  // first part of a split tile: the other parts' sums come first
+          n_parts = gemm_tail_dumps(blockIdx.x, w.tail_idx, num_tiles, num_kb, tail);
+          ok = gemm_tail_wait(tail.flags + w.tail_idx, 4u * (unsigned)n_parts, abort_flag, status);
+          if (!ok) break;
+        }
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status,
+                               tail.partials + ((size_t)(blockIdx.x + 1) * BM + row_in_tile) * BN, n_parts);
+        if (w.mode == 2) {
+          __syncwarp();
+          if (lane == 0 && atomicAdd(tail.done + w.tail_idx, 1u) == 3u) {  // last warp through: clean for the next launch
+            tail.flags[w.tail_idx] = 0u;
+            tail.done[w.tail_idx] = 0u;
+          }
+        }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[acc]));
@@ -207,19 +235,22 @@ bool gemm_pair_enabled() {
 
 template <int EPI>
 int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C,
-              int M, int N, int K, DevStatus *status, const RopeArgs &rope = RopeArgs()) {
+              int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
+              size_t scratch_bytes) {
   // TMA needs 16-byte aligned bases and row pitches; the epilogue stores 8 columns at a time.
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
-  if (M > BM && gemm_pair_enabled()) return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope);
+  if (M > BM && gemm_pair_enabled())
+    return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
   CUtensorMap ma, mb0, mb1;
   LAZY_TRY(make_map(&ma, A, M, K, BM));
   LAZY_TRY(make_map(&mb0, B0, N, K, BN / 2));
   LAZY_TRY(make_map(&mb1, B1, N, K, BN / 2));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, scratch, scratch_bytes);
+  const int grid = (tiles < sm_count() && tail.tail_units == 0) ? tiles : sm_count();
   auto kfn = gemm_bf16_tcgen05_kernel<EPI>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -227,23 +258,27 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
     attr_set = true;
   }
   kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N,
-                                                  status, rope);
+                                                  status, rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
 
 }  // namespace
 
+// Sized for up to 160 persistent CTAs whatever the device (the size is asked for without one, too); with
+// more SMs than that the kernels fall back to the plain tile loop.
+size_t gemm_scratch_bytes() { return gemm_tail_scratch_bytes(GEMM_TAIL_MAX_CTAS); }
+
 // Cross-check switch of the context-free entry points: the next launches use one CTA per tile.
 void gemm_force_single(int on) { g_force_single = on; }
 
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
-                int M, int N, int K, DevStatus *status) {
+                int M, int N, int K, DevStatus *status, void *scratch, size_t scratch_bytes) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, B, nullptr, R, C, M, N, K, 0);
   if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, B, nullptr, R, C, M, N, K, 0);
-  if (R) return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status);
-  return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status);
+  if (R) return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes);
+  return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes);
 }
 
 bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {
@@ -252,7 +287,8 @@ bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {
 
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
-                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status) {
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
+                         void *scratch, size_t scratch_bytes) {
   if (M == 0) return LAZY_OK;
   RopeArgs r;
   r.pos = pos;
@@ -263,15 +299,16 @@ int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void
   r.kv_row = kv_row;
   r.d_model = d_model;
   r.max_pos = max_pos;
-  return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, 3 * d_model, d_model, status, r);
+  return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, 3 * d_model, d_model, status, r, scratch,
+                                 scratch_bytes);
 }
 
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
-                       void *C, int M, int F, int K, DevStatus *status) {
+                       void *C, int M, int F, int K, DevStatus *status, void *scratch, size_t scratch_bytes) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
   if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  return launch_tc<EPI_SWIGLU>(st, A, Bg, Bu, nullptr, C, M, F, K, status);
+  return launch_tc<EPI_SWIGLU>(st, A, Bg, Bu, nullptr, C, M, F, K, status, RopeArgs(), scratch, scratch_bytes);
 }
 
 }  // namespace lazy

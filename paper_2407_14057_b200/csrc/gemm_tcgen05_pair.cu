@@ -44,7 +44,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                               const __grid_constant__ CUtensorMap map_b0,
                               const __grid_constant__ CUtensorMap map_b1, const bf16 *__restrict__ R,
                               bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
-                              const RopeArgs rope) {
+                              const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw_addr = smem_u32(smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;  // same in both CTAs of the pair
@@ -91,10 +91,11 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
-        const int m0 = (tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
-        const int n0 = (tile / m_tiles) * TILE_N_OUT;
-        for (int kb = 0; kb < num_kb; ++kb) {
+      GemmWork w;
+      for (int it = 0; ok && gemm_work_item(it, pair, n_pairs, num_tiles, num_kb, tail, w); ++it) {
+        const int m0 = (w.tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
+        const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status, W_GEMM_PRODUCER);
           if (!ok) break;
           const uint32_t full_local = smem_u32(&bars->full[stage]);
@@ -119,14 +120,15 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       uint32_t phase = 0;
       int local = 0;
       bool ok = true;
-      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs, ++local) {
+      GemmWork w;
+      for (; ok && gemm_work_item(local, pair, n_pairs, num_tiles, num_kb, tail, w); ++local) {
         const int acc = local & 1;
         const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
         ok = mbar_wait(smem_u32(&bars->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, status, W_GEMM_MMA_TMEM);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(acc * PBN);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->full[stage]), phase, abort_flag, status, W_GEMM_MMA_FULL);
           if (!ok) break;
           tc_fence_after();
@@ -136,7 +138,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           for (int k = 0; k < PBK / PUMMA_K; ++k) {
             const uint64_t adesc = umma_smem_desc(a_addr + k * PUMMA_K * 2);
             const uint64_t bdesc = umma_smem_desc(b_addr + k * PUMMA_K * 2);
-            umma_bf16_pair(tmem_d, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16_pair(tmem_d, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
           }
           // the stage is reusable in both CTAs once these MMAs retire
           const uint32_t empty_local = smem_u32(&bars->empty[stage]);
@@ -156,18 +158,48 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     const int quarter = warp & 3;  // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
     int local = 0;
     bool ok = true;
-    for (int tile = pair; tile < num_tiles && ok; tile += n_pairs, ++local) {
+    GemmWork w;
+    for (; ok && gemm_work_item(local, pair, n_pairs, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-      const int m0 = (tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
-      const int n0 = (tile / m_tiles) * TILE_N_OUT;
+      const int m0 = (w.tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
+      const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * PBN);
-      gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
+      // split tiles: slot of pair p, rank r = CTA 2p + r; one arrival counter per (tail tile, rank)
+      const int row_in_tile = quarter * 32 + lane;
+      const int flag_idx = 2 * w.tail_idx + (int)rank;
+      if (w.mode == 1) {
+        gemm_dump_row(taddr, tail.partials + ((size_t)(2 * pair + (int)rank) * PBM + row_in_tile) * PBN);
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          __threadfence();
+          atomicAdd(tail.flags + flag_idx, 1u);
+        }
+      } else {
+        int n_parts = 0;
+        if (w.mode == 2) {  // first part of a split tile: the other parts' sums come first
+          n_parts = gemm_tail_dumps(pair, w.tail_idx, num_tiles, num_kb, tail);
+          ok = gemm_tail_wait(tail.flags + flag_idx, 4u * (unsigned)n_parts, abort_flag, status);
+          if (!ok) break;
+        }
+        // the dumps of the following pairs, same rank: every second slot
+        gemm_epilogue_row<EPI, 2>(taddr, row, n0, M, N, ldc, R, C, rope, status,
+                                  tail.partials + ((size_t)(2 * (pair + 1) + (int)rank) * PBM + row_in_tile) * PBN,
+                                  n_parts);
+        if (w.mode == 2) {
+          __syncwarp();
+          if (lane == 0 && atomicAdd(tail.done + flag_idx, 1u) == 3u) {
+            tail.flags[flag_idx] = 0u;
+            tail.done[flag_idx] = 0u;
+          }
+        }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(cluster_map_shared(smem_u32(&bars->tmem_empty[acc]), 0));
@@ -186,7 +218,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
 
 template <int EPI>
 int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C, int M,
-                int N, int K, DevStatus *status, const RopeArgs &rope) {
+                int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch, size_t scratch_bytes) {
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
@@ -218,9 +250,10 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
     }
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, scratch, scratch_bytes);
+  const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
   kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
-                                                    rope);
+                                                    rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
@@ -251,12 +284,13 @@ int gemm_pair_max_clusters() {
 }
 
 int launch_gemm_pair(int epi, cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
-                     void *C, int M, int N, int K, DevStatus *status, const RopeArgs &rope) {
+                     void *C, int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
+                     size_t scratch_bytes) {
   switch (epi) {
-    case EPI_PLAIN: return launch_pair<EPI_PLAIN>(st, A, B0, B1, R, C, M, N, K, status, rope);
-    case EPI_RESIDUAL: return launch_pair<EPI_RESIDUAL>(st, A, B0, B1, R, C, M, N, K, status, rope);
-    case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(st, A, B0, B1, R, C, M, N, K, status, rope);
-    case EPI_QKV_ROPE: return launch_pair<EPI_QKV_ROPE>(st, A, B0, B1, R, C, M, N, K, status, rope);
+    case EPI_PLAIN: return launch_pair<EPI_PLAIN>(st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
+    case EPI_RESIDUAL: return launch_pair<EPI_RESIDUAL>(st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
+    case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
+    case EPI_QKV_ROPE: return launch_pair<EPI_QKV_ROPE>(st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
     default: return LAZY_E_BADARG;
   }
 }

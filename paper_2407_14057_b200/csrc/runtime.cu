@@ -181,6 +181,8 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
   c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)(16 * 2 + L) * (c->S + 1) * 4);
   c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
+  c->gemm_scratch_bytes = c->dtype == LAZY_BF16 ? gemm_scratch_bytes() : 0;
+  c->gemm_scratch = c->gemm_scratch_bytes ? k.take(c->gemm_scratch_bytes) : nullptr;
   c->capture = with_capture ? k.take((size_t)L * R * rb) : nullptr;
   return k.off;
 }
@@ -303,6 +305,10 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
     return LAZY_E_CUDA;
   }
   rc = launch_rope_table(0, c->rope_table, c->max_pos, c->dh, cfg->rope_theta);
+  // the GEMMs' arrival counters start at zero and return to zero after every launch
+  if (rc == LAZY_OK && c->gemm_scratch &&
+      cudaMemsetAsync(c->gemm_scratch, 0, c->gemm_scratch_bytes, 0) != cudaSuccess)
+    rc = LAZY_E_CUDA;
   if (rc == LAZY_OK && cudaStreamSynchronize(0) != cudaSuccess) rc = LAZY_E_CUDA;
   if (rc != LAZY_OK) {
     delete c;
@@ -463,10 +469,11 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       // rotary embedding and the K/V cache write ride in the projection's epilogue
       TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
             launch_gemm_qkv_rope(st, c->h, c->w_qkv[l], c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n,
-                                 d, c->max_pos, status));
+                                 d, c->max_pos, status, c->gemm_scratch, c->gemm_scratch_bytes));
     } else {
       TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
-            launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status));
+            launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status, c->gemm_scratch,
+                        c->gemm_scratch_bytes));
       TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
             launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
                            c->max_pos, status));
@@ -496,7 +503,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
             launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
                          c->score_scratch, sc));
-    TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status));
+    TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status,
+                                                      c->gemm_scratch, c->gemm_scratch_bytes));
 
     const int p = c->point_at[l + 1];
     if (p >= 0) {
@@ -536,9 +544,11 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     const int n2 = c->seg_cu[g][n_seqs];
     TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb, launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
     TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
-          launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status));
+          launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
+                             c->gemm_scratch_bytes));
     TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
-          launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status));
+          launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status, c->gemm_scratch,
+                      c->gemm_scratch_bytes));
     if (c->capture_on && c->capture)
       LAZY_CUDA_OK(cudaMemcpyAsync(c->capture + (size_t)l * c->cap_rows * rb, x, (size_t)n2 * rb,
                                    cudaMemcpyDeviceToDevice, st));

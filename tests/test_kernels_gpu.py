@@ -119,6 +119,36 @@ def test_gemm_bf16_cta_pair_kernel_against_one_cta_kernel_and_oracle(M, N, K):
     assert torch.equal(g_pair, g_one)
 
 
+@pytest.mark.parametrize("impl", [0, 2])
+@pytest.mark.parametrize("M,N,K", [(2364, 4096, 4096), (1013, 4096, 11008), (1688, 12288, 4096), (600, 2048, 1024),
+                                   (130, 256, 4096), (3376, 4096, 512)])
+def test_gemm_bf16_split_last_wave_matches_plain_tile_loop(M, N, K, impl):
+    """With a scratch the kernels cut the K loops of the last partial wave of tiles across all SMs and add
+    the parts in a fixed order: same answer as without (to fp32 re-association inside split tiles), right
+    against fp64, identical from run to run, and the scratch is all zero again afterwards."""
+    A = _rand((M, K), 31, torch.bfloat16).cuda()
+    Bm = _rand((N, K), 32, torch.bfloat16, 0.05).cuda()
+    R = _rand((M, N), 33, torch.bfloat16).cuda()
+    ws = B.lazy_k_gemm_scratch()
+    plain = B.lazy_k_gemm(A, Bm, R, impl=impl)
+    split = B.lazy_k_gemm(A, Bm, R, impl=impl, scratch=ws)
+    again = B.lazy_k_gemm(A, Bm, R, impl=impl, scratch=ws)
+    B.lazy_device_status()
+    ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(R))
+    assert rel_err(to_np(split), ref) < BF16_STEP_TOL
+    assert rel_err(to_np(split), to_np(plain).astype(np.float64)) < 2e-3
+    assert torch.equal(split, again)
+    assert int(ws[:2048].count_nonzero()) == 0   # the arrival counters (first 2 KiB) are back to zero
+    F = min(N // 2, 1408)
+    g_plain = B.lazy_k_gemm_swiglu(A, Bm[:F].contiguous(), Bm[F:2 * F].contiguous(), impl=impl)
+    g_split = B.lazy_k_gemm_swiglu(A, Bm[:F].contiguous(), Bm[F:2 * F].contiguous(), impl=impl, scratch=ws)
+    B.lazy_device_status()
+    a = O.f64(to_np(A))
+    ref = O.silu(a @ O.f64(to_np(Bm[:F])).T) * (a @ O.f64(to_np(Bm[F:2 * F])).T)
+    assert rel_err(to_np(g_split), ref) < BF16_STEP_TOL
+    assert rel_err(to_np(g_split), to_np(g_plain).astype(np.float64)) < 2e-3
+
+
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 5])
 def test_gemm_bf16_few_rows_weight_streaming_kernel(M):
     """M <= 4 takes the weight-streaming kernel, M = 5 the tensor-core one: same answers."""
