@@ -101,31 +101,57 @@ __device__ __forceinline__ int gemm_tail_dumps(int u, int tt, int num_tiles, int
   return n;
 }
 
-// v[0..32) += the same 32 columns of n partial accumulators, SLOT_STEP slots apart.
-template <int SLOT_STEP>
-__device__ __forceinline__ void gemm_add_partials(float (&v)[32], const float *part_row, int n, int col) {
-  for (int d = 0; d < n; ++d) {
-    const float4 *q = reinterpret_cast<const float4 *>(part_row + (size_t)d * SLOT_STEP * GEMM_SLOT_FLOATS + col);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float4 x = __ldcg(q + j);  // written by other SMs during this launch: read at L2
-      v[4 * j] += x.x;
-      v[4 * j + 1] += x.y;
-      v[4 * j + 2] += x.z;
-      v[4 * j + 3] += x.w;
-    }
-  }
-}
-
-// Dump of one accumulator row (a thread's 256 fp32 columns) to its slot.
-__device__ __forceinline__ void gemm_dump_row(uint32_t taddr, float *slot_row) {
+// A slot holds one CTA's 128 x 256 accumulator as [column quad q = col/4][row][4 floats]: a warp (32
+// consecutive rows) then moves 512 contiguous bytes per instruction, in the dump and in the fix-up.
+__device__ __forceinline__ void gemm_dump_row(uint32_t taddr, float *slot, int row_in_tile) {
 #pragma unroll 1
   for (int c = 0; c < GEMM_ACC_N; c += 32) {
     float v[32];
     tmem_ld_32x32(taddr + (uint32_t)c, v);
-    float4 *q = reinterpret_cast<float4 *>(slot_row + c);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) q[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    for (int j = 0; j < 8; ++j)
+      *reinterpret_cast<float4 *>(slot + ((size_t)(c / 4 + j) * 128 + row_in_tile) * 4) =
+          make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+  }
+}
+
+// Fix-up of a split tile, one thread per accumulator row: the n_parts dumps (slots slot0, slot0 +
+// slot_step, ...) are added, in that order, into the row's accumulator in tensor memory, after which the
+// ordinary epilogue runs as if the tile had been computed whole.  Each dump is first pulled into shared
+// memory with cp.async (64 x 16 bytes per thread in flight at once, where plain loads into registers would
+// leave the fix-up latency-bound); `stage` is 128 KiB of this CTA's operand ring, idle once the tile's last
+// MMA has retired (which the accumulator-full barrier has already told the caller).  A thread reads back
+// only what it copied itself, so no barrier is needed between the copy and the adds.
+__device__ __forceinline__ void gemm_fixup_row(uint32_t taddr, const float *slot0, int slot_step, int n_parts,
+                                               uint8_t *stage, int row_in_tile) {
+  const uint32_t sbase = smem_u32(stage) + (uint32_t)row_in_tile * 16u;
+  for (int p = 0; p < n_parts; ++p) {
+    const float *src = slot0 + (size_t)p * slot_step * GEMM_SLOT_FLOATS + (size_t)row_in_tile * 4;
+#pragma unroll 8
+    for (int q = 0; q < GEMM_ACC_N / 4; ++q)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + (uint32_t)q * 2048u),
+                   "l"(src + (size_t)q * 512)
+                   : "memory");
+    asm volatile("cp.async.wait_all;" ::: "memory");
+#pragma unroll 1
+    for (int c = 0; c < GEMM_ACC_N; c += 32) {
+      float v[32];
+      tmem_ld_32x32(taddr + (uint32_t)c, v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4 x;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                     : "r"(sbase + (uint32_t)(c / 4 + j) * 2048u)
+                     : "memory");
+        v[4 * j] += x.x;
+        v[4 * j + 1] += x.y;
+        v[4 * j + 2] += x.z;
+        v[4 * j + 3] += x.w;
+      }
+      tmem_st_32x32(taddr + (uint32_t)c, reinterpret_cast<const uint32_t *>(v));
+    }
+    tmem_st_wait();
   }
 }
 
@@ -155,15 +181,13 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
 }
 
 // One thread, one row.  taddr: TMEM address of the row's first accumulator column (lane field set);
-// row: global output row; n0: first output column of the tile as the caller sees it; part_row / n_parts:
-// this row in the first of n_parts partial accumulators to add first (finish part of a split tile).  C is [M, ldc];
+// row: global output row; n0: first output column of the tile as the caller sees it.  C is [M, ldc];
 // for EPI_SWIGLU accumulator columns [0,128) are gate features, [128,256) the matching up features and C
 // receives 128 columns per tile.
-template <int EPI, int SLOT_STEP = 1>
+template <int EPI>
 __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n0, int M, int N, int ldc,
                                                   const bf16 *__restrict__ R, bf16 *__restrict__ C,
-                                                  const RopeArgs &rope, DevStatus *status,
-                                                  const float *part_row = nullptr, int n_parts = 0) {
+                                                  const RopeArgs &rope, DevStatus *status) {
   constexpr int BN = GEMM_ACC_N;
   constexpr int TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   bf16 *crow = C + (size_t)row * ldc;
@@ -189,7 +213,6 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       for (int c = 0; c < BN; c += 32) {
         float v[32];
         tmem_ld_32x32(taddr + (uint32_t)c, v);
-        gemm_add_partials<SLOT_STEP>(v, part_row, n_parts, c);
         if (row < M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
@@ -208,8 +231,6 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
           float lo[32], hi[32];
           tmem_ld_32x32(taddr + (uint32_t)(hc + o), lo);
           tmem_ld_32x32(taddr + (uint32_t)(hc + o + 64), hi);
-          gemm_add_partials<SLOT_STEP>(lo, part_row, n_parts, hc + o);
-          gemm_add_partials<SLOT_STEP>(hi, part_row, n_parts, hc + o + 64);
           if (row < M) {
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
@@ -238,11 +259,9 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
   for (int c = 0; c < TILE_N; c += 32) {
     float v[32];
     tmem_ld_32x32(taddr + (uint32_t)c, v);
-    gemm_add_partials<SLOT_STEP>(v, part_row, n_parts, c);
     if (EPI == EPI_SWIGLU) {
       float u[32];
       tmem_ld_32x32(taddr + (uint32_t)(BN / 2 + c), u);
-      gemm_add_partials<SLOT_STEP>(u, part_row, n_parts, BN / 2 + c);
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
     }

@@ -175,7 +175,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       const int row_in_tile = quarter * 32 + lane;
       if (w.mode == 1) {  // partial accumulator of a split tile: to this CTA's slot, then tell the finisher
-        gemm_dump_row(taddr, tail.partials + ((size_t)blockIdx.x * BM + row_in_tile) * BN);
+        gemm_dump_row(taddr, tail.partials + (size_t)blockIdx.x * GEMM_SLOT_FLOATS, row_in_tile);
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -183,14 +183,14 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           atomicAdd(tail.flags + w.tail_idx, 1u);
         }
       } else {
-        int n_parts = 0;
         if (w.mode == 2) {  // first part of a split tile: the other parts' sums come first
-          n_parts = gemm_tail_dumps(blockIdx.x, w.tail_idx, num_tiles, num_kb, tail);
+          const int n_parts = gemm_tail_dumps(blockIdx.x, w.tail_idx, num_tiles, num_kb, tail);
           ok = gemm_tail_wait(tail.flags + w.tail_idx, 4u * (unsigned)n_parts, abort_flag, status);
           if (!ok) break;
+          gemm_fixup_row(taddr, tail.partials + (size_t)(blockIdx.x + 1) * GEMM_SLOT_FLOATS, 1, n_parts, smem,
+                         row_in_tile);
         }
-        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status,
-                               tail.partials + ((size_t)(blockIdx.x + 1) * BM + row_in_tile) * BN, n_parts);
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + w.tail_idx, 1u) == 3u) {  // last warp through: clean for the next launch

@@ -174,7 +174,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       const int row_in_tile = quarter * 32 + lane;
       const int flag_idx = 2 * w.tail_idx + (int)rank;
       if (w.mode == 1) {
-        gemm_dump_row(taddr, tail.partials + ((size_t)(2 * pair + (int)rank) * PBM + row_in_tile) * PBN);
+        gemm_dump_row(taddr, tail.partials + (size_t)(2 * pair + (int)rank) * GEMM_SLOT_FLOATS, row_in_tile);
         __threadfence();
         __syncwarp();
         if (lane == 0) {
@@ -182,16 +182,15 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           atomicAdd(tail.flags + flag_idx, 1u);
         }
       } else {
-        int n_parts = 0;
         if (w.mode == 2) {  // first part of a split tile: the other parts' sums come first
-          n_parts = gemm_tail_dumps(pair, w.tail_idx, num_tiles, num_kb, tail);
+          const int n_parts = gemm_tail_dumps(pair, w.tail_idx, num_tiles, num_kb, tail);
           ok = gemm_tail_wait(tail.flags + flag_idx, 4u * (unsigned)n_parts, abort_flag, status);
           if (!ok) break;
+          // the dumps of the following pairs, same rank: every second slot
+          gemm_fixup_row(taddr, tail.partials + (size_t)(2 * (pair + 1) + (int)rank) * GEMM_SLOT_FLOATS, 2, n_parts,
+                         smem, row_in_tile);
         }
-        // the dumps of the following pairs, same rank: every second slot
-        gemm_epilogue_row<EPI, 2>(taddr, row, n0, M, N, ldc, R, C, rope, status,
-                                  tail.partials + ((size_t)(2 * (pair + 1) + (int)rank) * PBM + row_in_tile) * PBN,
-                                  n_parts);
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + flag_idx, 1u) == 3u) {

@@ -136,7 +136,7 @@ def test_gemm_bf16_split_last_wave_matches_plain_tile_loop(M, N, K, impl):
     B.lazy_device_status()
     ref = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T + O.f64(to_np(R))
     assert rel_err(to_np(split), ref) < BF16_STEP_TOL
-    assert rel_err(to_np(split), to_np(plain).astype(np.float64)) < 2e-3
+    assert rel_err(to_np(split), to_np(plain).astype(np.float64)) < 2.0 ** -7   # one bf16 rounding flip
     assert torch.equal(split, again)
     assert int(ws[:2048].count_nonzero()) == 0   # the arrival counters (first 2 KiB) are back to zero
     F = min(N // 2, 1408)
@@ -146,7 +146,7 @@ def test_gemm_bf16_split_last_wave_matches_plain_tile_loop(M, N, K, impl):
     a = O.f64(to_np(A))
     ref = O.silu(a @ O.f64(to_np(Bm[:F])).T) * (a @ O.f64(to_np(Bm[F:2 * F])).T)
     assert rel_err(to_np(g_split), ref) < BF16_STEP_TOL
-    assert rel_err(to_np(g_split), to_np(g_plain).astype(np.float64)) < 2e-3
+    assert rel_err(to_np(g_split), to_np(g_plain).astype(np.float64)) < 2.0 ** -7
 
 
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 5])
