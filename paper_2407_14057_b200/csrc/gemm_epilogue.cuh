@@ -291,9 +291,14 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
   }  // epilogue kinds
 }
 
-// Splits the last partial wave along K when that pays: `units` persistent units, `cta_per_unit` CTAs each.
-// scratch NULL or too small, a whole number of waves, or a nearly full last wave: plain tile loop.
-inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, void *scratch, size_t scratch_bytes) {
+// Splits the last partial wave along K when that pays: `units` persistent units of `cta_per_unit` CTAs,
+// m_tiles row tiles, M x K activations.  Costs are in K slices (one slice of MMAs ~ 0.4 us): a split tile
+// pays ~5 slices for each dump and ~8 for each part its finisher adds, so tiles are cut into at most four
+// parts, and only when the wave ends at least a fifth earlier than a whole tile would.  The parts of
+// the tiles of one column block run skewed in K, so the B rows of the tail must stay L2-resident (next to
+// A) or they are re-read from HBM.  scratch NULL or too small, or no gain: plain tile loop.
+inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, int m_tiles, long long M,
+                          long long K, void *scratch, size_t scratch_bytes) {
   GemmTail t = {};
   t.first_tail = num_tiles;
   t.tail_units = 0;
@@ -302,16 +307,30 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
     return t;
   const int first = (num_tiles / units) * units, rem = num_tiles - first;
   if (rem == 0) return t;
-  // idle unit-time of the last wave, in K slices, must outweigh the dump and fix-up traffic
-  if ((long long)(units - rem) * num_kb < 16ll * units) return t;
-  long long tu = (long long)rem * num_kb / GEMM_TAIL_MIN_KB;
-  if (tu > units) tu = units;
-  if (tu <= rem) return t;
+  const long long b_tail = (long long)((rem + m_tiles - 1) / m_tiles + 1) * GEMM_ACC_N * K * 2;
+  if (m_tiles > 2 && b_tail + M * K * 2 > 96ll << 20) return t;  // one or two row tiles: B is read once anyway
+  int best_units = 0;
+  long long best_cost = (long long)num_kb * 4 / 5;
+  for (int parts = 2; parts <= 4; ++parts) {
+    long long tu = (long long)rem * parts;
+    if (tu > units) tu = units;
+    if (tu <= rem) continue;
+    const long long per_unit = ((long long)rem * num_kb + tu - 1) / tu;
+    if (per_unit < GEMM_TAIL_MIN_KB) continue;
+    const bool aligned = tu == (long long)rem * parts;  // ranges end on tile boundaries
+    const long long pieces = aligned ? parts : (num_kb + per_unit - 1) / per_unit + 1;
+    const long long cost = per_unit + 5 + 8 * (pieces - 1);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best_units = (int)tu;
+    }
+  }
+  if (best_units == 0) return t;
   t.flags = (unsigned *)scratch;
   t.done = t.flags + GEMM_TAIL_MAX_CTAS;
   t.partials = (float *)((char *)scratch + GEMM_TAIL_COUNTER_BYTES);
   t.first_tail = first;
-  t.tail_units = (int)tu;
+  t.tail_units = best_units;
   return t;
 }
 
