@@ -293,12 +293,13 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
 
 // Splits the last partial wave along K when that pays: `units` persistent units of `cta_per_unit` CTAs,
 // m_tiles row tiles, M x K activations.  Costs are in K slices (one slice of MMAs ~ 0.4 us): a split tile
-// pays ~5 slices for each dump and ~8 for each part its finisher adds, so tiles are cut into at most four
-// parts, and only when the wave ends at least a fifth earlier than a whole tile would.  The parts of
+// pays ~6 slices for its dump and ~10 for each part its finisher adds (measured; extra_cost more for a
+// heavy epilogue), so tiles are cut into at most four parts, and only when the wave then ends at least a
+// fifth earlier than a whole tile would.  The parts of
 // the tiles of one column block run skewed in K, so the B rows of the tail must stay L2-resident (next to
 // A) or they are re-read from HBM.  scratch NULL or too small, or no gain: plain tile loop.
 inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, int m_tiles, long long M,
-                          long long K, void *scratch, size_t scratch_bytes) {
+                          long long K, int extra_cost, void *scratch, size_t scratch_bytes) {
   GemmTail t = {};
   t.first_tail = num_tiles;
   t.tail_units = 0;
@@ -319,7 +320,7 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
     if (per_unit < GEMM_TAIL_MIN_KB) continue;
     const bool aligned = tu == (long long)rem * parts;  // ranges end on tile boundaries
     const long long pieces = aligned ? parts : (num_kb + per_unit - 1) / per_unit + 1;
-    const long long cost = per_unit + 5 + 8 * (pieces - 1);
+    const long long cost = per_unit + 6 + 10 * (pieces - 1) + extra_cost;
     if (cost < best_cost) {
       best_cost = cost;
       best_units = (int)tu;

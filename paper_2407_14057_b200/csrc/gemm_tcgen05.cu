@@ -249,7 +249,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   LAZY_TRY(make_map(&mb1, B1, N, K, BN / 2));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
-  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, cdiv(M, BM), M, K, scratch, scratch_bytes);
+  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, cdiv(M, BM), M, K, EPI == EPI_SWIGLU ? 8 : 0, scratch,
+                                  scratch_bytes);
   const int grid = (tiles < sm_count() && tail.tail_units == 0) ? tiles : sm_count();
   auto kfn = gemm_bf16_tcgen05_kernel<EPI>;
   static bool attr_set = false;

@@ -249,7 +249,8 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
     }
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
-  const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), M, K, scratch, scratch_bytes);
+  const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), M, K,
+                                  EPI == EPI_SWIGLU ? 8 : 0, scratch, scratch_bytes);
   const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
   kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
                                                     rope, tail);
