@@ -240,7 +240,13 @@ def test_7b_varlen_batch_of_8_equals_sequences_run_alone(model7b):
     for s in (0, 3, 7):
         solo.lazy_prefill_run(d_ids[cu[s]:cu[s + 1]].contiguous(), [0, lengths[s]], lg)
         solo.lazy_sync_status()
+        # Sequences are independent.  Not bit-identical, though: which output tiles of a GEMM get their K
+        # loop split across SMs depends on the total row count, and a split tile adds its fp32 partial
+        # sums in another order.  So: the same kept sets up to near-ties at the threshold, the same logits
+        # to bf16 noise.
         for i, (e, _) in enumerate(schedule):
-            assert np.array_equal(to_np(solo.lazy_get_kept(e, 0)), kept_batch[s][i])
-        assert torch.equal(lg[0], logits[s])           # sequences are independent: bit-identical
+            a, b = to_np(solo.lazy_get_kept(e, 0)), kept_batch[s][i]
+            assert len(a) == len(b)
+            assert len(np.intersect1d(a, b)) >= 0.97 * len(a)
+        assert rel_err(to_np(lg[0]), to_np(logits[s]).astype(np.float64)) < 2 * TOL
     solo.close()
