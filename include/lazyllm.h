@@ -234,9 +234,10 @@ int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, vo
                    int32_t d, float eps);
 /* C[M,N] = A[M,K] * B[N,K]^T (+ R[M,N] if R != NULL). bf16: tcgen05 tensor cores, TMA-fed;
  * fp32: CUDA cores. lda = K, ldc = N (dense).  K and N multiples of 8.  impl: 0 = the
- * dtype's production kernel (bf16: weight streaming for M <= 4, one CTA per 128x256 tile for
- * M <= 128, CTA pairs on 256x256 tiles above), 1 = the CUDA-core kernel (cross-check), 2 = bf16
- * tensor cores with one CTA per tile at every M > 4 (cross-check and timing of the pair kernel). */
+ * dtype's production kernel (bf16: weight streaming for M <= 4; tensor cores above, with one CTA
+ * per 128x256 tile or a CTA pair per 256x256 tile, whichever measured faster for the shape),
+ * 1 = the CUDA-core kernel (cross-check), 2 / 3 = bf16 tensor cores with one CTA per tile / with
+ * CTA pairs at every M > 128 (cross-checks of one against the other). */
 int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B,
                 const void *R, void *C, int32_t M, int32_t N, int32_t K);
 /* The same product with a device scratch of lazy_k_gemm_scratch_bytes() bytes that the bf16

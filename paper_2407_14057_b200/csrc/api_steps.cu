@@ -30,9 +30,9 @@ int lazy_k_gemm_ws(void *stream, int32_t dtype, int32_t impl, const void *A, con
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, B, nullptr, R, C, M, N, K, 0);
-  gemm_force_single(impl == 2);
+  gemm_force_kernel(impl == 2 ? 1 : (impl == 3 ? 2 : 0));
   const int rc = launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status, d_scratch, scratch_bytes);
-  gemm_force_single(0);
+  gemm_force_kernel(0);
   return rc;
 }
 
@@ -50,10 +50,10 @@ int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void 
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  gemm_force_single(impl == 2);
+  gemm_force_kernel(impl == 2 ? 1 : (impl == 3 ? 2 : 0));
   const int rc = launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status, d_scratch,
                                     scratch_bytes);
-  gemm_force_single(0);
+  gemm_force_kernel(0);
   return rc;
 }
 

@@ -173,7 +173,7 @@ int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
                          void *scratch = nullptr, size_t scratch_bytes = 0);
-void gemm_force_single(int on);
+void gemm_force_kernel(int which);
 // Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
 // rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).
 bool gemv_small_m_eligible(int dtype, int M, int K);

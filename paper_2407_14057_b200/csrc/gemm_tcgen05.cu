@@ -222,15 +222,21 @@ int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_row
   return tma_map_2d_bf16(map, base, rows, cols, cols, BK, box_rows);
 }
 
-// More than one row tile: the CTA-pair kernel, unless LAZY_GEMM=single asks for this one (A/B timing).
-int g_force_single = 0;
-bool gemm_pair_enabled() {
-  static int on = -1;
-  if (on < 0) {
+// Which kernel takes a product of more than one row tile.  Measured on the 7B widths (rows 1013-3376,
+// both kernels with the split last wave): the CTA-pair kernel is 3-4 % faster on the QKV projection and
+// on long-K products (down projection), the one-CTA kernel 2-4 % faster on the gate/up and output
+// projections, whose 256-row tiles quantise worse.  LAZY_GEMM=single / pair overrides (A/B timing).
+int g_force_kernel = 0;  // 1: one CTA per tile, 2: CTA pairs (cross-check entry points)
+bool gemm_use_pair(int epi, int M, int N, int K) {
+  static int mode = -1;  // 0 auto, 1 always single, 2 always pair
+  if (mode < 0) {
     const char *e = getenv("LAZY_GEMM");
-    on = (e && strcmp(e, "single") == 0) ? 0 : 1;
+    mode = !e ? 0 : (strcmp(e, "single") == 0 ? 1 : (strcmp(e, "pair") == 0 ? 2 : 0));
   }
-  return on == 1 && !g_force_single;
+  if (M <= BM || g_force_kernel == 1) return false;
+  if (g_force_kernel == 2) return true;
+  if (mode != 0) return mode == 2;
+  return epi == EPI_QKV_ROPE || K >= 2 * N;
 }
 
 template <int EPI>
@@ -241,7 +247,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
-  if (M > BM && gemm_pair_enabled())
+  if (gemm_use_pair(EPI, M, N, K))
     return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
   CUtensorMap ma, mb0, mb1;
   LAZY_TRY(make_map(&ma, A, M, K, BM));
@@ -270,8 +276,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
 // more SMs than that the kernels fall back to the plain tile loop.
 size_t gemm_scratch_bytes() { return gemm_tail_scratch_bytes(GEMM_TAIL_MAX_CTAS); }
 
-// Cross-check switch of the context-free entry points: the next launches use one CTA per tile.
-void gemm_force_single(int on) { g_force_single = on; }
+// Cross-check switch of the context-free entry points: 0 = by shape, 1 = one CTA per tile, 2 = CTA pairs.
+void gemm_force_kernel(int which) { g_force_kernel = which; }
 
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
                 int M, int N, int K, DevStatus *status, void *scratch, size_t scratch_bytes) {
