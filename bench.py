@@ -33,12 +33,22 @@ NCU_GEMM_TRAFFIC_BYTES = 193.4e6
 NCU_GEMM_SOURCE_SHA16 = "cefa092589e64b8c"
 
 
-def _gemm_traffic():
+GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "gemm_epilogue.cuh", "tc_common.cuh", "tc_pair.cuh")
+
+
+def _gemm_source_sha16():
     import hashlib
-    src = os.path.join(ROOT, "paper_2407_14057_b200", "csrc", "gemm_tcgen05.cu")
+    h = hashlib.sha256()
+    for name in GEMM_SOURCES:
+        with open(os.path.join(ROOT, "paper_2407_14057_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def _gemm_traffic():
+    """DRAM bytes per GEMM launch from the committed ncu capture, or None once the kernels' sources changed."""
     try:
-        with open(src, "rb") as f:
-            cur = hashlib.sha256(f.read()).hexdigest()[:16]
+        cur = _gemm_source_sha16()
     except OSError:
         return None
     return NCU_GEMM_TRAFFIC_BYTES if cur == NCU_GEMM_SOURCE_SHA16 else None
@@ -339,7 +349,7 @@ def run_gpu(args):
         "e2e": {"value": world * n / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": n * 4, "d2h_bytes_per_step": shape.vocab * 4},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel (QKV, O, gate/up+SwiGLU, down)",
+        "roofline": {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel + gemm_bf16_tcgen05_pair_kernel (QKV, O, gate/up+SwiGLU, down)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_kind": f"sustained bf16, {peaks['source']}", "launches_per_step": g_launch,
                      "ms_per_step": g_ms, "algorithmic_flops_per_launch": g_fl / max(g_launch, 1),
