@@ -21,7 +21,7 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
 }
 
 template <int M_ROWS, bool SWIGLU>
-__global__ void __launch_bounds__(GV_THREADS)
+__global__ void __launch_bounds__(GV_THREADS, 4)
 gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, const bf16 *__restrict__ B1,
                     const bf16 *__restrict__ R, void *__restrict__ C, int N, int K,
                     const bf16 *__restrict__ gain, float eps, int c_f32) {
@@ -29,6 +29,27 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   __shared__ float gv_red[M_ROWS][GV_THREADS / 32];
   const int kvec = K >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Weights do not depend on the kernel before this one: the first batch of this warp's first column is
+  // requested before waiting for that kernel (the launch allows this grid to start while it drains), and
+  // the kernel after this one is released to do the same.  Activations, gains and residuals are touched
+  // only after the wait.
+  constexpr int U = SWIGLU ? 4 : 8;  // weight vectors per lane in flight (x2 matrices for SwiGLU)
+  const int n_first = blockIdx.x * (GV_THREADS / 32) + warp;
+  uint4 wr[U], ur[SWIGLU ? U : 1];  // the batch in flight
+  if (n_first < N) {
+    const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n_first * K);
+    const uint4 *w1 = SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n_first * K) : nullptr;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int v = lane + 32 * u;
+      if (v < kvec) {
+        wr[u] = ld_stream(w0 + v);
+        if (SWIGLU) ur[u] = ld_stream(w1 + v);
+      }
+    }
+  }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int i = threadIdx.x; i < M_ROWS * kvec; i += GV_THREADS)
     gv_smem[i] = reinterpret_cast<const uint4 *>(A)[i];
   __syncthreads();
@@ -71,6 +92,7 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
     __syncthreads();
   }
   const int warps_total = gridDim.x * (GV_THREADS / 32);
+  bool have_first = true;
   for (int n = blockIdx.x * (GV_THREADS / 32) + warp; n < N; n += warps_total) {
     const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n * K);
     const uint4 *w1 = SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n * K) : nullptr;
@@ -78,15 +100,17 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
 #pragma unroll
     for (int m = 0; m < M_ROWS; ++m) acc0[m] = acc1[m] = 0.f;
     // U weight vectors per lane are requested before the first is used: 8 x 16 bytes in flight
-    constexpr int U = SWIGLU ? 4 : 8;
     for (int v0 = lane; v0 < kvec; v0 += 32 * U) {
-      uint4 wr[U], ur[SWIGLU ? U : 1];
+      if (have_first) {  // on its way since before the wait
+        have_first = false;
+      } else {
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int v = v0 + 32 * u;
-        if (v < kvec) {
-          wr[u] = ld_stream(w0 + v);
-          if (SWIGLU) ur[u] = ld_stream(w1 + v);
+        for (int u = 0; u < U; ++u) {
+          const int v = v0 + 32 * u;
+          if (v < kvec) {
+            wr[u] = ld_stream(w0 + v);
+            if (SWIGLU) ur[u] = ld_stream(w1 + v);
+          }
         }
       }
 #pragma unroll
@@ -140,8 +164,19 @@ int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, c
   int blocks = cdiv(N, GV_THREADS / 32);
   const int cap = sm_count() * 4;
   if (blocks > cap) blocks = cap;
-  kfn<<<blocks, GV_THREADS, smem, st>>>((const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R, C,
-                                       N, K, (const bf16 *)gain, eps, c_f32);
+  // programmatic dependent launch: this grid may start while the kernel before it in the stream drains
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks, 1, 1);
+  cfg.blockDim = dim3(GV_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  LAZY_CUDA_OK(cudaLaunchKernelEx(&cfg, kfn, (const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R, C,
+                                  N, K, (const bf16 *)gain, eps, c_f32));
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

@@ -99,6 +99,9 @@ __global__ void score_stats_kernel(const float *__restrict__ logits, const int32
 __global__ void score_mean_kernel(const float *__restrict__ logits, const float *__restrict__ stats,
                                   const int32_t *__restrict__ cu_q, int n_seqs, int n_total,
                                   int n_heads, float *__restrict__ scores) {
+  // lets a following kernel launched as a programmatic dependent (decode: the output projection's weight
+  // streaming) start its weight reads now; it still waits for this grid before touching activations
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int r = t >> 3, sub = t & 7;
   float acc = 0.f;
