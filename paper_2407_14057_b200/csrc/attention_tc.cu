@@ -420,7 +420,6 @@ __global__ void score_from_attention_kernel(const float *__restrict__ p, const f
                                             const float *__restrict__ stats, const int32_t *__restrict__ cu_q,
                                             int n_seqs, int n_total, int n_heads, int max_tiles,
                                             float *__restrict__ scores) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the output projection may set itself up
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int r = t >> 3, part = t & 7;
   float acc = 0.f;

@@ -113,8 +113,6 @@ template <typename T, int THREADS>
 __global__ void rmsnorm_kernel(const T *__restrict__ x, const int32_t *__restrict__ row_idx,
                                const T *__restrict__ g, T *__restrict__ y, int d, float eps) {
   constexpr int V = Elem<T>::kPerVec;
-  // a projection launched as a programmatic dependent may set itself up while this grid runs
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int r = blockIdx.x;
   const size_t src_row = row_idx ? (size_t)row_idx[r] : (size_t)r;
   const T *xr = x + src_row * d;

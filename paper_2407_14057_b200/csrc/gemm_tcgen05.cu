@@ -91,9 +91,6 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  // Launched as a programmatic dependent: everything above (barriers, TMEM, descriptor prefetch) may have
-  // run while the kernel before this one was still draining; operands are touched only from here on.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
   volatile int *abort_flag = &bars->abort_flag;
 
@@ -267,18 +264,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
     LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
     attr_set = true;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3(GEMM_THREADS, 1, 1);
-  cfg.dynamicSmemBytes = GEMM_SMEM_BYTES;
-  cfg.stream = st;
-  cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  LAZY_CUDA_OK(cudaLaunchKernelEx(&cfg, kfn, ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status, rope,
-                                  tail));
+  kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N,
+                                                  status, rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

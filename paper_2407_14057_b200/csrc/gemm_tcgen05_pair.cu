@@ -82,8 +82,6 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   __syncthreads();
   cluster_sync_all();  // both CTAs' barriers exist before anything signals across
   tc_fence_after();
-  // programmatic dependent launch: the set-up above may overlap the end of the kernel before this one
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&bars->tmem_base);
   volatile int *abort_flag = &bars->abort_flag;
 
@@ -254,18 +252,8 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
   const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), M, K,
                                   EPI == EPI_SWIGLU ? 8 : 0, scratch, scratch_bytes);
   const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3(PTHREADS, 1, 1);
-  cfg.dynamicSmemBytes = PAIR_SMEM_BYTES;
-  cfg.stream = st;
-  cudaLaunchAttribute attr;  // the cluster shape is a compile-time attribute of the kernel
-  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr.val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = &attr;
-  cfg.numAttrs = 1;
-  LAZY_CUDA_OK(cudaLaunchKernelEx(&cfg, kfn, ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status, rope,
-                                  tail));
+  kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
+                                                    rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
