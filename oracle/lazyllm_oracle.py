@@ -17,7 +17,9 @@ Readings of points the paper leaves open (all listed in the design document):
     "pruned at layer l+1" by s^l); the cut sits between attention (+ output
     projection + residual) and the MLP of layer e-1, so that MLP already runs on
     the kept rows only and the Aux Cache of layer e-1 holds post-attention,
-    pre-MLP hidden states.
+    pre-MLP hidden states.  The literal alternative (cut after the whole layer, Aux
+    Cache = the layer's output) is the aux_point="post_layer" switch; both give the
+    kept and revived tokens identical values downstream (pinned in the tests).
   * The keep fraction is cumulative, of the ORIGINAL token count, in integer basis
     points; count = ceil(bp*N/10000) clamped to [1, rows present]; count-based
     top-k; ties go to the lower position; the last token is never pruned; kept
@@ -155,12 +157,23 @@ def lm_head(cfg, W, x_row):
 
 
 # --------------------------------------------------------------------------- caches
+# Where in the scoring layer the token set is cut (Section 3.2, Aux Cache paragraph).
+#   "pre_mlp":    between the attention half (attention, output projection, residual) and the MLP, so the
+#                 layer's MLP already runs on the kept rows and the Aux Cache holds post-attention states;
+#                 a revived token first gets the MLP of that layer.
+#   "post_layer": after the whole layer, the literal wording ("stores the hidden states of those pruned
+#                 tokens"): the MLP runs on every row and the Aux Cache holds the layer's output.
+# The MLP is row-wise, so both give every kept or revived token the same values in every later layer.
+AUX_POINTS = ("pre_mlp", "post_layer")
+
+
 class LayerCache:
     """KV cache of one layer with position tags, and the Aux Cache that follows it.
 
     kv: position -> (k [H,dh], v [H,dh]) for every token whose KV exists at this layer.
-    aux: position -> hidden state (post-attention residual stream of this layer) of tokens
-    whose KV exists here but not in the next layer's cache (Aux Cache paragraph).
+    aux: position -> hidden state (post-attention residual stream of this layer, or the layer's
+    output with aux_point "post_layer") of tokens whose KV exists here but not in the next layer's
+    cache (Aux Cache paragraph).
     """
 
     def __init__(self):
@@ -176,8 +189,11 @@ class LayerCache:
 class LazyState:
     """Everything one sequence carries from prefill into decode, plus per-call records."""
 
-    def __init__(self, cfg, schedule):
+    def __init__(self, cfg, schedule, aux_point: str = "pre_mlp"):
+        if aux_point not in AUX_POINTS:
+            raise ValueError(f"aux_point must be one of {AUX_POINTS}")
         self.cfg = cfg
+        self.aux_point = aux_point
         self.schedule = {int(e): int(bp) for e, bp in schedule}
         self.layers = [LayerCache() for _ in range(cfg.n_layers)]
         self.n_tokens = 0                      # tokens seen so far (prompt + generated)
@@ -216,16 +232,16 @@ def validate_schedule(cfg, schedule) -> None:
 
 # --------------------------------------------------------------------------- prefill
 def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]]] = None,
-            keep_records: bool = True) -> LazyState:
+            keep_records: bool = True, aux_point: str = "pre_mlp") -> LazyState:
     """Token-pruned prefill of one prompt (Sections 3.1 and 3.2).
 
     ids: [N] token ids.  schedule: iterable of (layer_entered, cumulative keep in basis
     points of N); layer 0 always sees the whole prompt.  forced_keep: optional
     {layer_entered: kept positions} that replaces the score-based selection at that
-    point (used to replay another implementation's kept sets).
+    point (used to replay another implementation's kept sets).  aux_point: see AUX_POINTS.
     """
     validate_schedule(cfg, schedule)
-    st = LazyState(cfg, schedule)
+    st = LazyState(cfg, schedule, aux_point)
     ids = np.asarray(ids).astype(np.int64)
     N = ids.shape[0]
     st.n_tokens = N
@@ -245,7 +261,8 @@ def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]
             st.score_pos.append(pos.copy())
             st.rows_pos.append(pos.copy())
             st.hidden_after_attn.append(x.copy())
-        if (l + 1) in st.schedule:
+        cut = (l + 1) in st.schedule
+        if cut:   # the selection itself only needs this layer's scores
             n = x.shape[0]
             if forced_keep is not None and (l + 1) in forced_keep:
                 want = set(int(p) for p in forced_keep[l + 1])
@@ -253,12 +270,17 @@ def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]
                 drop = np.asarray([r for r in range(n) if int(pos[r]) not in want], dtype=np.int64)
             else:
                 keep, drop = select_top(s, keep_count(N, st.schedule[l + 1], n), n - 1)
-            for r in drop:
-                cache.aux[int(pos[r])] = x[r].copy()
             st.kept_pos[l + 1] = pos[keep].copy()
             st.dropped_pos[l + 1] = pos[drop].copy()
+        if cut and aux_point == "pre_mlp":
+            for r in drop:
+                cache.aux[int(pos[r])] = x[r].copy()
             x, pos = x[keep], pos[keep]
         x = x + mlp(cfg, lw, x)
+        if cut and aux_point == "post_layer":
+            for r in drop:
+                cache.aux[int(pos[r])] = x[r].copy()
+            x, pos = x[keep], pos[keep]
         if keep_records:
             st.hidden_out.append(x.copy())
     st.logits = lm_head(cfg, W, x[-1])
@@ -343,6 +365,10 @@ def decode_step(cfg, W, st: LazyState, token_id: int,
         st.rows_pos.append(xpos.copy())
         st.hidden_after_attn.append(x.copy())
         X = {int(r): x[i] for i, r in enumerate(xpos)}
+        if (l + 1) in st.schedule and st.aux_point == "post_layer":
+            x = x + mlp(cfg, lw, x)                   # the cut comes after the whole layer
+            st.hidden_out.append(x.copy())
+            X = {int(r): x[i] for i, r in enumerate(xpos)}
         if (l + 1) in st.schedule:
             if forced_keep is not None and (l + 1) in forced_keep:
                 want = set(int(t) for t in forced_keep[l + 1]) | {p}
@@ -364,6 +390,8 @@ def decode_step(cfg, W, st: LazyState, token_id: int,
             st.kept_pos[l + 1] = sel.copy()
             st.revived_pos[l + 1] = np.asarray(need, dtype=np.int64)
             T = sel[sel != p]
+            if st.aux_point == "post_layer":
+                continue                              # revived rows already hold this layer's output
         xpos = np.asarray(sorted(X.keys()), dtype=np.int64)
         x = np.stack([X[int(r)] for r in xpos])
         x = x + mlp(cfg, lw, x)

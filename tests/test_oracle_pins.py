@@ -400,6 +400,67 @@ def test_decode_revived_row_feeds_deferred_mlp():
     assert np.allclose(st.layers[1].kv[p0][1], v[0], atol=1e-13)
 
 
+# ------------------------------------------------------- the cut after the whole layer ("post_layer")
+def test_post_layer_aux_point_prefill_same_tokens_same_values_aux_is_layer_output():
+    """The MLP is row-wise, so cutting after the whole scoring layer instead of before its MLP changes
+    nothing downstream: same kept sets, same hidden states of kept rows, same logits.  Only the Aux Cache
+    differs, and by exactly that layer's MLP (with its residual) applied to the pre-MLP rows."""
+    shape = MINI.with_layers(5)
+    W = weights_to_np(mini_weights(seed=23, shape=shape))
+    ids = to_np(synth.make_prompt(shape.vocab, 47, seed=23))
+    schedule = ((1, 7000), (3, 4000), (4, 2500))
+    a = O.prefill(shape, W, ids, schedule)
+    b = O.prefill(shape, W, ids, schedule, aux_point="post_layer")
+    for e, _ in schedule:
+        assert np.array_equal(a.kept_pos[e], b.kept_pos[e])
+        assert np.array_equal(a.dropped_pos[e], b.dropped_pos[e])
+    for l in range(shape.n_layers):
+        assert np.allclose(a.hidden_out[l], b.hidden_out[l], rtol=0, atol=1e-12)
+        assert set(a.layers[l].kv) == set(b.layers[l].kv)
+        assert set(a.layers[l].aux) == set(b.layers[l].aux)
+        for pos_, xa in a.layers[l].aux.items():
+            want = xa[None] + O.mlp(shape, W["layers"][l], xa[None])
+            assert np.allclose(b.layers[l].aux[pos_], want[0], rtol=0, atol=1e-12)
+    assert np.allclose(a.logits, b.logits, rtol=0, atol=1e-11)
+    with pytest.raises(ValueError):
+        O.prefill(shape, W, ids, schedule, aux_point="mid_layer")
+
+
+def test_post_layer_aux_point_decode_same_logits_selection_and_revivals():
+    """Through decode steps with revival the two cut points stay equivalent: same logits, same re-selected
+    contexts, same revived tokens, each token still computed at most once per layer, Aux = C_l minus
+    C_{l+1}; and a revived token's K/V in the next layer comes straight from its Aux row (no deferred MLP)."""
+    shape = MINI.with_layers(5)
+    W = weights_to_np(mini_weights(seed=29, shape=shape))
+    ids = to_np(synth.make_prompt(shape.vocab, 40, seed=29))
+    schedule = ((1, 7000), (2, 5000), (4, 3000))
+    a = O.prefill(shape, W, ids, schedule)
+    b = O.prefill(shape, W, ids, schedule, aux_point="post_layer")
+    tok = O.greedy(a.logits)
+    revived_total = 0
+    for step in range(8):
+        aux_b_before = [{p_: x.copy() for p_, x in l.aux.items()} for l in b.layers]
+        la = O.decode_step(shape, W, a, tok)
+        lb = O.decode_step(shape, W, b, tok)
+        assert np.allclose(la, lb, rtol=0, atol=1e-10)
+        for e, _ in schedule:
+            assert np.array_equal(a.kept_pos[e], b.kept_pos[e])
+            assert np.array_equal(np.sort(a.revived_pos[e]), np.sort(b.revived_pos[e]))
+            for r in b.revived_pos[e]:                                  # straight from the Aux row
+                x = aux_b_before[e - 1][int(r)][None]
+                _, k, v = O._layer_qkv(shape, W["layers"][e], x, np.array([int(r)]))
+                assert np.allclose(b.layers[e].kv[int(r)][0], k[0], atol=1e-13)
+                assert np.allclose(b.layers[e].kv[int(r)][1], v[0], atol=1e-13)
+            revived_total += len(b.revived_pos[e])
+        c = [set(l.kv.keys()) for l in b.layers]
+        for l in range(shape.n_layers - 1):
+            assert c[l + 1] <= c[l]
+            assert set(b.layers[l].aux.keys()) == c[l] - c[l + 1]
+        assert all(v == 1 for v in b.compute_count.values())
+        tok = O.greedy(la)
+    assert revived_total > 0
+
+
 def test_prune_op_agrees_with_prefill_first_layer():
     shape = MINI
     W = weights_to_np(mini_weights(seed=23))
