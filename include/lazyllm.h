@@ -195,6 +195,14 @@ typedef struct {
 } lazy_kernel_times;
 int lazy_set_kernel_timing(lazy_ctx *ctx, int32_t on);
 int lazy_get_kernel_times(lazy_ctx *ctx, void *stream, lazy_kernel_times *out);
+/* Where the scoring layer is cut (Section 3.2, Aux Cache paragraph).  after_layer = 0 (default): between
+ * the layer's attention half and its MLP, so that MLP already runs on the kept rows, the Aux Cache holds
+ * post-attention hidden states and a revived token first gets that layer's MLP.  after_layer = 1: after
+ * the whole layer, as the paragraph is worded: the MLP runs on every row and the Aux Cache holds layer
+ * outputs.  The MLP is row-wise, so logits, kept sets and revivals are the same either way; what changes
+ * is the Aux Cache content and the number of MLP rows.  Call before lazy_prefill_run: a change of the
+ * setting invalidates the caches of an earlier prefill (decode then returns LAZY_E_STATE). */
+int lazy_set_aux_point(lazy_ctx *ctx, int32_t after_layer);
 /* Synchronises `stream` and returns the first device-side error recorded since the last call
  * of this function (LAZY_OK if none), clearing it. */
 int lazy_sync_status(lazy_ctx *ctx, void *stream);

@@ -96,6 +96,7 @@ _SIGNATURES = {
     "lazy_k_rmsnorm": (_I, [_P, _I, _P, _P, _P, _I, _I, _F]),
     "lazy_k_gemm": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
     "lazy_k_gemm_swiglu": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
+    "lazy_set_aux_point": (_I, [_P, _I]),
     "lazy_k_gemm_scratch_bytes": (_Z, []),
     "lazy_k_gemm_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
     "lazy_k_gemm_swiglu_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
@@ -252,6 +253,9 @@ class LazyPrefill:
         if d_pos is not None:
             self._keep_alive.append(d_pos)
         _check("lazy_set_forced_keep", lib().lazy_set_forced_keep(self.ctx, layer_entered, seq, _ptr(d_pos), n))
+
+    def lazy_set_aux_point(self, after_layer: bool) -> None:
+        _check("lazy_set_aux_point", lib().lazy_set_aux_point(self.ctx, 1 if after_layer else 0))
 
     def lazy_get_hidden(self, layer: int) -> torch.Tensor:
         rows = C.c_int32()

@@ -371,6 +371,24 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status, c->gemm_scratch, c->gemm_scratch_bytes));
 
     const int pt = c->point_at[l + 1];
+    // The layer's MLP on the rows in flight (revived rows included, under the default cut point).
+    auto run_mlp = [&]() -> int {
+      if (gemv_small_m_eligible(dt, M, d)) {
+        LAZY_TRY(launch_gemv_small_m(st, x, c->w_gate[l], c->w_up[l], nullptr, c->act, M, c->F, d, 1, c->g_mlp[l],
+                                     c->cfg.rms_eps, 0));
+      } else {
+        LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
+        LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status,
+                                    c->gemm_scratch, c->gemm_scratch_bytes));
+      }
+      LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status, c->gemm_scratch,
+                           c->gemm_scratch_bytes));
+      return LAZY_OK;
+    };
+    // cut after the whole layer: the MLP runs before the re-selection, and rows revived from the Aux Cache
+    // (layer outputs under that reading) skip it
+    const bool cut_after = pt >= 0 && c->aux_after_layer;
+    if (cut_after) LAZY_TRY(run_mlp());
     if (pt >= 0) {
       // ---- re-select the context by the new token's score
       const float *sel = sc;
@@ -469,16 +487,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
       KLAUNCH_OK();
       c->stats.revived[l + 1] = revived_total;
     }
-    if (gemv_small_m_eligible(dt, M, d)) {
-      LAZY_TRY(launch_gemv_small_m(st, x, c->w_gate[l], c->w_up[l], nullptr, c->act, M, c->F, d, 1, c->g_mlp[l],
-                                   c->cfg.rms_eps, 0));
-    } else {
-      LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
-      LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status, c->gemm_scratch,
-                                  c->gemm_scratch_bytes));
-    }
-    LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status, c->gemm_scratch,
-                         c->gemm_scratch_bytes));
+    if (!cut_after) LAZY_TRY(run_mlp());
   }
   for (int s = 0; s < S; ++s) tab(T_LAST)[s] = tab(T_CU_X)[s + 1] - 1;
   LAZY_TRY(upload(T_LAST));

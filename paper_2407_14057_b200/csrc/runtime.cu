@@ -318,6 +318,15 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
   return LAZY_OK;
 }
 
+int lazy_set_aux_point(lazy_ctx *c, int32_t after_layer) {
+  if (!c || (after_layer != 0 && after_layer != 1)) return LAZY_E_BADARG;
+  if (c->aux_after_layer != (after_layer != 0)) {
+    c->aux_after_layer = after_layer != 0;
+    c->have_prefill = false;  // caches filled under the other reading cannot be decoded from
+  }
+  return LAZY_OK;
+}
+
 void lazy_destroy(lazy_ctx *ctx) { delete ctx; }
 
 const char *lazy_strerror(int status) {
@@ -507,8 +516,23 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
                                                       c->gemm_scratch, c->gemm_scratch_bytes));
 
     const int p = c->point_at[l + 1];
+    // The layer's MLP, on the rows of the current segment.
+    auto run_mlp = [&]() -> int {
+      const int n2 = c->seg_cu[g][n_seqs];
+      TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb, launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
+      TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
+            launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
+                               c->gemm_scratch_bytes));
+      TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
+            launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status, c->gemm_scratch,
+                        c->gemm_scratch_bytes));
+      return LAZY_OK;
+    };
+    // Default: the cut sits between attention and MLP, so the MLP of this layer already runs on the kept
+    // rows.  With aux_after_layer the MLP runs on every row first and the Aux Cache receives layer outputs.
+    const bool cut_after = p >= 0 && c->aux_after_layer;
+    if (cut_after) LAZY_TRY(run_mlp());
     if (p >= 0) {
-      // cut between attention and MLP: the MLP of this layer already runs on the kept rows
       const float *sel = sc;
       bool any_forced = false;
       for (int s = 0; s < n_seqs; ++s)
@@ -541,14 +565,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       char *t = x; x = x2; x2 = t;
       ++g;
     }
+    if (!cut_after) LAZY_TRY(run_mlp());
     const int n2 = c->seg_cu[g][n_seqs];
-    TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb, launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
-    TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
-          launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
-                             c->gemm_scratch_bytes));
-    TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
-          launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status, c->gemm_scratch,
-                      c->gemm_scratch_bytes));
     if (c->capture_on && c->capture)
       LAZY_CUDA_OK(cudaMemcpyAsync(c->capture + (size_t)l * c->cap_rows * rb, x, (size_t)n2 * rb,
                                    cudaMemcpyDeviceToDevice, st));

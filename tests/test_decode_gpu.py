@@ -62,13 +62,14 @@ def _check_state(eng, states, shape, schedule, tol):
                 assert rel_err(to_np(ahid), ref) < tol
 
 
-def run_decode_case(shape, schedule, lengths, dtype, seed, steps, forced=True):
+def run_decode_case(shape, schedule, lengths, dtype, seed, steps, forced=True, aux_point="pre_mlp"):
     tol = 1e-4 if dtype == torch.float32 else 2e-2
     Wn, ids, cu, eng = _setup(shape, schedule, lengths, dtype, seed, max_new=steps)
     S = len(lengths)
     logits = torch.empty((S, shape.vocab), dtype=torch.float32, device="cuda")
     nxt = torch.empty(S, dtype=torch.int32, device="cuda")
-    states = [O.prefill(shape, Wn, to_np(ids)[cu[s]:cu[s + 1]], schedule) for s in range(S)]
+    states = [O.prefill(shape, Wn, to_np(ids)[cu[s]:cu[s + 1]], schedule, aux_point=aux_point) for s in range(S)]
+    eng.lazy_set_aux_point(aux_point == "post_layer")
     if forced:
         for s in range(S):
             for e, _ in schedule:
@@ -140,6 +141,47 @@ def test_decode_bf16_small_model():
 def test_decode_bf16_varlen_batch():
     run_decode_case(synth.SMALL.with_layers(3), ((1, 6000), (2, 3000)), [130, 65, 200], torch.bfloat16,
                     seed=6, steps=3)
+
+
+def test_decode_fp32_cut_after_the_whole_layer():
+    """The literal reading of the Aux Cache paragraph: Aux rows are layer outputs, revived rows skip the MLP."""
+    shape = synth.TINY.with_layers(4)
+    rv = run_decode_case(shape, ((1, 7000), (2, 5000), (3, 3000)), [90, 33], torch.float32, seed=7, steps=5,
+                         aux_point="post_layer")
+    assert rv > 0
+
+
+def test_decode_bf16_cut_after_the_whole_layer():
+    rv = run_decode_case(synth.SMALL, ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16, seed=8, steps=3,
+                         aux_point="post_layer")
+    assert rv > 0
+
+
+def test_both_cut_points_give_the_same_tokens_and_logits_on_the_gpu():
+    shape, schedule, n = synth.SMALL, ((1, 7000), (2, 5000), (3, 3000)), 260
+    W = synth.make_weights(shape, 9, bf16=True)
+    ids = synth.make_prompt(shape.vocab, n, 9).cuda()
+    out = []
+    for after in (False, True):
+        eng = B.LazyPrefill(shape, _to_cuda(W), schedule, torch.bfloat16, 1, n, max_new_tokens=2)
+        eng.lazy_set_aux_point(after)
+        lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+        eng.lazy_prefill_run(ids, [0, n], lg)
+        eng.lazy_sync_status()
+        kept = [to_np(eng.lazy_get_kept(e, 0)) for e, _ in schedule]
+        aux = [to_np(eng.lazy_get_aux(e - 1, 0)[1]).copy() for e, _ in schedule]
+        out.append((to_np(lg[0]).copy(), kept, aux, list(eng.lazy_get_stats().rows_computed)[:shape.n_layers]))
+        if after:   # changing the setting drops the caches of the earlier prefill
+            eng.lazy_set_aux_point(False)
+            with pytest.raises(B.LazyError) as e:
+                eng.lazy_decode_step(torch.zeros(1, dtype=torch.int32, device="cuda"), lg, None)
+            assert e.value.status == -7
+        eng.close()
+    (la, ka, aa, ra), (lb, kb, ab, rb) = out
+    assert all(np.array_equal(x, y) for x, y in zip(ka, kb))        # scores come from attention: same sets
+    assert ra == rb
+    assert rel_err(lb, la.astype(np.float64)) < 2e-2
+    assert all(x.shape == y.shape and not np.array_equal(x, y) for x, y in zip(aa, ab))   # Aux content differs
 
 
 def test_decode_errors():
