@@ -142,14 +142,18 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
                 const bf16 *__restrict__ v, int ldkv, bf16 *__restrict__ o,
                 const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base,
                 const int32_t *__restrict__ cu_kv, const int32_t *__restrict__ kv_idx,
-                const int32_t *__restrict__ q_kvlen, int n_heads) {
+                const int32_t *__restrict__ q_kvlen, int n_heads, int n_splits,
+                float *__restrict__ part_o, float *__restrict__ part_ml) {
   extern __shared__ __align__(128) uint8_t fa_smem[];
   const int seq = blockIdx.z, h = blockIdx.y;
   const int q_start = cu_q[seq];
   const int n = cu_q[seq + 1] - q_start;
   const int q_tiles = (n + FA_BM - 1) / FA_BM;
-  if ((int)blockIdx.x >= q_tiles) return;
-  const int qt = q_tiles - 1 - blockIdx.x;  // longest rows first
+  // n_splits > 1 (few query rows, long key lists: decode with revived rows): blockIdx.x also names a
+  // slice of the key tiles; the CTA then leaves an unnormalised partial result per row for a merge kernel
+  const int split = (int)blockIdx.x % n_splits, bx = (int)blockIdx.x / n_splits;
+  if (bx >= q_tiles) return;
+  const int qt = q_tiles - 1 - bx;  // longest rows first
   const int q0 = qt * FA_BM;
   // keys: either the sequence's contiguous cache rows, or the rows a list names (decode)
   const int32_t *kidx = kv_idx ? kv_idx + cu_kv[seq] : nullptr;
@@ -168,15 +172,28 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   // Row i sees the first vis(i) keys; vis is non-decreasing in i (prefill: i + 1).
   const int last_row = min(q0 + FA_BM, n) - 1;
   const int vis_tile = q_kvlen ? min(q_kvlen[q_start + last_row], n_kv) : last_row + 1;
-  const int n_kt = (vis_tile + FA_BN - 1) / FA_BN;  // key tiles up to the diagonal
+  const int n_kt_all = (vis_tile + FA_BN - 1) / FA_BN;  // key tiles up to the diagonal
+  const int tiles_per_split = ((n_kv + FA_BN - 1) / FA_BN + n_splits - 1) / n_splits;
+  const int kt0 = split * tiles_per_split;
+  const int n_kt = min(n_kt_all, kt0 + tiles_per_split);  // this CTA walks key tiles [kt0, n_kt)
+  if (kt0 >= n_kt) {  // nothing visible in this slice: empty partials (n_splits > 1 only)
+    for (int r = threadIdx.x; r < FA_BM; r += FA_THREADS) {
+      if (q0 + r < n) {
+        const size_t pidx = ((size_t)(q_start + q0 + r) * n_heads + h) * n_splits + split;
+        part_ml[pidx * 2] = -INFINITY;
+        part_ml[pidx * 2 + 1] = 0.f;
+      }
+    }
+    return;
+  }
   const int wrow0 = min(q0 + warp * 16 + g, n - 1), wrow1 = min(q0 + warp * 16 + g + 8, n - 1);
   const int vis0 = q_kvlen ? q_kvlen[q_start + wrow0] : wrow0 + 1;
   const int vis1 = q_kvlen ? q_kvlen[q_start + wrow1] : wrow1 + 1;
   const int wfirst = min(q0 + warp * 16, n - 1);
   const int vis_first = q_kvlen ? q_kvlen[q_start + wfirst] : wfirst + 1;
   load_tile(sQ, qg, ldq, q0, n);
-  load_tile(sK, kg, ldkv, 0, n_kv, kidx);
-  load_tile(sV, vg, ldkv, 0, n_kv, kidx);
+  load_tile(sK, kg, ldkv, kt0 * FA_BN, n_kv, kidx);
+  load_tile(sV, vg, ldkv, kt0 * FA_BN, n_kv, kidx);
   cp_async_commit();
 
   uint32_t qf[8][4];
@@ -186,8 +203,8 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
   const float sl2 = rsqrtf((float)FA_D) * 1.4426950408889634f;  // softmax scale in log2 units
 
-  for (int kt = 0; kt < n_kt; ++kt) {
-    const int buf = kt & 1;
+  for (int kt = kt0; kt < n_kt; ++kt) {
+    const int buf = (kt - kt0) & 1;
     if (kt + 1 < n_kt) {  // prefetch the next K/V tile into the other buffer
       load_tile(sK + (buf ^ 1) * FA_TILE_BYTES, kg, ldkv, (kt + 1) * FA_BN, n_kv, kidx);
       load_tile(sV + (buf ^ 1) * FA_TILE_BYTES, vg, ldkv, (kt + 1) * FA_BN, n_kv, kidx);
@@ -197,7 +214,7 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
       cp_async_wait<0>();
     }
     __syncthreads();
-    if (kt == 0) {
+    if (kt == kt0) {
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const int r = warp * 16 + (lane & 15);
@@ -243,16 +260,19 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
     for (int rr = 0; rr < 2; ++rr) {
       mx[rr] = fmaxf(mx[rr], __shfl_xor_sync(0xffffffffu, mx[rr], 1));
       mx[rr] = fmaxf(mx[rr], __shfl_xor_sync(0xffffffffu, mx[rr], 2));
-      const float m_new = fmaxf(m_run[rr], mx[rr]);  // finite: key 0 is visible to every row
-      corr[rr] = exp2f(m_run[rr] - m_new);
+      // finite from the first tile on when the walk starts at key 0 (visible to every row); a later slice
+      // may show a row nothing yet: then everything stays zero and no exponent sees inf - inf
+      const float m_new = fmaxf(m_run[rr], mx[rr]);
+      corr[rr] = m_new == -INFINITY ? 1.f : exp2f(m_run[rr] - m_new);
       m_run[rr] = m_new;
     }
+    const float mref[2] = {m_run[0] == -INFINITY ? 0.f : m_run[0], m_run[1] == -INFINITY ? 0.f : m_run[1]};
     float rs[2] = {0.f, 0.f};
     uint32_t pf[4][4];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const float p0 = exp2f(s[i][0] - m_run[0]), p1 = exp2f(s[i][1] - m_run[0]);
-      const float p2 = exp2f(s[i][2] - m_run[1]), p3 = exp2f(s[i][3] - m_run[1]);
+      const float p0 = exp2f(s[i][0] - mref[0]), p1 = exp2f(s[i][1] - mref[0]);
+      const float p2 = exp2f(s[i][2] - mref[1]), p3 = exp2f(s[i][3] - mref[1]);
       rs[0] += p0 + p1;
       rs[1] += p2 + p3;
       pf[i >> 1][(i & 1) * 2 + 0] = bf16x2_pack(p0, p1);
@@ -287,6 +307,24 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
     l_run[rr] += __shfl_xor_sync(0xffffffffu, l_run[rr], 1);
     l_run[rr] += __shfl_xor_sync(0xffffffffu, l_run[rr], 2);
   }
+  if (n_splits > 1) {  // unnormalised partials: [row, head, split] x (128 fp32 | max in log2 units, sum)
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int row = q0 + warp * 16 + g + rr * 8;
+      if (row < n) {
+        const size_t pidx = ((size_t)(q_start + row) * n_heads + h) * n_splits + split;
+        float *po = part_o + pidx * FA_D + 2 * t4;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          *reinterpret_cast<float2 *>(po + i * 8) = make_float2(oacc[i][rr * 2], oacc[i][rr * 2 + 1]);
+        if (t4 == 0) {
+          part_ml[pidx * 2] = m_run[rr];
+          part_ml[pidx * 2 + 1] = l_run[rr];
+        }
+      }
+    }
+    return;
+  }
   const int ldo = n_heads * FA_D;
 #pragma unroll
   for (int rr = 0; rr < 2; ++rr) {
@@ -320,6 +358,44 @@ int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const v
                              n_seqs, max_len, n_total, n_heads, head_dim);
 }
 
+bool attention_list_split_eligible(int dtype, int head_dim) { return dtype == LAZY_BF16 && head_dim == FA_D; }
+
+// Splits of the key list that put ~4 CTAs on every SM for n_rows query rows (1 = do not split).
+int attention_list_splits(int n_seqs, int max_rows, int n_heads, int max_ctx) {
+  const int ctas = cdiv(max_rows, FA_BM) * n_heads * n_seqs;
+  int s = (4 * sm_count()) / (ctas > 0 ? ctas : 1);
+  const int key_tiles = cdiv(max_ctx, FA_BN);
+  if (s > key_tiles / 4) s = key_tiles / 4;  // at least four key tiles per slice
+  if (s > 8) s = 8;
+  return s < 2 ? 1 : s;
+}
+
+// Key-list attention (decode with many rows in flight) with the key tiles of every (query tile, head) cut
+// into n_splits slices; part: n_total * n_heads * n_splits * 130 floats.  The merge kernel of the
+// split-key decode attention finishes the rows (and leaves the score row's softmax statistics in stats).
+int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const void *k, const void *v, int ldkv,
+                                void *o, const int32_t *cu_q, const int32_t *cu_kv, const int32_t *kv_idx,
+                                const int32_t *q_kvlen, const int32_t *score_row, int n_seqs, int max_rows,
+                                int n_total, int n_heads, int n_splits, float *part, float *stats) {
+  if (n_total == 0 || n_seqs == 0) return LAZY_OK;
+  if (!part || !stats || !score_row || n_splits < 2 || (ldq % 8) || (ldkv % 8)) return LAZY_E_BADARG;
+  static bool attr_set = false;
+  if (!attr_set) {
+    LAZY_CUDA_OK(cudaFuncSetAttribute(attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FA_SMEM_BYTES));
+    attr_set = true;
+  }
+  float *part_o = part;
+  float *part_ml = part + (size_t)n_total * n_heads * n_splits * FA_D;
+  dim3 grid(cdiv(max_rows, FA_BM) * n_splits, n_heads, n_seqs);
+  attn_mma_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>((const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v,
+                                                           ldkv, (bf16 *)o, cu_q, nullptr, cu_kv, kv_idx, q_kvlen,
+                                                           n_heads, n_splits, part_o, part_ml);
+  LAZY_COUNT_LAUNCH();
+  if (launch_ok() != LAZY_OK) return LAZY_E_CUDA;
+  return launch_attention_combine(st, part_o, part_ml, n_splits, cu_q, score_row, n_seqs, n_total, n_heads, o,
+                                  n_heads * FA_D, stats);
+}
+
 int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                         const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                         const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
@@ -335,7 +411,8 @@ int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, cons
     dim3 grid(cdiv(max_len, FA_BM), n_heads, n_seqs);
     attn_mma_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>((const bf16 *)q, ldq, (const bf16 *)k,
                                                              (const bf16 *)v, ldkv, (bf16 *)o, cu_q,
-                                                             kv_base, cu_kv, kv_idx, q_kvlen, n_heads);
+                                                             kv_base, cu_kv, kv_idx, q_kvlen, n_heads, 1, nullptr,
+                                                             nullptr);
     LAZY_COUNT_LAUNCH();
     return launch_ok();
   }

@@ -208,6 +208,18 @@ attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__rest
 
 }  // namespace
 
+// The merge step alone: partials [n_rows, n_heads, n_splits] x (128 fp32 | max in log2 units, sum).
+int launch_attention_combine(cudaStream_t st, const float *part_o, const float *part_ml, int n_splits,
+                             const int32_t *cu_x, const int32_t *score_row, int n_seqs, int n_rows, int n_heads,
+                             void *o, int ldo, float *stats) {
+  if (n_rows == 0) return LAZY_OK;
+  if (n_splits < 1 || n_splits > DK_MAX_SPLITS) return LAZY_E_CAPACITY;
+  attn_decode_combine_kernel<<<dim3(n_heads, n_rows), DK_THREADS, 0, st>>>(part_o, part_ml, n_splits, cu_x, score_row,
+                                                                        n_seqs, (bf16 *)o, ldo, stats);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
 bool attention_decode_eligible(int dtype, int head_dim, int n_rows, int max_ctx) {
   return dtype == LAZY_BF16 && head_dim == DK_HD && n_rows >= 1 && n_rows <= 8 &&
          max_ctx <= DK_MAX_SPLITS * DK_SPLIT;

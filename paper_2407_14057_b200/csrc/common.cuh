@@ -227,6 +227,16 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
                             const int32_t *ctx_rows, const int32_t *q_kvlen, const int32_t *score_row,
                             int n_seqs, int n_rows, int n_ctx_total, int max_ctx, int n_heads,
                             float *part, float *logits, float *stats);
+int launch_attention_combine(cudaStream_t st, const float *part_o, const float *part_ml, int n_splits,
+                             const int32_t *cu_x, const int32_t *score_row, int n_seqs, int n_rows, int n_heads,
+                             void *o, int ldo, float *stats);
+// Key-list attention for many query rows with the key tiles cut into slices (see attention.cu).
+bool attention_list_split_eligible(int dtype, int head_dim);
+int attention_list_splits(int n_seqs, int max_rows, int n_heads, int max_ctx);
+int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const void *k, const void *v, int ldkv,
+                                void *o, const int32_t *cu_q, const int32_t *cu_kv, const int32_t *kv_idx,
+                                const int32_t *q_kvlen, const int32_t *score_row, int n_seqs, int max_rows,
+                                int n_total, int n_heads, int n_splits, float *part, float *stats);
 int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                     const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
                     const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,

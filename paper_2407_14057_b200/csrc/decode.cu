@@ -363,8 +363,17 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
                                        (float *)c->act, logits, stats));
       LAZY_TRY(launch_score_mean(st, logits, stats, dtab(T_CU_CTX), S, n_ctx, c->H, sc));
     } else {
-      LAZY_TRY(launch_attention_ex(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), nullptr,
-                                   dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh));
+      // many rows in flight: the tile kernel, with the key list cut into slices when there are too few
+      // (query tile, head) pairs to fill the machine
+      const int splits = attention_list_split_eligible(dt, c->dh) ? attention_list_splits(S, max_m, c->H, max_ctx) : 1;
+      if (splits > 1 && (size_t)M * c->H * splits * 130 * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
+        LAZY_TRY(launch_attention_list_split(st, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), dtab(T_CU_CTX),
+                                             ctx_rows, q_kvlen, dtab(T_QROW), S, max_m, M, c->H, splits,
+                                             (float *)c->act, c->score_scratch + (size_t)c->H * n_ctx));
+      } else {
+        LAZY_TRY(launch_attention_ex(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), nullptr,
+                                     dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh));
+      }
       LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
                                n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
     }

@@ -138,6 +138,13 @@ def test_decode_bf16_small_model():
     assert rv > 0
 
 
+def test_decode_bf16_long_context_many_rows_in_flight():
+    """1200-token context, hundreds of revived rows per step: the key-list attention then runs with its key
+    tiles cut into slices and merged (too few query tiles x heads to fill the GPU otherwise)."""
+    rv = run_decode_case(synth.SMALL, ((1, 6000), (2, 4000), (3, 2500)), [1200], torch.bfloat16, seed=10, steps=2)
+    assert rv > 50
+
+
 def test_decode_bf16_varlen_batch():
     run_decode_case(synth.SMALL.with_layers(3), ((1, 6000), (2, 3000)), [130, 65, 200], torch.bfloat16,
                     seed=6, steps=3)
