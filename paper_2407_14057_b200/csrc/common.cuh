@@ -180,6 +180,9 @@ bool gemv_small_m_eligible(int dtype, int M, int K);
 int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
                         void *C, int M, int N, int K, int swiglu, const void *gain = nullptr,
                         float eps = 0.f, int c_f32 = 0);
+int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
+                         const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
 int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
                      const void *R, void *C, int M, int N, int K, int swiglu);
 // Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows

@@ -63,6 +63,9 @@ __global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, c
                                    const int32_t *append_at, const int32_t *xpos, const int32_t *ctx_pos,
                                    const int32_t *xmap, int n_seqs, int m, int n, int32_t *kv_row_new,
                                    int32_t *kv_map, int32_t *q_kvlen, int32_t *ctx_rows, DevStatus *status) {
+  // the projection that follows is a programmatic dependent: it may start fetching weights now and
+  // still waits for this grid before it reads the rows computed here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     const int s = seq_of(cu_ctx, n_seqs, i);
@@ -333,24 +336,29 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     if (M > c->cap_rows) return LAZY_E_CAPACITY;
     c->stats.rows_computed[l] = M;
 
-    // one to four rows: the weight-streaming kernel normalises its input rows itself
-    if (gemv_small_m_eligible(dt, M, d)) {
-      LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, 3 * d, d, 0, c->g_attn[l],
-                                   c->cfg.rms_eps, 0));
-    } else {
-      LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
-      LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status, c->gemm_scratch,
-                           c->gemm_scratch_bytes));
-    }
-    {
+    {  // bookkeeping first: the projection below may already write the rows' K/V into their cache rows
       const int n_thr = M > n_ctx ? M : n_ctx;
       dec_prepare_kernel<<<cdiv(n_thr, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), dtab(T_BASE),
                                                            d_append + (size_t)l * W, xpos, ctx_pos, xmap, S, M, n_ctx,
                                                            kv_row_new, kvm, q_kvlen, ctx_rows, status);
       KLAUNCH_OK();
     }
-    LAZY_TRY(launch_rope_kv(st, dt, c->qkv, xpos, c->rope_table, kc, vc, kvp, kv_row_new, M, c->H, c->dh,
-                            c->max_pos, status));
+    if (gemv_small_m_eligible(dt, M, d) && c->dh == 128) {
+      // one to four rows: one weight-streaming kernel does RMSNorm, the projection, RoPE and the cache write
+      LAZY_TRY(launch_gemv_qkv_rope(st, x, c->w_qkv[l], c->qkv, c->g_attn[l], c->cfg.rms_eps, xpos, c->rope_table,
+                                    kc, vc, kvp, kv_row_new, M, d, c->max_pos, status));
+    } else {
+      if (gemv_small_m_eligible(dt, M, d)) {
+        LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, 3 * d, d, 0, c->g_attn[l],
+                                     c->cfg.rms_eps, 0));
+      } else {
+        LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
+        LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status, c->gemm_scratch,
+                             c->gemm_scratch_bytes));
+      }
+      LAZY_TRY(launch_rope_kv(st, dt, c->qkv, xpos, c->rope_table, kc, vc, kvp, kv_row_new, M, c->H, c->dh,
+                              c->max_pos, status));
+    }
     for (int s = 0; s < S; ++s) c->kv_count[l][s] += m_of[s];
     int max_ctx = 0;
     for (int s = 0; s < S; ++s) max_ctx = ctx_n[s] > max_ctx ? ctx_n[s] : max_ctx;

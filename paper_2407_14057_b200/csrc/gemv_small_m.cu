@@ -2,7 +2,9 @@
 // accumulation).  At these sizes the step is pure weight streaming, so the kernel is laid out for
 // HBM: every warp owns output columns, reads each weight row exactly once with 16-byte loads
 // (several in flight per lane), keeps the few activation rows in shared memory, and reduces with
-// shuffles.  Same epilogues as the tensor-core GEMM: plain, + residual, SiLU(gate) * up.
+// shuffles.  Same epilogues as the tensor-core GEMM: plain, + residual, SiLU(gate) * up, and the QKV
+// projection with the rotary embedding and the K/V cache write (a warp then owns the two columns i and
+// i + 64 of a head that rotate together).
 #include "common.cuh"
 
 namespace lazy {
@@ -20,11 +22,43 @@ __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
   return r;
 }
 
-template <int M_ROWS, bool SWIGLU>
+enum { GV_PLAIN = 0, GV_SWIGLU = 1, GV_QKV_ROPE = 2 };
+
+// Operands of the QKV mode (head_dim 128): positions and the (cos, sin) table, the layer's cache rows.
+struct GemvRope {
+  const int32_t *pos;     // [M] original positions
+  const float2 *table;    // [max_pos][64]
+  bf16 *kcache, *vcache;  // [rows, d_model]
+  int32_t *kv_pos;        // position tag per cache row
+  const int32_t *kv_row;  // cache row of input row m
+  int d_model, max_pos;
+  DevStatus *status;
+};
+
+// The weight rows a warp streams for its n-th task.  Plain: output column n.  SwiGLU: gate row n and up
+// row n.  QKV: task n = (section q/k/v, head, i < 64) -> rows of output columns i and i + 64 of that head.
+template <int MODE>
+__device__ __forceinline__ void gv_task_rows(int n, const bf16 *B0, const bf16 *B1, int K, int d_model,
+                                             const uint4 *&w0, const uint4 *&w1, int &col0) {
+  if (MODE == GV_QKV_ROPE) {
+    const int half_d = d_model >> 1;
+    const int sect = n / half_d, u = n - sect * half_d;
+    col0 = sect * d_model + (u >> 6) * 128 + (u & 63);
+    w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)col0 * K);
+    w1 = reinterpret_cast<const uint4 *>(B0 + (size_t)(col0 + 64) * K);
+  } else {
+    col0 = n;
+    w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n * K);
+    w1 = MODE == GV_SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n * K) : nullptr;
+  }
+}
+
+template <int M_ROWS, int MODE>
 __global__ void __launch_bounds__(GV_THREADS, 4)
 gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, const bf16 *__restrict__ B1,
                     const bf16 *__restrict__ R, void *__restrict__ C, int N, int K,
-                    const bf16 *__restrict__ gain, float eps, int c_f32) {
+                    const bf16 *__restrict__ gain, float eps, int c_f32, const GemvRope rope) {
+  constexpr bool SWIGLU = MODE != GV_PLAIN;  // two weight rows per task
   extern __shared__ uint4 gv_smem[];  // [M_ROWS][K/8] activation rows as 16-byte vectors
   __shared__ float gv_red[M_ROWS][GV_THREADS / 32];
   const int kvec = K >> 3;
@@ -37,8 +71,9 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   const int n_first = blockIdx.x * (GV_THREADS / 32) + warp;
   uint4 wr[U], ur[SWIGLU ? U : 1];  // the batch in flight
   if (n_first < N) {
-    const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n_first * K);
-    const uint4 *w1 = SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n_first * K) : nullptr;
+    const uint4 *w0, *w1;
+    int col0;
+    gv_task_rows<MODE>(n_first, B0, B1, K, rope.d_model, w0, w1, col0);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int v = lane + 32 * u;
@@ -94,8 +129,9 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   const int warps_total = gridDim.x * (GV_THREADS / 32);
   bool have_first = true;
   for (int n = blockIdx.x * (GV_THREADS / 32) + warp; n < N; n += warps_total) {
-    const uint4 *w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)n * K);
-    const uint4 *w1 = SWIGLU ? reinterpret_cast<const uint4 *>(B1 + (size_t)n * K) : nullptr;
+    const uint4 *w0, *w1;
+    int col0;
+    gv_task_rows<MODE>(n, B0, B1, K, rope.d_model, w0, w1, col0);
     float acc0[M_ROWS], acc1[M_ROWS];
 #pragma unroll
     for (int m = 0; m < M_ROWS; ++m) acc0[m] = acc1[m] = 0.f;
@@ -144,9 +180,30 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
     for (int m = 0; m < M_ROWS; ++m) {
       float g = warp_sum(acc0[m]);
       float u = SWIGLU ? warp_sum(acc1[m]) : 0.f;
-      if (lane == 0) {
+      if (MODE == GV_QKV_ROPE) {
+        if (lane == 0) {
+          const int d = rope.d_model, sect = col0 / d, cin = col0 - sect * d;  // cin: column i of its head
+          int p = rope.pos[m];
+          if (p < 0 || p >= rope.max_pos) {
+            dev_fail(rope.status, LAZY_E_CAPACITY, W_ROPE_POS, m, p);
+            p = 0;
+          }
+          float o0 = g, o1 = u;
+          if (sect < 2) {  // q and k rotate by the row's original position
+            const float2 cs = rope.table[(size_t)p * 64 + (cin & 63)];
+            o0 = g * cs.x - u * cs.y;
+            o1 = u * cs.x + g * cs.y;
+          }
+          const size_t krow = (size_t)rope.kv_row[m];
+          bf16 *dst = sect == 0 ? reinterpret_cast<bf16 *>(C) + (size_t)m * 3 * d + cin
+                                : (sect == 1 ? rope.kcache : rope.vcache) + krow * d + cin;
+          dst[0] = __float2bfloat16_rn(o0);
+          dst[64] = __float2bfloat16_rn(o1);
+          if (n == 0) rope.kv_pos[krow] = p;
+        }
+      } else if (lane == 0) {
         float out = g;
-        if (SWIGLU) out = g / (1.f + __expf(-g)) * u;
+        if (MODE == GV_SWIGLU) out = g / (1.f + __expf(-g)) * u;
         else if (R) out += __bfloat162float(R[(size_t)m * N + n]);
         if (c_f32) reinterpret_cast<float *>(C)[(size_t)m * N + n] = out;
         else reinterpret_cast<bf16 *>(C)[(size_t)m * N + n] = __float2bfloat16_rn(out);
@@ -155,11 +212,11 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   }
 }
 
-template <int M_ROWS, bool SWIGLU>
+template <int M_ROWS, int MODE>
 int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C, int N,
-               int K, const void *gain, float eps, int c_f32) {
+               int K, const void *gain, float eps, int c_f32, const GemvRope &rope = GemvRope()) {
   const size_t smem = (size_t)M_ROWS * K * 2;
-  auto kfn = gemv_small_m_kernel<M_ROWS, SWIGLU>;
+  auto kfn = gemv_small_m_kernel<M_ROWS, MODE>;
   LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int blocks = cdiv(N, GV_THREADS / 32);
   const int cap = sm_count() * 4;
@@ -176,7 +233,7 @@ int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, c
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   LAZY_CUDA_OK(cudaLaunchKernelEx(&cfg, kfn, (const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R, C,
-                                  N, K, (const bf16 *)gain, eps, c_f32));
+                                  N, K, (const bf16 *)gain, eps, c_f32, rope));
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
@@ -195,8 +252,40 @@ int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const vo
     return LAZY_E_BADARG;
 #define GV_CASE(m)                                                                            \
   case m:                                                                                     \
-    return swiglu ? launch_one<m, true>(st, A, B0, B1, nullptr, C, N, K, gain, eps, c_f32)    \
-                  : launch_one<m, false>(st, A, B0, nullptr, R, C, N, K, gain, eps, c_f32);
+    return swiglu ? launch_one<m, GV_SWIGLU>(st, A, B0, B1, nullptr, C, N, K, gain, eps, c_f32) \
+                  : launch_one<m, GV_PLAIN>(st, A, B0, nullptr, R, C, N, K, gain, eps, c_f32);
+  switch (M) {
+    GV_CASE(1)
+    GV_CASE(2)
+    GV_CASE(3)
+    GV_CASE(4)
+    default: return LAZY_E_BADARG;
+  }
+#undef GV_CASE
+}
+
+// QKV projection of one to four rows (optionally RMS-normalised first) with the rotary embedding and the
+// K/V cache write in its epilogue: qkv [M, 3d] receives the rotated q (its k and v thirds are left
+// untouched), rotated k and v go to cache rows kv_row[m] with their position tag.  head_dim 128.
+int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
+                         const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status) {
+  if (((uintptr_t)x & 15) || ((uintptr_t)w_qkv & 15) || ((uintptr_t)gain & 15) || !pos || !table || !kcache ||
+      !vcache || !kv_pos || !kv_row || (d_model % 128))
+    return LAZY_E_BADARG;
+  GemvRope r;
+  r.pos = pos;
+  r.table = (const float2 *)table;
+  r.kcache = (bf16 *)kcache;
+  r.vcache = (bf16 *)vcache;
+  r.kv_pos = kv_pos;
+  r.kv_row = kv_row;
+  r.d_model = d_model;
+  r.max_pos = max_pos;
+  r.status = status;
+  const int tasks = 3 * d_model / 2;
+#define GV_CASE(m) \
+  case m: return launch_one<m, GV_QKV_ROPE>(st, x, w_qkv, nullptr, nullptr, qkv, tasks, d_model, gain, eps, 0, r);
   switch (M) {
     GV_CASE(1)
     GV_CASE(2)
