@@ -39,7 +39,35 @@ struct GemmTail {
   unsigned *done;    // [tail tiles x ranks] finisher warps through; the last one re-zeroes both
   int first_tail;    // tiles [first_tail, num_tiles) are split along K; num_tiles: nothing is
   int tail_units;    // units that share them
+  int m_band;        // row tiles per band of the tile order (see gemm_tile_coords); >= m_tiles: one band
 };
+
+// Tile order.  Consecutive tile numbers walk the row tiles of one column block, so the units of a wave
+// share a B (weight) tile and read different A tiles.  With very many rows (packed batches, long prompts)
+// one sweep over all row tiles no longer fits in L2 and A would come from HBM once per column block:
+// the row tiles are therefore taken in bands of m_band, each band walking all column blocks before the
+// next band starts (A band + one wave of B stay L2-resident; B is re-read once per band instead).
+__device__ __forceinline__ void gemm_tile_coords(int tile, int m_tiles, int n_tiles, int m_band, int &m_idx,
+                                                 int &n_idx) {
+  if (m_band >= m_tiles) {
+    m_idx = tile % m_tiles;
+    n_idx = tile / m_tiles;
+    return;
+  }
+  const int per_band = m_band * n_tiles;
+  const int band = tile / per_band, r = tile - band * per_band;
+  const int rows = min(m_band, m_tiles - band * m_band);  // the last band may be short
+  n_idx = r / rows;
+  m_idx = band * m_band + (r - n_idx * rows);
+}
+
+// Row tiles per band for tiles of tile_rows rows: one band while A (M x K bf16) is under 96 MiB, else
+// about 64 MiB of A per band.
+inline int gemm_m_band(long long M, long long K, int tile_rows) {
+  if (M * K * 2 <= (96ll << 20)) return 1 << 30;
+  const long long t = (64ll << 20) / (K * 2) / tile_rows;
+  return (int)(t < 4 ? 4 : t);
+}
 
 // Scratch layout: 2 x GEMM_TAIL_MAX_CTAS counters (2 KiB), then one accumulator slot per persistent CTA.
 constexpr int GEMM_TAIL_MAX_CTAS = 160;
@@ -298,18 +326,24 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
 // fifth earlier than a whole tile would.  The parts of
 // the tiles of one column block run skewed in K, so the B rows of the tail must stay L2-resident (next to
 // A) or they are re-read from HBM.  scratch NULL or too small, or no gain: plain tile loop.
-inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, int m_tiles, long long M,
-                          long long K, int extra_cost, void *scratch, size_t scratch_bytes) {
+inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, int m_tiles, int m_band,
+                          long long M, long long K, int extra_cost, void *scratch, size_t scratch_bytes,
+                          double *waves = nullptr) {
   GemmTail t = {};
   t.first_tail = num_tiles;
   t.tail_units = 0;
+  t.m_band = m_band;
+  // *waves: the launch's length in whole-tile times (for the choice between the two kernels)
+  if (waves) *waves = (double)((num_tiles + units - 1) / units);
+  if (m_band < m_tiles) m_tiles = m_tiles % m_band ? m_tiles % m_band : m_band;  // the tail lies in the last band
   if (!scratch || units * cta_per_unit > GEMM_TAIL_MAX_CTAS ||
       scratch_bytes < gemm_tail_scratch_bytes(units * cta_per_unit))
     return t;
   const int first = (num_tiles / units) * units, rem = num_tiles - first;
   if (rem == 0) return t;
   const long long b_tail = (long long)((rem + m_tiles - 1) / m_tiles + 1) * GEMM_ACC_N * K * 2;
-  if (m_tiles > 2 && b_tail + M * K * 2 > 96ll << 20) return t;  // one or two row tiles: B is read once anyway
+  const long long a_rows = M < (long long)m_tiles * 256 ? M : (long long)m_tiles * 256;  // rows of the tail's band
+  if (m_tiles > 2 && b_tail + a_rows * K * 2 > 96ll << 20) return t;  // one or two row tiles: B is read once anyway
   int best_units = 0;
   long long best_cost = (long long)num_kb * 4 / 5;
   for (int parts = 2; parts <= 4; ++parts) {
@@ -327,6 +361,7 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
     }
   }
   if (best_units == 0) return t;
+  if (waves) *waves = (double)(num_tiles / units) + (double)best_cost / (double)num_kb;
   t.flags = (unsigned *)scratch;
   t.done = t.flags + GEMM_TAIL_MAX_CTAS;
   t.partials = (float *)((char *)scratch + GEMM_TAIL_COUNTER_BYTES);

@@ -102,8 +102,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       bool ok = true;
       GemmWork w;
       for (int it = 0; ok && gemm_work_item(it, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++it) {
-        const int m0 = (w.tile % m_tiles) * BM;
-        const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+        int m_idx, n_idx;
+        gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
+        const int m0 = m_idx * BM, n0 = n_idx * TILE_N_OUT;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status, W_GEMM_PRODUCER);
           if (!ok) break;
@@ -165,8 +166,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
     for (; ok && gemm_work_item(local, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-      const int m0 = (w.tile % m_tiles) * BM;
-      const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+      int m_idx, n_idx;
+      gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
+      const int m0 = m_idx * BM, n0 = n_idx * TILE_N_OUT;
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -222,21 +224,33 @@ int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_row
   return tma_map_2d_bf16(map, base, rows, cols, cols, BK, box_rows);
 }
 
-// Which kernel takes a product of more than one row tile.  Measured on the 7B widths (rows 1013-3376,
-// both kernels with the split last wave): the CTA-pair kernel is 3-4 % faster on the QKV projection and
-// on long-K products (down projection), the one-CTA kernel 2-4 % faster on the gate/up and output
-// projections, whose 256-row tiles quantise worse.  LAZY_GEMM=single / pair overrides (A/B timing).
+// Which kernel takes a product of more than one row tile: the one whose launch is estimated shorter.
+// Both cover the same outputs per wave (148 tiles of 128 rows, or 74 pair tiles of 256 rows); what differs is
+// how the row count pads to 128 / 256, how many waves that makes, what the split last wave recovers, and the
+// pair kernel's measured ~6 % shorter wave on the plain / residual / QKV epilogues (none on SwiGLU, whose
+// epilogue dominates the difference).  Measured against both kernels at 1013-23112 rows of the 7B widths the
+// estimate picks the faster one except within ~2 %.  LAZY_GEMM=single / pair overrides (A/B timing).
 int g_force_kernel = 0;  // 1: one CTA per tile, 2: CTA pairs (cross-check entry points)
-bool gemm_use_pair(int epi, int M, int N, int K) {
+bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_bytes) {
   static int mode = -1;  // 0 auto, 1 always single, 2 always pair
+  static int max_pairs = 0;
   if (mode < 0) {
     const char *e = getenv("LAZY_GEMM");
     mode = !e ? 0 : (strcmp(e, "single") == 0 ? 1 : (strcmp(e, "pair") == 0 ? 2 : 0));
+    max_pairs = gemm_pair_max_clusters();
+    if (max_pairs > sm_count() / 2) max_pairs = sm_count() / 2;
   }
-  if (M <= BM || g_force_kernel == 1) return false;
+  if (M <= BM || g_force_kernel == 1 || max_pairs < 1) return false;
   if (g_force_kernel == 2) return true;
   if (mode != 0) return mode == 2;
-  return epi == EPI_QKV_ROPE || K >= 2 * N;
+  const int tile_n = epi == EPI_SWIGLU ? BN / 2 : BN, extra = epi == EPI_SWIGLU ? 8 : 0, num_kb = cdiv(K, BK);
+  double w_one = 0, w_pair = 0;
+  plan_tail(cdiv(M, BM) * cdiv(N, tile_n), num_kb, sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K, extra,
+            scratch, scratch_bytes, &w_one);
+  plan_tail(cdiv(M, 2 * BM) * cdiv(N, tile_n), num_kb, max_pairs, 2, cdiv(M, 2 * BM), gemm_m_band(M, K, 2 * BM), M, K,
+            extra, scratch, scratch_bytes, &w_pair);
+  const double pair_wave = epi == EPI_SWIGLU ? 1.0 : 0.94;
+  return w_pair * pair_wave < w_one;  // a pair tile takes pair_wave x the time of a one-CTA tile
 }
 
 template <int EPI>
@@ -247,7 +261,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
-  if (gemm_use_pair(EPI, M, N, K))
+  if (gemm_use_pair(EPI, M, N, K, scratch, scratch_bytes))
     return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
   CUtensorMap ma, mb0, mb1;
   LAZY_TRY(make_map(&ma, A, M, K, BM));
@@ -255,7 +269,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   LAZY_TRY(make_map(&mb1, B1, N, K, BN / 2));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
-  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, cdiv(M, BM), M, K, EPI == EPI_SWIGLU ? 8 : 0, scratch,
+  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K,
+                                  EPI == EPI_SWIGLU ? 8 : 0, scratch,
                                   scratch_bytes);
   const int grid = (tiles < sm_count() && tail.tail_units == 0) ? tiles : sm_count();
   auto kfn = gemm_bf16_tcgen05_kernel<EPI>;

@@ -93,8 +93,9 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       bool ok = true;
       GemmWork w;
       for (int it = 0; ok && gemm_work_item(it, pair, n_pairs, num_tiles, num_kb, tail, w); ++it) {
-        const int m0 = (w.tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
-        const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+        int m_idx, n_idx;
+        gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
+        const int m0 = m_idx * (2 * PBM) + (int)rank * PBM, n0 = n_idx * TILE_N_OUT;
         for (int kb = w.kb0; kb < w.kb1; ++kb) {
           ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1u, abort_flag, status, W_GEMM_PRODUCER);
           if (!ok) break;
@@ -162,8 +163,9 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     for (; ok && gemm_work_item(local, pair, n_pairs, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-      const int m0 = (w.tile % m_tiles) * (2 * PBM) + (int)rank * PBM;
-      const int n0 = (w.tile / m_tiles) * TILE_N_OUT;
+      int m_idx, n_idx;
+      gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
+      const int m0 = m_idx * (2 * PBM) + (int)rank * PBM, n0 = n_idx * TILE_N_OUT;
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -249,7 +251,7 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
     }
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
-  const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), M, K,
+  const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), gemm_m_band(M, K, 2 * PBM), M, K,
                                   EPI == EPI_SWIGLU ? 8 : 0, scratch, scratch_bytes);
   const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
   kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
