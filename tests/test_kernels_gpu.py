@@ -94,7 +94,8 @@ def test_gemm_fp32(M, N, K):
 
 
 @pytest.mark.parametrize("M,N,K", [(129, 256, 64), (256, 512, 128), (300, 1376, 688), (513, 4096, 4096),
-                                   (3376, 768, 4096), (1013, 4096, 11008)])
+                                   (3376, 768, 4096), (1013, 4096, 11008),
+                                   (13000, 512, 4096), (4600, 768, 11008)])   # A beyond 96 MiB: banded tile order
 def test_gemm_bf16_cta_pair_kernel_against_one_cta_kernel_and_oracle(M, N, K):
     """Above 128 rows a product runs on CTA pairs (256x256 tiles over two SMs, impl=3) or with one CTA per
     128x256 tile (impl=2), whichever is faster for the shape.  Both accumulate a tile's K range in the same
@@ -122,7 +123,7 @@ def test_gemm_bf16_cta_pair_kernel_against_one_cta_kernel_and_oracle(M, N, K):
 
 @pytest.mark.parametrize("impl", [3, 2])
 @pytest.mark.parametrize("M,N,K", [(2364, 4096, 4096), (1013, 4096, 11008), (1688, 12288, 4096), (600, 2048, 1024),
-                                   (130, 256, 4096), (3376, 4096, 512)])
+                                   (130, 256, 4096), (3376, 4096, 512), (12500, 768, 4096)])
 def test_gemm_bf16_split_last_wave_matches_plain_tile_loop(M, N, K, impl):
     """With a scratch the kernels cut the K loops of the last partial wave of tiles across all SMs and add
     the parts in a fixed order: same answer as without (to fp32 re-association inside split tiles), right
