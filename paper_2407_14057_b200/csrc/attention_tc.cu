@@ -9,8 +9,14 @@
 //                S_j = Q K_j^T   (M128 N64 K16 x 8, operands in shared memory, both K-major)
 //                O  += P_j V_j   (M128 N128 K16 x 4, A = P_j read from TMEM, B = V_j as an
 //                                 MN-major shared-memory operand: V stays [key][dh] as loaded)
-//              S is double-buffered: S_{j+1} is issued (once P_{j-1} V_{j-1}, whose P shares its
-//              columns, has retired) before waiting for P_j;
+//              TMEM columns: S (64) | P of even tiles (32) | P of odd tiles (32) | O (128).  P has its
+//              own columns, so the single S buffer is free again as soon as the softmax threads
+//              have loaded S_j into registers ("s free"): S_{j+1} is then issued at once and is
+//              computed underneath the exponentials of tile j, and P_j V_j is issued the moment P_j
+//              arrives.  (With P written over a double-buffered S, S_{j+2} had to wait for
+//              P_j V_j to retire, and the softmax threads sat waiting for S 38 % of the time.)
+//              A tcgen05.commit covers every MMA issued before it, so when S_j is announced
+//              P_{j-2} V_{j-2}, the last reader of the P columns tile j will overwrite, has retired;
 //   warps 2-5  softmax: thread = query row (TMEM lane).  tcgen05.ld its 64 logits, mask the
 //              diagonal tile, running max / sum in registers, P_j packed to bf16 pairs and written
 //              back over S_j's columns with tcgen05.st.  The running max is only raised when
@@ -30,7 +36,7 @@ constexpr int Q_BYTES = TQ * HD * 2;       // 32 KiB: two [128][64] blocks
 constexpr int KV_TILE_BYTES = TK * HD * 2; // 16 KiB: two [64][64] blocks
 constexpr int Q_BLK = TQ * 64 * 2;         // 16 KiB
 constexpr int KV_BLK = TK * 64 * 2;        // 8 KiB
-constexpr int ATT_TMEM_COLS = 256;         // S0 | S1 (64 columns each) | O (128 columns)
+constexpr int ATT_TMEM_COLS = 256;         // S (64) | P even (32) | P odd (32) | O (128 columns)
 constexpr int ATT_THREADS = 192;
 constexpr float RESCALE_LOG2 = 8.f;
 
@@ -40,7 +46,8 @@ struct __align__(8) AttBarriers {
   unsigned long long k_empty[KV_STAGES];
   unsigned long long v_full[KV_STAGES];
   unsigned long long v_empty[KV_STAGES];
-  unsigned long long s_full[2];
+  unsigned long long s_full;   // S_j computed (phase j)
+  unsigned long long s_free;   // S_j loaded into registers by all four softmax warps (phase j)
   unsigned long long p_full[2];
   unsigned long long pv_done;
   uint32_t tmem_base;
@@ -110,10 +117,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(smem_u32(&bars->v_full[s]), 1);
       mbar_init(smem_u32(&bars->v_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars->s_full[b]), 1);
-      mbar_init(smem_u32(&bars->p_full[b]), 4);  // one arrival per softmax warp
-    }
+    mbar_init(smem_u32(&bars->s_full), 1);
+    mbar_init(smem_u32(&bars->s_free), 4);       // one arrival per softmax warp
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->p_full[b]), 4);
     mbar_init(smem_u32(&bars->pv_done), 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -177,27 +183,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (!mbar_wait(smem_u32(&bars->k_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA))
           return false;
         tc_fence_after();
-        const uint32_t tmem_s = tmem_base + (uint32_t)(st * 64);
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
           const uint64_t ad = umma_smem_desc(sQ + (k >> 2) * Q_BLK + (k & 3) * 32);
           const uint64_t bd = umma_smem_desc(sK + st * KV_TILE_BYTES + (k >> 2) * KV_BLK + (k & 3) * 32);
-          umma_bf16(tmem_s, ad, bd, idesc_s, k != 0 ? 1u : 0u);
+          umma_bf16(tmem_base, ad, bd, idesc_s, k != 0 ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars->k_empty[st]));  // K_j is free once S_j is computed
-        umma_commit(smem_u32(&bars->s_full[st]));
+        umma_commit(smem_u32(&bars->s_full));
         return true;
       };
       if (ok) ok = issue_s(0);
       for (int j = 0; j < n_kt && ok; ++j) {
         const int st = j & 1;
-        if (j + 1 < n_kt) {
-          // S_{j+1} lands on the columns that still hold P_{j-1}: MMAs that write different
-          // accumulators are not ordered among themselves, so P_{j-1} V_{j-1} has to retire first.
-          if (j >= 1) {
-            ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_MMA);
-            if (!ok) break;
-          }
+        if (j + 1 < n_kt) {  // S_{j+1} as soon as the softmax threads hold S_j in registers
+          ok = mbar_wait(smem_u32(&bars->s_free), (uint32_t)j & 1u, abort_flag, status, W_ATTN_MMA);
+          if (!ok) break;
           ok = issue_s(j + 1);
           if (!ok) break;
         }
@@ -206,7 +207,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tmem_p = tmem_base + (uint32_t)(st * 64);
+        const uint32_t tmem_p = tmem_base + 64u + (uint32_t)(st * 32);
 #pragma unroll
         for (int k = 0; k < TK / 16; ++k) {
           const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
@@ -233,15 +234,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     float *sc_m = score_row ? sc.mtile + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles : nullptr;
     for (int j = 0; j < n_kt && ok; ++j) {
       const int b = j & 1;
-      ok = mbar_wait(smem_u32(&bars->s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = mbar_wait(smem_u32(&bars->s_full), (uint32_t)j & 1u, abort_flag, status, W_ATTN_SOFTMAX);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const uint32_t t_s = tmem_base + lane_base + (uint32_t)(b * 64);
+      const uint32_t t_s = tmem_base + lane_base;
       uint32_t raw[64];
       tmem_ld_32x32_raw(t_s, raw);
       tmem_ld_32x32_raw(t_s + 32u, raw + 32);
       tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->s_free));  // S's columns may take the next tile
       // running maximum on the raw logits (the softmax scale is positive); the mask only matters on
       // tiles that cross the row's diagonal, so the common tile takes the short path
       const int col0 = j * TK;
@@ -319,7 +323,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           sc_m[j] = m;
         }
       }
-      tmem_st_32x32(t_s, pk);  // P_j over the first 32 columns of S_j
+      tmem_st_32x32(t_s + 64u + (uint32_t)(b * 32), pk);  // P_j: 64 bf16 = 32 columns of its own
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
