@@ -178,72 +178,43 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const uint32_t idesc_s = idesc_bf16(TQ, TK, 0, 0);
       const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
       bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, W_ATTN_MMA);
-      // Two chains of MMAs are in flight at a time: S_{s} = Q K_s^T (8 steps into the S columns) and
-      // O += P_{t} V_{t} (4 steps), t <= s.  The steps of one chain accumulate into the same columns and
-      // pay the tensor pipe's latency one after the other (about 90 / 130 clocks per step against 32 / 64 of
-      // arithmetic), so the chains are issued step by step in turn: a chain advances as soon as what it
-      // reads is there (S: the softmax threads have S_{s-1} in registers and K_s has landed; P V: P_t written
-      // and V_t landed), and neither waits behind the other's latency.
-      int s_tile = 0, s_step = 0, pv_tile = 0, pv_step = 0;
-      bool s_go = false, pv_go = false;
-      unsigned long long idle_since = 0;
-      uint32_t spins = 0;
-      while (ok && pv_tile < n_kt) {
-        bool did = false;
-        if (!s_go && s_tile < n_kt) {
-          const int st = s_tile & 1;
-          s_go = (s_tile == 0 || mbar_try_wait(smem_u32(&bars->s_free), (uint32_t)(s_tile - 1) & 1u)) &&
-                 mbar_try_wait(smem_u32(&bars->k_full[st]), (uint32_t)(s_tile >> 1) & 1u);
-          if (s_go) tc_fence_after();
-        }
-        if (!pv_go) {
-          const int st = pv_tile & 1;
-          pv_go = mbar_try_wait(smem_u32(&bars->p_full[st]), (uint32_t)(pv_tile >> 1) & 1u) &&
-                  mbar_try_wait(smem_u32(&bars->v_full[st]), (uint32_t)(pv_tile >> 1) & 1u);
-          if (pv_go) tc_fence_after();
-        }
-        // The commit that announces S_s covers every MMA issued before it, and the softmax threads rely on
-        // that to overwrite the P columns of tile s-2: the last step of S_s waits until P_{s-2} V_{s-2} has
-        // been issued in full.
-        if (s_go && !(s_step == HD / 16 - 1 && pv_tile < s_tile - 1)) {
-          const int st = s_tile & 1, k = s_step;
+      auto issue_s = [&](int j) -> bool {
+        const int st = j & 1;
+        if (!mbar_wait(smem_u32(&bars->k_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA))
+          return false;
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
           const uint64_t ad = umma_smem_desc(sQ + (k >> 2) * Q_BLK + (k & 3) * 32);
           const uint64_t bd = umma_smem_desc(sK + st * KV_TILE_BYTES + (k >> 2) * KV_BLK + (k & 3) * 32);
           umma_bf16(tmem_base, ad, bd, idesc_s, k != 0 ? 1u : 0u);
-          if (++s_step == HD / 16) {
-            umma_commit(smem_u32(&bars->k_empty[st]));  // K_s is free once S_s is computed
-            umma_commit(smem_u32(&bars->s_full));
-            s_step = 0;
-            s_go = false;
-            ++s_tile;
-          }
-          did = true;
         }
-        if (pv_go) {
-          const int st = pv_tile & 1, k = pv_step;
-          const uint32_t tmem_p = tmem_base + 64u + (uint32_t)(st * 32);
+        umma_commit(smem_u32(&bars->k_empty[st]));  // K_j is free once S_j is computed
+        umma_commit(smem_u32(&bars->s_full));
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < n_kt && ok; ++j) {
+        const int st = j & 1;
+        if (j + 1 < n_kt) {  // S_{j+1} as soon as the softmax threads hold S_j in registers
+          ok = mbar_wait(smem_u32(&bars->s_free), (uint32_t)j & 1u, abort_flag, status, W_ATTN_MMA);
+          if (!ok) break;
+          ok = issue_s(j + 1);
+          if (!ok) break;
+        }
+        ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tmem_p = tmem_base + 64u + (uint32_t)(st * 32);
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
           const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
-          umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (pv_tile | k) != 0 ? 1u : 0u);
-          if (++pv_step == TK / 16) {
-            umma_commit(smem_u32(&bars->v_empty[st]));  // V_t is free once these MMAs retire
-            umma_commit(smem_u32(&bars->pv_done));
-            pv_step = 0;
-            pv_go = false;
-            ++pv_tile;
-          }
-          did = true;
+          umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
         }
-        if (did) {
-          spins = 0;
-        } else if ((++spins & 255u) == 0) {  // nothing to issue: bounded wait for the softmax threads / TMA
-          if (spins == 256u) idle_since = global_timer_ns();
-          if (*abort_flag) ok = false;
-          else if (global_timer_ns() - idle_since > WAIT_LIMIT_NS) {
-            *abort_flag = 1;
-            dev_fail(status, LAZY_E_TIMEOUT, W_ATTN_MMA, (int)blockIdx.x, pv_tile);
-            ok = false;
-          }
-        }
+        umma_commit(smem_u32(&bars->v_empty[st]));  // V_j is free once these MMAs retire
+        umma_commit(smem_u32(&bars->pv_done));
       }
     }
   } else {
