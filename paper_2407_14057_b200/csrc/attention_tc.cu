@@ -5,7 +5,7 @@
 // TMEM columns each), so that one CTA's softmax overlaps the other's MMAs.  Warp roles:
 //   warp 0     TMA: Q once (two 128x64 boxes), then 64-key tiles of K and of V (two 64x64 boxes
 //              each) into two 2-stage rings with their own barriers (one lane per ring);
-//   warp 1     owns TMEM and issues the MMAs from one lane:
+//   warp 1     owns TMEM and issues the S MMAs from one lane (warp 6 the P V MMAs):
 //                S_j = Q K_j^T   (M128 N64 K16 x 8, operands in shared memory, both K-major)
 //                O  += P_j V_j   (M128 N128 K16 x 4, A = P_j read from TMEM, B = V_j as an
 //                                 MN-major shared-memory operand: V stays [key][dh] as loaded)
@@ -15,11 +15,11 @@
 //              computed underneath the exponentials of tile j, and P_j V_j is issued the moment P_j
 //              arrives.  (With P written over a double-buffered S, S_{j+2} had to wait for
 //              P_j V_j to retire, and the softmax threads sat waiting for S 38 % of the time.)
-//              A tcgen05.commit covers every MMA issued before it, so when S_j is announced
-//              P_{j-2} V_{j-2}, the last reader of the P columns tile j will overwrite, has retired;
+//   warp 6     issues P_j V_j from one lane (its own thread: a chain of MMAs blocks its issuer while
+//              the pipe takes it, and S_{j+1} must not queue behind that);
 //   warps 2-5  softmax: thread = query row (TMEM lane).  tcgen05.ld its 64 logits, mask the
 //              diagonal tile, running max / sum in registers, P_j packed to bf16 pairs and written
-//              back over S_j's columns with tcgen05.st.  The running max is only raised when
+//              to the tile's P columns with tcgen05.st (once P_{j-1} V_{j-1} has retired).  The running max is only raised when
 //              it grows by more than 2^8 (then O is rescaled in TMEM after the previous P V
 //              retired); otherwise P is allowed to exceed 1, which fp32/bf16 ranges absorb.
 //              After the last tile: O / l -> bf16 -> global.
@@ -37,7 +37,7 @@ constexpr int KV_TILE_BYTES = TK * HD * 2; // 16 KiB: two [64][64] blocks
 constexpr int Q_BLK = TQ * 64 * 2;         // 16 KiB
 constexpr int KV_BLK = TK * 64 * 2;        // 8 KiB
 constexpr int ATT_TMEM_COLS = 256;         // S (64) | P even (32) | P odd (32) | O (128 columns)
-constexpr int ATT_THREADS = 192;
+constexpr int ATT_THREADS = 224;          // TMA warp, S-issuing warp, 4 softmax warps, P V-issuing warp
 constexpr float RESCALE_LOG2 = 8.f;
 
 struct __align__(8) AttBarriers {
@@ -176,7 +176,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(TQ, TK, 0, 0);
-      const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
       bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag, status, W_ATTN_MMA);
       auto issue_s = [&](int j) -> bool {
         const int st = j & 1;
@@ -194,14 +193,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         return true;
       };
       if (ok) ok = issue_s(0);
+      for (int j = 0; j + 1 < n_kt && ok; ++j) {  // S_{j+1} as soon as the softmax threads hold S_j in registers
+        ok = mbar_wait(smem_u32(&bars->s_free), (uint32_t)j & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        ok = issue_s(j + 1);
+      }
+    }
+  } else if (warp == 6) {
+    // ---------------------------------------------------------------- P V issuer
+    // A thread of its own: issuing a chain of MMAs blocks the issuing thread for as long as the pipe needs
+    // to take them (both resident CTAs queue there), and one thread issuing S_{j+1} and then P_j V_j spent
+    // nearly the whole tile period blocked while the softmax threads idled 30-40 % of it.
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
+      bool ok = true;
       for (int j = 0; j < n_kt && ok; ++j) {
         const int st = j & 1;
-        if (j + 1 < n_kt) {  // S_{j+1} as soon as the softmax threads hold S_j in registers
-          ok = mbar_wait(smem_u32(&bars->s_free), (uint32_t)j & 1u, abort_flag, status, W_ATTN_MMA);
-          if (!ok) break;
-          ok = issue_s(j + 1);
-          if (!ok) break;
-        }
         ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
         if (!ok) break;
         ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
@@ -322,6 +329,14 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           }
           sc_m[j] = m;
         }
+      }
+      // P_j goes where P_{j-2} was.  P_{j-2} V_{j-2} is issued by another thread than the S MMAs, so S_j's
+      // arrival says nothing about it; P_{j-1} V_{j-1} having retired does (same thread, issued in order), and
+      // that phase cannot be overtaken before P_j exists.
+      if (j >= 2) {
+        ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
       }
       tmem_st_32x32(t_s + 64u + (uint32_t)(b * 32), pk);  // P_j: 64 bf16 = 32 columns of its own
       tmem_st_wait();
