@@ -261,62 +261,25 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         for (int c = 0; c < 64; ++c)
           if (col0 + c > row) raw[c] = 0xff800000u;  // -inf
       }
-      // One pass over the row's 64 logits: p = 2^(s * scale - m) against the running reference m (one FFMA
-      // and one ex2 per element), the row sum, P packed to bf16 pairs, and the tile's own maximum on the raw
-      // logits (the softmax scale is positive).  The reference is only raised when a tile's maximum exceeds it
-      // by more than 2^8, which the pass finds out at its end: that tile is then done again with the new
-      // reference (rare after the first tiles); otherwise P simply exceeds 1, which fp32/bf16 ranges absorb.
-      float sm[4];
-      float mx[4];
-      uint32_t pk[32];
-      auto pass = [&](float neg_ref) {
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: shorter dependency
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          sm[i] = 0.f;
-          mx[i] = -INFINITY;
-        }
-#pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          const float s0 = __uint_as_float(raw[c]), s1 = __uint_as_float(raw[c + 1]);
-          const float s2 = __uint_as_float(raw[c + 2]), s3 = __uint_as_float(raw[c + 3]);
-          const float p0 = ex2_approx(fmaf(s0, sl2, neg_ref));
-          const float p1 = ex2_approx(fmaf(s1, sl2, neg_ref));
-          const float p2 = ex2_approx(fmaf(s2, sl2, neg_ref));
-          const float p3 = ex2_approx(fmaf(s3, sl2, neg_ref));
-          mx[0] = fmaxf(mx[0], s0);
-          mx[1] = fmaxf(mx[1], s1);
-          mx[2] = fmaxf(mx[2], s2);
-          mx[3] = fmaxf(mx[3], s3);
-          sm[0] += p0;
-          sm[1] += p1;
-          sm[2] += p2;
-          sm[3] += p3;
-          pk[c >> 1] = bf16x2_pack(p0, p1);
-          pk[(c >> 1) + 1] = bf16x2_pack(p2, p3);
-        }
-      };
+      for (int c = 0; c < 64; c += 4) {
+        mx[0] = fmaxf(mx[0], __uint_as_float(raw[c]));
+        mx[1] = fmaxf(mx[1], __uint_as_float(raw[c + 1]));
+        mx[2] = fmaxf(mx[2], __uint_as_float(raw[c + 2]));
+        mx[3] = fmaxf(mx[3], __uint_as_float(raw[c + 3]));
+      }
+      const float mj = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;  // log2 units
       float alpha = 1.f;
-      if (j == 0) {  // no reference yet: the maximum first (key 0 is visible to every row: finite)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) mx[i] = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          mx[0] = fmaxf(mx[0], __uint_as_float(raw[c]));
-          mx[1] = fmaxf(mx[1], __uint_as_float(raw[c + 1]));
-          mx[2] = fmaxf(mx[2], __uint_as_float(raw[c + 2]));
-          mx[3] = fmaxf(mx[3], __uint_as_float(raw[c + 3]));
-        }
-        m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;  // log2 units
-        pass(-m);
+      if (j == 0) {
+        m = mj;  // key 0 is visible to every row: finite
       } else {
-        pass(-m);
-        const float mj = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;
         const bool need = mj - m > RESCALE_LOG2;
+        if (need) {
+          alpha = ex2_approx(m - mj);
+          m = mj;
+        }
         if (__any_sync(0xffffffffu, need)) {
-          if (need) {
-            alpha = ex2_approx(m - mj);
-            m = mj;
-          }
           // O must be at rest: the previous P V has to retire before it is rescaled in place
           ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
           ok = __all_sync(0xffffffffu, ok);
@@ -332,10 +295,25 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             tmem_st_32x32(tmem_o + lane_base + (uint32_t)c, ov);
           }
           tmem_st_wait();
-          pass(-m);  // the rows whose reference moved get their P again; the others recompute the same values
         }
       }
+      // p = 2^(s * scale - m): one FFMA and one ex2 per element
+      float sm[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[32];
       const float neg_m = -m;
+#pragma unroll
+      for (int c = 0; c < 64; c += 4) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
+        const float p2 = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
+        const float p3 = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
+        sm[0] += p0;
+        sm[1] += p1;
+        sm[2] += p2;
+        sm[3] += p3;
+        pk[c >> 1] = bf16x2_pack(p0, p1);
+        pk[(c >> 1) + 1] = bf16x2_pack(p2, p3);
+      }
       l = l * alpha + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
       if (score_warp) {  // warp-uniform: only the warp that owns the sequence's last row gets here
         if (score_row) {
