@@ -74,21 +74,6 @@ struct AttnScoreOut {
 
 namespace {
 
-// 2^x on the FMA pipe, for a share of the score elements (the softmax threads of the two resident CTAs
-// share four special-function units, and those are the busiest pipe of the kernel): x = i + r with
-// i = round(x), 2^r by a degree-3 polynomial on [-0.5, 0.5] (relative error 7.5e-5, a thirtieth of the bf16
-// step P is rounded to), 2^i by adding i to the exponent field.  x is clamped at -126 (masked keys: 2^-126
-// rounds to a zero weight).
-__device__ __forceinline__ float ex2_fma(float x) {
-  x = fmaxf(x, -126.f);
-  const float xi = x + 12582912.f;  // 1.5 * 2^23: the integer part lands in the low mantissa bits
-  const float r = x - (xi - 12582912.f);
-  float p = fmaf(r, 0.0551716685f, 0.2426111251f);
-  p = fmaf(p, r, 0.6932609677f);
-  p = fmaf(p, r, 0.9999280572f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(xi) << 23));
-}
-
 // 2^x on the special-function unit; ex2(-inf) = 0.
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -321,7 +306,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const float p0 = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
         const float p1 = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
         const float p2 = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
-        const float p3 = ex2_fma(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));  // every fourth on the FMA pipe
+        const float p3 = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
         sm[0] += p0;
         sm[1] += p1;
         sm[2] += p2;
