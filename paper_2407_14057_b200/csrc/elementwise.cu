@@ -118,37 +118,14 @@ __global__ void rmsnorm_kernel(const T *__restrict__ x, const int32_t *__restric
   const T *xr = x + src_row * d;
   T *yr = y + (size_t)r * d;
   const int nvec = d / V;
-  // up to four 16-byte vectors per thread stay in registers between the two passes (d <= 4096 in bf16
-  // with 128 threads): the row is then read once
-  constexpr int KEEP = 4;
-  const bool cached = nvec <= KEEP * THREADS;
-  Vec16<T> keep[KEEP];
   float ss = 0.f;
-  if (cached) {
+  for (int i = threadIdx.x; i < nvec; i += THREADS) {
+    Vec16<T> v;
+    v.load(xr + i * V);
+    float f[V];
+    v.unpack(f);
 #pragma unroll
-    for (int u = 0; u < KEEP; ++u) {
-      const int i = threadIdx.x + u * THREADS;
-      if (i < nvec) keep[u].load(xr + i * V);
-    }
-#pragma unroll
-    for (int u = 0; u < KEEP; ++u) {
-      const int i = threadIdx.x + u * THREADS;
-      if (i < nvec) {
-        float f[V];
-        keep[u].unpack(f);
-#pragma unroll
-        for (int j = 0; j < V; ++j) ss += f[j] * f[j];
-      }
-    }
-  } else {
-    for (int i = threadIdx.x; i < nvec; i += THREADS) {
-      Vec16<T> v;
-      v.load(xr + i * V);
-      float f[V];
-      v.unpack(f);
-#pragma unroll
-      for (int j = 0; j < V; ++j) ss += f[j] * f[j];
-    }
+    for (int j = 0; j < V; ++j) ss += f[j] * f[j];
   }
   __shared__ float part[THREADS / 32];
   ss = warp_sum(ss);
@@ -158,24 +135,6 @@ __global__ void rmsnorm_kernel(const T *__restrict__ x, const int32_t *__restric
 #pragma unroll
   for (int w = 0; w < THREADS / 32; ++w) tot += part[w];
   const float scale = rsqrtf(tot / (float)d + eps);
-  if (cached) {
-#pragma unroll
-    for (int u = 0; u < KEEP; ++u) {
-      const int i = threadIdx.x + u * THREADS;
-      if (i < nvec) {
-        Vec16<T> gv, o;
-        gv.load(g + i * V);
-        float f[V], gf[V];
-        keep[u].unpack(f);
-        gv.unpack(gf);
-#pragma unroll
-        for (int j = 0; j < V; ++j) f[j] = f[j] * scale * gf[j];
-        o.pack(f);
-        o.store(yr + i * V);
-      }
-    }
-    return;
-  }
   for (int i = threadIdx.x; i < nvec; i += THREADS) {
     Vec16<T> v, gv, o;
     v.load(xr + i * V);
