@@ -304,6 +304,16 @@ int lazy_k_score_static(void *stream, int32_t dtype, const void *q, int32_t ldq,
  * d_cu_in[s]-d_cu_keep[s]. */
 int lazy_k_select(void *stream, const float *scores, const int32_t *d_cu_in,
                   const int32_t *d_cu_keep, int32_t n_seqs, int32_t *keep_idx, int32_t *drop_idx);
+/* The same selection read as a threshold (Section 3.2: a token is pruned if its score is smaller than the
+ * k-th percentile among the input tokens): per sequence of n rows, tau = the order statistic with
+ * index floor((n-1) * prune_bp / 10000) from below (prune_bp = percentile in basis points, 0..9999; the
+ * "lower" percentile definition, no interpolation), every row with score >= tau is kept, the last row
+ * always.  Ties at tau are all kept, so the count depends on the data: keep_idx / drop_idx (device
+ * int32[n_total]) are packed per sequence from d_cu_in[s], ascending, and d_counts[s] (device
+ * int32[n_seqs]) receives the number kept.  A step-level call: the prefill and decode calls above use
+ * the count-based form, whose counts the host knows before launching. */
+int lazy_k_select_threshold(void *stream, const float *scores, const int32_t *d_cu_in, int32_t n_seqs,
+                            uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *d_counts);
 /* dst[i,:] = src[idx[i],:] for i < n (row gather), rows of `row_bytes` bytes (multiple of 16);
  * src has src_rows rows (indices outside are reported, not dereferenced). */
 int lazy_k_gather_rows(void *stream, const void *src, const int32_t *idx, void *dst, int32_t n,

@@ -129,6 +129,27 @@ def select_top(scores: np.ndarray, n_keep: int, forced: int) -> Tuple[np.ndarray
 
 
 # --------------------------------------------------------------------------- model pieces
+def select_threshold(scores: np.ndarray, prune_bp: int) -> Tuple[np.ndarray, np.ndarray]:
+    """The selection of Section 3.2 read as a threshold: a token is pruned if its score is smaller than
+    the prune_bp/100-th percentile of the scores; the last token is never pruned.
+
+    Percentile = the order statistic with index floor((n-1) * prune_bp / 10000) from below (the "lower"
+    definition: no interpolation, so the threshold is one of the scores and comparisons are exact in
+    the scores' own precision).  Ties at the threshold are all kept: the count depends on the data.
+    Returns (kept, dropped) row indices, ascending.
+    """
+    s = np.asarray(scores)
+    n = s.shape[0]
+    if n == 0:
+        return np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int64)
+    if not 0 <= prune_bp <= 9999:
+        raise ValueError("prune_bp must be in 0..9999")
+    tau = np.sort(s)[((n - 1) * int(prune_bp)) // 10000]
+    keep = np.asarray([i for i in range(n) if s[i] >= tau or i == n - 1], dtype=np.int64)
+    drop = np.asarray([i for i in range(n) if not (s[i] >= tau or i == n - 1)], dtype=np.int64)
+    return keep, drop
+
+
 def _layer_qkv(cfg, lw, x, pos):
     """Pre-norm, QKV projection, head split, RoPE on q and k."""
     H, dh, d = cfg.n_heads, cfg.head_dim, cfg.d_model

@@ -106,6 +106,7 @@ _SIGNATURES = {
     "lazy_k_score": (_I, [_P, _I, _P, _I, _P, _I, _P, _I, _I, _I, _I, _P, _P]),
     "lazy_k_score_static": (_I, [_P, _I, _P, _I, _P, _I, _P, _I, _I, _I, _I, _P]),
     "lazy_k_select": (_I, [_P, _P, _P, _P, _I, _P, _P]),
+    "lazy_k_select_threshold": (_I, [_P, _P, _P, _I, C.c_uint32, _P, _P, _P]),
     "lazy_k_gather_rows": (_I, [_P, _P, _P, _P, _I, _I, _I]),
 }
 
@@ -417,6 +418,19 @@ def lazy_k_select(scores: torch.Tensor, cu_in: torch.Tensor, cu_keep: torch.Tens
     _check("lazy_k_select", lib().lazy_k_select(_stream(), _ptr(scores), _ptr(cu_in), _ptr(cu_keep), n_seqs,
                                                 _ptr(keep), _ptr(drop)))
     return keep[:n_keep], drop[:n_in - n_keep]
+
+
+def lazy_k_select_threshold(scores: torch.Tensor, cu_in: torch.Tensor, prune_bp: int):
+    """Returns (keep_idx, drop_idx, counts): index buffers packed per sequence from cu_in[s], counts per sequence."""
+    n_seqs = cu_in.numel() - 1
+    n_in = int(cu_in[-1].item())
+    keep = torch.full((max(n_in, 1),), -1, dtype=torch.int32, device=scores.device)
+    drop = torch.full((max(n_in, 1),), -1, dtype=torch.int32, device=scores.device)
+    counts = torch.zeros(max(n_seqs, 1), dtype=torch.int32, device=scores.device)
+    _check("lazy_k_select_threshold",
+           lib().lazy_k_select_threshold(_stream(), _ptr(scores), _ptr(cu_in), n_seqs, prune_bp, _ptr(keep),
+                                         _ptr(drop), _ptr(counts)))
+    return keep, drop, counts[:n_seqs]
 
 
 def lazy_k_gather_rows(src: torch.Tensor, idx: torch.Tensor) -> torch.Tensor:

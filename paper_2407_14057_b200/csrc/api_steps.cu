@@ -112,6 +112,14 @@ int lazy_k_select(void *stream, const float *scores, const int32_t *d_cu_in, con
   return launch_select((cudaStream_t)stream, scores, d_cu_in, d_cu_keep, n_seqs, keep_idx, drop_idx, status);
 }
 
+int lazy_k_select_threshold(void *stream, const float *scores, const int32_t *d_cu_in, int32_t n_seqs,
+                            uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *d_counts) {
+  if (!scores || !d_cu_in || !keep_idx || !drop_idx || !d_counts || n_seqs < 0 || prune_bp > 9999)
+    return LAZY_E_BADARG;
+  return launch_select_threshold((cudaStream_t)stream, scores, d_cu_in, n_seqs, prune_bp, keep_idx, drop_idx,
+                                 d_counts);
+}
+
 int lazy_k_gather_rows(void *stream, const void *src, const int32_t *idx, void *dst, int32_t n,
                        int32_t row_bytes, int32_t src_rows) {
   if (n < 0 || row_bytes < 16 || row_bytes % 16 || src_rows < 0) return LAZY_E_BADARG;

@@ -244,6 +244,8 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
                     const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
                     const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,
                     int head_dim, float *scratch, float *scores);
+int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t *cu_in, int n_seqs,
+                            uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts);
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
                   const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
                   DevStatus *status);

@@ -217,6 +217,70 @@ select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_i
   if (threadIdx.x == 0 && kept_so_far != n_keep) dev_fail(status, LAZY_E_STATE, W_SELECT, seq, kept_so_far);
 }
 
+// Threshold form of the selection: tau = the score at the prune_bp/10000 quantile of the sequence's n scores
+// (the order statistic with index floor((n-1) * prune_bp / 10000) from below), every row with score >= tau is
+// kept, and the last row always.  The count depends on the data (ties at tau are all kept), so kept / dropped
+// indices are packed from the sequence's input offset and the count is written to counts[seq].
+__global__ void __launch_bounds__(SEL_THREADS)
+select_threshold_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_in, uint32_t prune_bp,
+                        int32_t *__restrict__ keep_idx, int32_t *__restrict__ drop_idx,
+                        int32_t *__restrict__ counts) {
+  const int seq = blockIdx.x;
+  const int in0 = cu_in[seq], n = cu_in[seq + 1] - in0;
+  if (n == 0) {
+    if (threadIdx.x == 0) counts[seq] = 0;
+    return;
+  }
+  const float *s = scores + in0;
+  __shared__ int hist[256];
+  __shared__ int warp_tot[32];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_k;
+  const int lo = (int)(((long long)(n - 1) * prune_bp) / 10000);
+  // ---- radix select of the (n - lo)-th largest key = the lo-th smallest
+  uint32_t prefix = 0, mask = 0;
+  int k = n - lo;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += SEL_THREADS) {
+      const uint32_t key = score_key(s[i]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int above = 0, b = 255;
+      for (; b > 0; --b) {
+        if (above + hist[b] >= k) break;
+        above += hist[b];
+      }
+      sh_prefix = prefix | ((uint32_t)b << shift);
+      sh_k = k - above;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    k = sh_k;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t tau = prefix;
+  // ---- emit in index order
+  int kept_so_far = 0;
+  for (int base = 0; base < n; base += SEL_THREADS) {
+    const int i = base + threadIdx.x;
+    const bool valid = i < n;
+    const int keep = valid && (i == n - 1 || score_key(s[i]) >= tau);
+    int keep_total;
+    const int keep_rank = kept_so_far + block_excl_scan(keep, warp_tot, &keep_total);
+    if (valid) {
+      if (keep) keep_idx[in0 + keep_rank] = in0 + i;
+      else drop_idx[in0 + (i - keep_rank)] = in0 + i;
+    }
+    kept_so_far += keep_total;
+  }
+  if (threadIdx.x == 0) counts[seq] = kept_so_far;
+}
+
 __global__ void forced_scores_kernel(const int32_t *__restrict__ pos, int r0, int n,
                                      const int32_t *__restrict__ forced, int n_forced,
                                      float *__restrict__ scores) {
@@ -282,6 +346,14 @@ int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, 
   if (!logits || !stats || !cu_q || !scores) return LAZY_E_BADARG;
   score_mean_kernel<<<cdiv(n_total, 32), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
                                                         scores);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t *cu_in, int n_seqs,
+                            uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts) {
+  if (n_seqs == 0) return LAZY_OK;
+  select_threshold_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, prune_bp, keep_idx, drop_idx, counts);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

@@ -189,6 +189,29 @@ def test_gemm_empty_rows_is_a_no_op():
     assert B.lazy_k_gemm(A, Bm).shape == (0, 256)
 
 
+# ------------------------------------------------------------------- selection, threshold form
+@pytest.mark.parametrize("prune_bp", [0, 3000, 5000, 9999])
+def test_select_threshold_matches_oracle_bit_for_bit_with_ties(prune_bp):
+    rng = np.random.default_rng(3)
+    lengths = [1, 5, 1024, 1025, 4097, 300, 0, 2]
+    parts = []
+    for n in lengths:
+        sc = rng.random(n).astype(np.float32)
+        if n >= 300:
+            sc[rng.integers(0, n, n // 3)] = sc[n // 2]        # plant ties, some of them at the threshold
+        parts.append(sc)
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    scores = torch.tensor(np.concatenate(parts)).cuda()
+    keep, drop, counts = B.lazy_k_select_threshold(scores, torch.tensor(cu).cuda(), prune_bp)
+    B.lazy_device_status()
+    keep, drop, counts = to_np(keep), to_np(drop), to_np(counts)
+    for s, n in enumerate(lengths):
+        k_ref, d_ref = O.select_threshold(parts[s], prune_bp)
+        assert counts[s] == len(k_ref)
+        assert np.array_equal(keep[cu[s]:cu[s] + counts[s]] - cu[s], k_ref)
+        assert np.array_equal(drop[cu[s]:cu[s] + n - counts[s]] - cu[s], d_ref)
+
+
 # ------------------------------------------------------------------------------------------ RoPE
 @pytest.mark.parametrize("dtype,H,dh", [(torch.float32, 4, 64), (torch.bfloat16, 4, 128)])
 def test_rope_and_kv_write(dtype, H, dh):

@@ -204,6 +204,32 @@ def test_select_matches_rank_count_brute_force(kind, n):
             assert min(s[free]) >= max(s[drop])
 
 
+def test_select_threshold_is_the_lower_percentile_with_ties_kept():
+    rng = np.random.default_rng(5)
+    for n in (1, 2, 7, 64, 501):
+        s = rng.random(n).astype(np.float32)
+        for bp in (0, 1, 2500, 3000, 5000, 9999):
+            keep, drop = O.select_threshold(s, bp)
+            tau = np.percentile(s, bp / 100.0, method="lower")            # library pin for the threshold
+            want = sorted(set(np.nonzero(s >= tau)[0].tolist()) | {n - 1})
+            assert keep.tolist() == want
+            assert sorted(keep.tolist() + drop.tolist()) == list(range(n))
+            assert len(keep) >= n - ((n - 1) * bp) // 10000                # at least the rank says; more on ties
+    # hand-worked: scores 5 1 3 3 2, 50th percentile (lower) = sorted[2] = 3 -> keep rows 0, 2, 3 and the last
+    keep, drop = O.select_threshold(np.array([5, 1, 3, 3, 2], dtype=np.float32), 5000)
+    assert keep.tolist() == [0, 2, 3, 4] and drop.tolist() == [1]
+    # all equal: nothing can be below the threshold
+    keep, drop = O.select_threshold(np.ones(9, dtype=np.float32), 9000)
+    assert keep.tolist() == list(range(9)) and drop.tolist() == []
+    # without ties the count agrees with the count-based form at the matching count
+    s = rng.permutation(200).astype(np.float32)
+    keep, _ = O.select_threshold(s, 4000)
+    k2, _ = O.select_top(s, len(keep), len(s) - 1)     # the last token counts toward the kept set there too
+    assert keep.tolist() == sorted(k2.tolist())
+    with pytest.raises(ValueError):
+        O.select_threshold(s, 10000)
+
+
 def test_keep_count_worked_values():
     with open(os.path.join(GOLDEN, "keep_counts.txt")) as f:
         rows = [l for l in f if l.strip() and not l.startswith("#")]
