@@ -37,7 +37,7 @@ constexpr int KV_TILE_BYTES = TK * HD * 2; // 16 KiB: two [64][64] blocks
 constexpr int Q_BLK = TQ * 64 * 2;         // 16 KiB
 constexpr int KV_BLK = TK * 64 * 2;        // 8 KiB
 constexpr int ATT_TMEM_COLS = 256;         // S (64) | P even (32) | P odd (32) | O (128 columns)
-constexpr int ATT_THREADS = 320;          // TMA + P V-issuing warp, S-issuing warp, 8 softmax warps
+constexpr int ATT_THREADS = 224;          // TMA warp, S-issuing warp, 4 softmax warps, P V-issuing warp
 constexpr float RESCALE_LOG2 = 8.f;
 
 struct __align__(8) AttBarriers {
@@ -47,14 +47,11 @@ struct __align__(8) AttBarriers {
   unsigned long long v_full[KV_STAGES];
   unsigned long long v_empty[KV_STAGES];
   unsigned long long s_full;   // S_j computed (phase j)
-  unsigned long long s_free;   // S_j loaded into registers by all eight softmax warps (phase j)
+  unsigned long long s_free;   // S_j loaded into registers by all four softmax warps (phase j)
   unsigned long long p_full[2];
   unsigned long long pv_done;
-  unsigned long long xch[4];   // one per TMEM lane quarter: its two softmax warps meet here once per key tile
   uint32_t tmem_base;
   int abort_flag;
-  float xmax[2][2][TQ];        // [tile parity][half][row]: local maxima of the two halves of a tile
-  float xsum[2][TQ];           // [half][row]: partial row sums, exchanged once at the end
 };
 constexpr int ATT_SMEM_BYTES = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 1024 + (int)sizeof(AttBarriers);
 
@@ -76,16 +73,6 @@ struct AttnScoreOut {
 };
 
 namespace {
-
-// 32 lanes x 16 consecutive 32-bit columns from registers to tensor memory.
-__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t *r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
 
 // 2^x on the special-function unit; ex2(-inf) = 0.
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -131,9 +118,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(smem_u32(&bars->v_empty[s]), 1);
     }
     mbar_init(smem_u32(&bars->s_full), 1);
-    mbar_init(smem_u32(&bars->s_free), 8);       // one arrival per softmax warp
-    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->p_full[b]), 8);
-    for (int qd = 0; qd < 4; ++qd) mbar_init(smem_u32(&bars->xch[qd]), 2);
+    mbar_init(smem_u32(&bars->s_free), 4);       // one arrival per softmax warp
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->p_full[b]), 4);
     mbar_init(smem_u32(&bars->pv_done), 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -185,27 +171,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tma_load_2d(sV + st * KV_TILE_BYTES, &map_v, full, h * HD, row);
         tma_load_2d(sV + st * KV_TILE_BYTES + KV_BLK, &map_v, full, h * HD + 64, row);
       }
-    } else if (lane == 2) {
-      // P V issuer: a thread of its own, because issuing a chain of MMAs blocks the issuing thread for as
-      // long as the pipe needs to take them (both resident CTAs queue there); S_{j+1} must not queue behind it.
-      const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
-      bool ok = true;
-      for (int j = 0; j < n_kt && ok; ++j) {
-        const int st = j & 1;
-        ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
-        if (!ok) break;
-        ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t tmem_p = tmem_base + 64u + (uint32_t)(st * 32);
-#pragma unroll
-        for (int k = 0; k < TK / 16; ++k) {
-          const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
-          umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
-        }
-        umma_commit(smem_u32(&bars->v_empty[st]));  // V_j is free once these MMAs retire
-        umma_commit(smem_u32(&bars->pv_done));
-      }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
@@ -234,22 +199,44 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         ok = issue_s(j + 1);
       }
     }
+  } else if (warp == 6) {
+    // ---------------------------------------------------------------- P V issuer
+    // A thread of its own: issuing a chain of MMAs blocks the issuing thread for as long as the pipe needs
+    // to take them (both resident CTAs queue there), and one thread issuing S_{j+1} and then P_j V_j spent
+    // nearly the whole tile period blocked while the softmax threads idled 30-40 % of it.
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16(TQ, HD, 0, 1);
+      bool ok = true;
+      for (int j = 0; j < n_kt && ok; ++j) {
+        const int st = j & 1;
+        ok = mbar_wait(smem_u32(&bars->p_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        ok = mbar_wait(smem_u32(&bars->v_full[st]), (uint32_t)(j >> 1) & 1u, abort_flag, status, W_ATTN_MMA);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tmem_p = tmem_base + 64u + (uint32_t)(st * 32);
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
+          const uint64_t vd = umma_smem_desc_mn(sV + st * KV_TILE_BYTES + k * 2048, KV_BLK, 1024);
+          umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars->v_empty[st]));  // V_j is free once these MMAs retire
+        umma_commit(smem_u32(&bars->pv_done));
+      }
+    }
   } else {
     // ---------------------------------------------------------------- softmax warps
-    const int quarter = warp & 3;          // TMEM lanes [32*quarter, 32*quarter + 32)
-    const int half = (warp - 2) >> 2;      // keys [32*half, 32*half + 32) of every tile
+    const int quarter = warp & 3;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const int rit = quarter * 32 + lane;   // row inside the query tile
-    const int row = q0 + rit;              // index inside the sequence
-    const uint32_t xbar = smem_u32(&bars->xch[quarter]);
+    const int row = q0 + quarter * 32 + lane;  // index inside the sequence
     const float sl2 = rsqrtf((float)HD) * 1.4426950408889634f;
-    float m = -INFINITY, l = 0.f;          // l: this thread's half of the row sum
+    float m = -INFINITY, l = 0.f;
     bool ok = true;
-    // the two threads that own the sequence's last row also record that row's softmax numerators
+    // the thread that owns the sequence's last row also records that row's softmax numerators
     const bool score_row = sc.p != nullptr && row == n - 1;
     const bool score_warp = __any_sync(0xffffffffu, score_row);
     const int seq_id = cu_q ? (int)blockIdx.z : sc.seq_id;
-    // row (seq, h) of P: max_tiles * 64 floats, 16-byte aligned, so half tiles are stored as float4
+    // row (seq, h) of P: max_tiles * 64 floats, 16-byte aligned, so whole tiles are stored as float4
     float *sc_p = score_row ? sc.p + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles * TK : nullptr;
     float *sc_m = score_row ? sc.mtile + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles : nullptr;
     for (int j = 0; j < n_kt && ok; ++j) {
@@ -259,37 +246,30 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if (!ok) break;
       tc_fence_after();
       const uint32_t t_s = tmem_base + lane_base;
-      uint32_t raw[32];
-      tmem_ld_32x32_raw(t_s + (uint32_t)(half * 32), raw);
+      uint32_t raw[64];
+      tmem_ld_32x32_raw(t_s, raw);
+      tmem_ld_32x32_raw(t_s + 32u, raw + 32);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->s_free));  // S's columns may take the next tile
-      // the mask only matters on tiles that cross the row's diagonal: the common tile takes the short path
-      const int col0 = j * TK + half * 32;
-      if (col0 + 31 > row) {
+      // running maximum on the raw logits (the softmax scale is positive); the mask only matters on
+      // tiles that cross the row's diagonal, so the common tile takes the short path
+      const int col0 = j * TK;
+      if (col0 + TK - 1 > row) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c)
+        for (int c = 0; c < 64; ++c)
           if (col0 + c > row) raw[c] = 0xff800000u;  // -inf
       }
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: shorter dependency
 #pragma unroll
-      for (int c = 0; c < 32; c += 4) {
+      for (int c = 0; c < 64; c += 4) {
         mx[0] = fmaxf(mx[0], __uint_as_float(raw[c]));
         mx[1] = fmaxf(mx[1], __uint_as_float(raw[c + 1]));
         mx[2] = fmaxf(mx[2], __uint_as_float(raw[c + 2]));
         mx[3] = fmaxf(mx[3], __uint_as_float(raw[c + 3]));
       }
-      const float mloc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      // meet the thread that holds the other half of the row (bounded wait)
-      bars->xmax[b][half][rit] = mloc;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(xbar);
-      ok = mbar_wait(xbar, (uint32_t)j & 1u, abort_flag, status, W_ATTN_SOFTMAX);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      // running maximum on the raw logits (the softmax scale is positive); identical in both threads
-      const float mj = fmaxf(mloc, bars->xmax[b][half ^ 1][rit]) * sl2;  // log2 units
+      const float mj = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;  // log2 units
       float alpha = 1.f;
       if (j == 0) {
         m = mj;  // key 0 is visible to every row: finite
@@ -306,7 +286,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (!ok) break;
           tc_fence_after();
 #pragma unroll 1
-          for (int c = half * (HD / 2); c < (half + 1) * (HD / 2); c += 32) {  // this thread's 64 columns
+          for (int c = 0; c < HD; c += 32) {
             uint32_t ov[32];
             tmem_ld_32x32_raw(tmem_o + lane_base + (uint32_t)c, ov);
             tmem_ld_wait();
@@ -319,10 +299,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
       // p = 2^(s * scale - m): one FFMA and one ex2 per element
       float sm[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pk[16];
+      uint32_t pk[32];
       const float neg_m = -m;
 #pragma unroll
-      for (int c = 0; c < 32; c += 4) {
+      for (int c = 0; c < 64; c += 4) {
         const float p0 = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
         const float p1 = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
         const float p2 = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
@@ -335,11 +315,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         pk[(c >> 1) + 1] = bf16x2_pack(p2, p3);
       }
       l = l * alpha + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
-      if (score_warp) {  // warp-uniform: only the two warps that own the sequence's last row get here
+      if (score_warp) {  // warp-uniform: only the warp that owns the sequence's last row gets here
         if (score_row) {
           float4 *dst = reinterpret_cast<float4 *>(sc_p + col0);
 #pragma unroll
-          for (int c = 0; c < 32; c += 4) {
+          for (int c = 0; c < 64; c += 4) {
             float4 pv;
             pv.x = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
             pv.y = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
@@ -347,7 +327,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             pv.w = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
             dst[c >> 2] = pv;  // keys past the row hold 0 (masked) and land in the row's padding
           }
-          if (half == 0) sc_m[j] = m;
+          sc_m[j] = m;
         }
       }
       // P_j goes where P_{j-2} was.  P_{j-2} V_{j-2} is issued by another thread than the S MMAs, so S_j's
@@ -358,7 +338,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
-      tmem_st_32x16(t_s + 64u + (uint32_t)(b * 32 + half * 16), pk);  // this half of P_j: 32 bf16 = 16 columns
+      tmem_st_32x32(t_s + 64u + (uint32_t)(b * 32), pk);  // P_j: 64 bf16 = 32 columns of its own
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
@@ -375,25 +355,17 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
       ok = __all_sync(0xffffffffu, ok);
     }
-    if (ok) {  // the row sum is the sum of the two halves
-      bars->xsum[half][rit] = l;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(xbar);
-      ok = mbar_wait(xbar, (uint32_t)n_kt & 1u, abort_flag, status, W_ATTN_SOFTMAX);
-      ok = __all_sync(0xffffffffu, ok);
+    if (ok && score_row) {
+      float *stt = sc.stats + ((size_t)seq_id * gridDim.y + h) * 2;
+      stt[0] = m;
+      stt[1] = 1.f / l;
     }
     if (ok) {
-      l += bars->xsum[half ^ 1][rit];
-      if (score_row && half == 0) {
-        float *stt = sc.stats + ((size_t)seq_id * gridDim.y + h) * 2;
-        stt[0] = m;
-        stt[1] = 1.f / l;
-      }
       tc_fence_after();
       const float inv = 1.f / l;
       bf16 *orow = o + (size_t)(q_start + row) * ldo + h * HD;
 #pragma unroll 1
-      for (int c = half * (HD / 2); c < (half + 1) * (HD / 2); c += 32) {
+      for (int c = 0; c < HD; c += 32) {
         float v[32];
         tmem_ld_32x32(tmem_o + lane_base + (uint32_t)c, v);
         if (row < n) {
