@@ -47,6 +47,7 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
   __shared__ int32_t srow[DK_SPLIT];
   __shared__ float sl[DK_SPLIT];
   __shared__ float so[DK_THREADS / 16][DK_HD];
+  LAZY_PDL_ENTER();
   const int split = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
   const int n_splits = gridDim.x, H = gridDim.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -155,6 +156,7 @@ attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__rest
                            int ldo, float *__restrict__ stats) {
   __shared__ float sw[DK_MAX_SPLITS];  // weight of each split: 2^(m_i - m), 0 for an empty one
   __shared__ float red[DK_THREADS / 32];
+  LAZY_PDL_ENTER();
   const int h = blockIdx.x, r = blockIdx.y, H = gridDim.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const size_t base = ((size_t)r * H + h) * n_splits;
@@ -248,12 +250,13 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
   if (n_splits > DK_MAX_SPLITS) return LAZY_E_CAPACITY;
   float *part_o = part;
   float *part_ml = part + (size_t)n_rows * n_heads * n_splits * DK_HD;
-  attn_decode_partial_kernel<<<dim3(n_splits, n_heads, n_rows), DK_THREADS, 0, st>>>(
-      (const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v, ldkv, cu_x, cu_ctx, ctx_rows, q_kvlen,
-      score_row, n_seqs, n_ctx_total, part_o, part_ml, logits);
+  LAZY_TRY(launch_pdl(attn_decode_partial_kernel, dim3(n_splits, n_heads, n_rows), dim3(DK_THREADS), 0, st,
+                      (const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v, ldkv, cu_x, cu_ctx, ctx_rows, q_kvlen,
+                      score_row, n_seqs, n_ctx_total, part_o, part_ml, logits));
   LAZY_COUNT_LAUNCH();
-  attn_decode_combine_kernel<<<dim3(n_heads, n_rows), DK_THREADS, 0, st>>>(
-      part_o, part_ml, n_splits, cu_x, score_row, n_seqs, (bf16 *)o, ldo, stats);
+  LAZY_TRY(launch_pdl(attn_decode_combine_kernel, dim3(n_heads, n_rows), dim3(DK_THREADS), 0, st,
+                      (const float *)part_o, (const float *)part_ml, n_splits, cu_x, score_row, n_seqs, (bf16 *)o,
+                      ldo, stats));
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

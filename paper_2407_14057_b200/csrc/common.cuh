@@ -141,6 +141,32 @@ extern long long g_launches;
     if (rc__ != LAZY_OK) return rc__; \
   } while (0)
 
+// Programmatic dependent launch, used along the chain of small kernels of a decode step: the grid may be
+// set up while the kernel before it in the stream drains.  Such a kernel starts with LAZY_PDL_ENTER(): it
+// releases its own dependent right away and then waits for the grid before it to complete and flush (which,
+// that grid having waited in its turn, covers everything earlier in the stream).  Launched the ordinary
+// way the two instructions do nothing.
+#define LAZY_PDL_ENTER()                                                  \
+  do {                                                                    \
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");       \
+    asm volatile("griddepcontrol.wait;" ::: "memory");                    \
+  } while (0)
+
+template <typename... KArgs, typename... Args>
+inline int launch_pdl(void (*kfn)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kfn, static_cast<KArgs>(args)...) == cudaSuccess ? LAZY_OK : LAZY_E_CUDA;
+}
+
 inline int launch_ok() { return cudaPeekAtLastError() == cudaSuccess ? LAZY_OK : LAZY_E_CUDA; }
 
 // ---- launchers (one per step of the path); all enqueue on `st` and return a lazy_status ----

@@ -64,8 +64,8 @@ __global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, c
                                    const int32_t *xmap, int n_seqs, int m, int n, int32_t *kv_row_new,
                                    int32_t *kv_map, int32_t *q_kvlen, int32_t *ctx_rows, DevStatus *status) {
   // the projection that follows is a programmatic dependent: it may start fetching weights now and
-  // still waits for this grid before it reads the rows computed here
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // still waits for this grid before it reads the rows computed here; this grid is one too
+  LAZY_PDL_ENTER();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     const int s = seq_of(cu_ctx, n_seqs, i);
@@ -338,9 +338,11 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
 
     {  // bookkeeping first: the projection below may already write the rows' K/V into their cache rows
       const int n_thr = M > n_ctx ? M : n_ctx;
-      dec_prepare_kernel<<<cdiv(n_thr, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_CU_CTX), dtab(T_BASE),
-                                                           d_append + (size_t)l * W, xpos, ctx_pos, xmap, S, M, n_ctx,
-                                                           kv_row_new, kvm, q_kvlen, ctx_rows, status);
+      LAZY_TRY(launch_pdl(dec_prepare_kernel, dim3(cdiv(n_thr, 256)), dim3(256), 0, st, (const int32_t *)dtab(T_CU_X),
+                          (const int32_t *)dtab(T_CU_CTX), (const int32_t *)dtab(T_BASE),
+                          (const int32_t *)(d_append + (size_t)l * W), (const int32_t *)xpos,
+                          (const int32_t *)ctx_pos, (const int32_t *)xmap, S, M, n_ctx, kv_row_new, kvm, q_kvlen,
+                          ctx_rows, status));
       KLAUNCH_OK();
     }
     if (gemv_small_m_eligible(dt, M, d) && c->dh == 128) {

@@ -99,9 +99,9 @@ __global__ void score_stats_kernel(const float *__restrict__ logits, const int32
 __global__ void score_mean_kernel(const float *__restrict__ logits, const float *__restrict__ stats,
                                   const int32_t *__restrict__ cu_q, int n_seqs, int n_total,
                                   int n_heads, float *__restrict__ scores) {
-  // lets a following kernel launched as a programmatic dependent (decode: the output projection's weight
-  // streaming) start its weight reads now; it still waits for this grid before touching activations
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // releases a following programmatic dependent (decode: the output projection's weight streaming can start
+  // its weight reads now) and, launched as one itself, waits for the kernel before it
+  LAZY_PDL_ENTER();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int r = t >> 3, sub = t & 7;
   float acc = 0.f;
@@ -344,8 +344,8 @@ int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, 
                       int n_seqs, int n_total, int n_heads, float *scores) {
   if (n_total == 0) return LAZY_OK;
   if (!logits || !stats || !cu_q || !scores) return LAZY_E_BADARG;
-  score_mean_kernel<<<cdiv(n_total, 32), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
-                                                        scores);
+  LAZY_TRY(launch_pdl(score_mean_kernel, dim3(cdiv(n_total, 32)), dim3(256), 0, st, logits, stats, cu_q, n_seqs,
+                      n_total, n_heads, scores));
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
