@@ -146,30 +146,38 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
   }
 }
 
-// grid (H, M): merges the splits of one (row, head).  Thread t finishes output column t.  For a score
-// row the final (max, 1/sum) pair goes to stats[(seq*H + h)*2], max in natural-log units.
+// grid (H, M): merges the splits of one (row, head).  512 threads: thread (g, t) adds the splits i = g mod 4
+// of output column t (four chains of loads in flight per column: with 32 CTAs on the whole GPU the kernel is
+// a latency chain), then the four groups are summed through shared memory.  For a score row the final
+// (max, 1/sum) pair goes to stats[(seq*H + h)*2], max in natural-log units.
 constexpr int DK_MAX_SPLITS = 2048;  // 131072 keys
-__global__ void __launch_bounds__(DK_THREADS)
+constexpr int DK_CGROUPS = 4;
+constexpr int DK_CTHREADS = DK_CGROUPS * DK_HD;
+__global__ void __launch_bounds__(DK_CTHREADS)
 attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__restrict__ part_ml,
                            int n_splits, const int32_t *__restrict__ cu_x,
                            const int32_t *__restrict__ score_row, int n_seqs, bf16 *__restrict__ o,
                            int ldo, float *__restrict__ stats) {
   __shared__ float sw[DK_MAX_SPLITS];  // weight of each split: 2^(m_i - m), 0 for an empty one
-  __shared__ float red[DK_THREADS / 32];
+  __shared__ float red[DK_CTHREADS / 32];
+  __shared__ float sacc[DK_CGROUPS][DK_HD];
   LAZY_PDL_ENTER();
   const int h = blockIdx.x, r = blockIdx.y, H = gridDim.x;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = threadIdx.x / DK_HD, t = threadIdx.x - g * DK_HD;
   const size_t base = ((size_t)r * H + h) * n_splits;
   const float2 *ml = reinterpret_cast<const float2 *>(part_ml) + base;
   float m = -INFINITY;
-  for (int i = threadIdx.x; i < n_splits; i += DK_THREADS) m = fmaxf(m, ml[i].x);
+  for (int i = threadIdx.x; i < n_splits; i += DK_CTHREADS) m = fmaxf(m, ml[i].x);
   m = warp_max(m);
   if (lane == 0) red[warp] = m;
   __syncthreads();
-  m = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  m = red[0];
+#pragma unroll
+  for (int w = 1; w < DK_CTHREADS / 32; ++w) m = fmaxf(m, red[w]);
   __syncthreads();
   float l = 0.f;
-  for (int i = threadIdx.x; i < n_splits; i += DK_THREADS) {
+  for (int i = threadIdx.x; i < n_splits; i += DK_CTHREADS) {
     const float2 v = ml[i];
     const float w = v.y > 0.f ? ex2f_fast(v.x - m) : 0.f;
     sw[i] = w;
@@ -178,32 +186,35 @@ attn_decode_combine_kernel(const float *__restrict__ part_o, const float *__rest
   l = warp_sum(l);
   if (lane == 0) red[warp] = l;
   __syncthreads();
-  l = (red[0] + red[1]) + (red[2] + red[3]);
-  const float *po = part_o + base * DK_HD + threadIdx.x;
-  float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
-  int i = 0;
-  for (; i + 4 <= n_splits; i += 4) {  // an empty split never wrote its slot: do not touch it
-    const float w0 = sw[i], w1 = sw[i + 1], w2 = sw[i + 2], w3 = sw[i + 3];
+  l = 0.f;
+#pragma unroll
+  for (int w = 0; w < DK_CTHREADS / 32; ++w) l += red[w];  // fixed order: the same in every thread
+  const float *po = part_o + base * DK_HD + t;
+  float acc0 = 0.f, acc1 = 0.f;
+  int i = g;
+  for (; i + DK_CGROUPS < n_splits; i += 2 * DK_CGROUPS) {  // an empty split never wrote its slot: do not touch it
+    const float w0 = sw[i], w1 = sw[i + DK_CGROUPS];
     const float v0 = w0 > 0.f ? po[(size_t)i * DK_HD] : 0.f;
-    const float v1 = w1 > 0.f ? po[(size_t)(i + 1) * DK_HD] : 0.f;
-    const float v2 = w2 > 0.f ? po[(size_t)(i + 2) * DK_HD] : 0.f;
-    const float v3 = w3 > 0.f ? po[(size_t)(i + 3) * DK_HD] : 0.f;
+    const float v1 = w1 > 0.f ? po[(size_t)(i + DK_CGROUPS) * DK_HD] : 0.f;
     acc0 = fmaf(v0, w0, acc0);
     acc1 = fmaf(v1, w1, acc1);
-    acc2 = fmaf(v2, w2, acc2);
-    acc3 = fmaf(v3, w3, acc3);
   }
-  for (; i < n_splits; ++i) {
+  if (i < n_splits) {
     const float w = sw[i];
     if (w > 0.f) acc0 = fmaf(po[(size_t)i * DK_HD], w, acc0);
   }
-  const float inv = l > 0.f ? 1.f / l : 0.f;
-  o[(size_t)r * ldo + h * DK_HD + threadIdx.x] = __float2bfloat16(((acc0 + acc1) + (acc2 + acc3)) * inv);
-  if (threadIdx.x == 0) {
-    const int s = seq_of_row(cu_x, n_seqs, r);
-    if (score_row[s] == r) {
-      stats[((size_t)s * H + h) * 2] = m * LN2;
-      stats[((size_t)s * H + h) * 2 + 1] = inv;
+  sacc[g][t] = acc0 + acc1;
+  __syncthreads();
+  if (g == 0) {
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    const float acc = (sacc[0][t] + sacc[1][t]) + (sacc[2][t] + sacc[3][t]);
+    o[(size_t)r * ldo + h * DK_HD + t] = __float2bfloat16(acc * inv);
+    if (t == 0) {
+      const int s = seq_of_row(cu_x, n_seqs, r);
+      if (score_row[s] == r) {
+        stats[((size_t)s * H + h) * 2] = m * LN2;
+        stats[((size_t)s * H + h) * 2 + 1] = inv;
+      }
     }
   }
 }
@@ -216,7 +227,7 @@ int launch_attention_combine(cudaStream_t st, const float *part_o, const float *
                              void *o, int ldo, float *stats) {
   if (n_rows == 0) return LAZY_OK;
   if (n_splits < 1 || n_splits > DK_MAX_SPLITS) return LAZY_E_CAPACITY;
-  attn_decode_combine_kernel<<<dim3(n_heads, n_rows), DK_THREADS, 0, st>>>(part_o, part_ml, n_splits, cu_x, score_row,
+  attn_decode_combine_kernel<<<dim3(n_heads, n_rows), DK_CTHREADS, 0, st>>>(part_o, part_ml, n_splits, cu_x, score_row,
                                                                         n_seqs, (bf16 *)o, ldo, stats);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
@@ -254,7 +265,7 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
                       (const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v, ldkv, cu_x, cu_ctx, ctx_rows, q_kvlen,
                       score_row, n_seqs, n_ctx_total, part_o, part_ml, logits));
   LAZY_COUNT_LAUNCH();
-  LAZY_TRY(launch_pdl(attn_decode_combine_kernel, dim3(n_heads, n_rows), dim3(DK_THREADS), 0, st,
+  LAZY_TRY(launch_pdl(attn_decode_combine_kernel, dim3(n_heads, n_rows), dim3(DK_CTHREADS), 0, st,
                       (const float *)part_o, (const float *)part_ml, n_splits, cu_x, score_row, n_seqs, (bf16 *)o,
                       ldo, stats));
   LAZY_COUNT_LAUNCH();
