@@ -112,9 +112,7 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
  * Writes fp32 next-token logits [n_seqs, vocab] to d_logits (device) and leaves per-layer KV
  * caches and Aux Caches in the workspace for decode.  Resets any earlier generation state.
  * Row counts follow from (lengths, schedule) alone, so nothing is read back: the call only
- * enqueues work.  All of it is ordered after what `stream` held before the call and before what
- * is enqueued on `stream` afterwards; a small per-layer kernel (the head mean of Eq. 1) runs on a
- * stream the context creates on its first run, forked from and joined back to `stream` by events. */
+ * enqueues work on `stream`. */
 int lazy_prefill_run(lazy_ctx *ctx, void *stream, const int32_t *d_prompt_ids,
                      const int32_t *h_cu_seqlens, int32_t n_seqs, float *d_logits);
 

@@ -214,9 +214,6 @@ using namespace lazy;
 
 lazy_ctx::~lazy_ctx() {
   for (cudaEvent_t e : ev_pool) cudaEventDestroy(e);
-  if (ev_attn) cudaEventDestroy(ev_attn);
-  if (ev_score) cudaEventDestroy(ev_score);
-  if (side_stream) cudaStreamDestroy(side_stream);
 }
 int lazy_ctx::time_begin(cudaStream_t st, int kind, double flops, double bytes) {
   if (!timing_on || !((timing_mask >> kind) & 1u)) return -1;
@@ -453,32 +450,6 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   TIMED(LAZY_K_EMBED, 0, 2.0 * N * rb, launch_embed(st, dt, c->tok_embed, d_prompt_ids, c->x, N, d, c->V, status));
   LAZY_TRY(launch_iota_pos(st, c->pos_seg[0], d_cu(0), n_seqs, N));
 
-  // side stream and its two events, created on the first run (a failure just keeps everything in line)
-  if (!c->side_stream) {
-    cudaStream_t ss = nullptr;
-    cudaEvent_t e0 = nullptr, e1 = nullptr;
-    if (cudaStreamCreateWithFlags(&ss, cudaStreamNonBlocking) == cudaSuccess &&
-        cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) == cudaSuccess &&
-        cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) == cudaSuccess) {
-      c->side_stream = ss;
-      c->ev_attn = e0;
-      c->ev_score = e1;
-    } else {
-      cudaGetLastError();
-      if (e0) cudaEventDestroy(e0);
-      if (e1) cudaEventDestroy(e1);
-      if (ss) cudaStreamDestroy(ss);
-    }
-  }
-  bool score_pending = false;
-  auto join_score = [&]() -> int {  // the caller's stream waits for the head-mean kernel on the side stream
-    if (score_pending) {
-      LAZY_CUDA_OK(cudaStreamWaitEvent(st, c->ev_score, 0));
-      score_pending = false;
-    }
-    return LAZY_OK;
-  };
-
   char *x = c->x, *x2 = c->x2;
   int g = 0;
   for (int l = 0; l < L; ++l) {
@@ -518,7 +489,6 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     }
     bool fused_score = false;
     if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
-      LAZY_TRY(join_score());  // the previous layer's head-mean still reads the scratch these launches rewrite
       // one launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
       // read as zeros instead of whatever the cache region holds
       for (int s = 0; s < n_seqs; ++s) {
@@ -529,20 +499,9 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
                                   nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status, c->score_scratch,
                                   cdiv(seg_max, 64), n_seqs, s));
       }
-      // Eq. 1 from the last row's softmax numerators the attention kernel left behind.  Nothing needs the
-      // scores before the cut (or the next layer's attention, which reuses the scratch), so the small
-      // head-mean kernel runs on a side stream beside the output projection; the timing pass keeps it in line.
-      if (c->side_stream && !c->timing_on) {
-        LAZY_CUDA_OK(cudaEventRecord(c->ev_attn, st));
-        LAZY_CUDA_OK(cudaStreamWaitEvent(c->side_stream, c->ev_attn, 0));
-        LAZY_TRY(launch_score_from_attention(c->side_stream, c->score_scratch, d_cu(g), n_seqs, n, c->H,
-                                             cdiv(seg_max, 64), sc));
-        LAZY_CUDA_OK(cudaEventRecord(c->ev_score, c->side_stream));
-        score_pending = true;
-      } else {
-        TIMED(LAZY_K_SCORE, 0, 4.0 * c->H * n + 4.0 * n,
-              launch_score_from_attention(st, c->score_scratch, d_cu(g), n_seqs, n, c->H, cdiv(seg_max, 64), sc));
-      }
+      // Eq. 1 from the last row's softmax numerators the attention kernel left behind
+      TIMED(LAZY_K_SCORE, 0, 4.0 * c->H * n + 4.0 * n,
+            launch_score_from_attention(st, c->score_scratch, d_cu(g), n_seqs, n, c->H, cdiv(seg_max, 64), sc));
       fused_score = true;
     } else {
       TIMED(LAZY_K_ATTENTION, attn_flops, 0,
@@ -574,7 +533,6 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     const bool cut_after = p >= 0 && c->aux_after_layer;
     if (cut_after) LAZY_TRY(run_mlp());
     if (p >= 0) {
-      LAZY_TRY(join_score());
       const float *sel = sc;
       bool any_forced = false;
       for (int s = 0; s < n_seqs; ++s)
@@ -613,7 +571,6 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       LAZY_CUDA_OK(cudaMemcpyAsync(c->capture + (size_t)l * c->cap_rows * rb, x, (size_t)n2 * rb,
                                    cudaMemcpyDeviceToDevice, st));
   }
-  LAZY_TRY(join_score());
   // ---- first-token logits from the last row of every sequence
   TIMED(LAZY_K_RMSNORM, 0, 2.0 * n_seqs * rb,
         launch_rmsnorm_rows(st, dt, x, d_last, c->g_final, c->h_last, n_seqs, d, c->cfg.rms_eps));

@@ -52,9 +52,6 @@ struct lazy_ctx {
   int32_t *dec_i32;  // integer scratch of the decode step
   float *dec_f32;
   bool aux_after_layer = false;  // cut after the whole scoring layer (Aux rows = layer output) instead of before its MLP
-  // side stream for the head-mean of the Eq. 1 by-product: it runs beside the output projection
-  cudaStream_t side_stream = nullptr;
-  cudaEvent_t ev_attn = nullptr, ev_score = nullptr;
   void *gemm_scratch;  // split-wave partials and counters of the tensor-core GEMMs (bf16 only)
   size_t gemm_scratch_bytes;
 
