@@ -96,13 +96,15 @@ typedef struct {
 
 /* ---- context ------------------------------------------------------------------------- */
 
-/* Bytes of device workspace a context of this shape and schedule needs (0 on bad args). */
+/* Bytes of device workspace a context of this shape and schedule needs (0 on bad args).
+ * Plumbing: no counterpart in the paper. */
 size_t lazy_prefill_workspace_bytes(const lazy_model_cfg *cfg, const lazy_schedule *sched);
 
 /* Validates cfg and schedule, records the weight pointers and carves `d_workspace`
  * (256-byte aligned, at least lazy_prefill_workspace_bytes).  Enqueues a few small set-up
  * kernels (RoPE table) on the default stream and synchronises before returning.  On success
- * *out owns host memory only. */
+ * *out owns host memory only.  Plumbing: no counterpart in the paper (the schedule it records
+ * is Section 3.2's; the weights must stay unmodified while the context lives). */
 int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const lazy_schedule *sched,
                       void *d_workspace, size_t workspace_bytes, lazy_ctx **out);
 
@@ -129,9 +131,12 @@ int lazy_decode_step(lazy_ctx *ctx, void *stream, const int32_t *d_new_ids, floa
 /* Reads hidden states of pruned tokens from the Aux Cache that follows `layer` (Section 3.2,
  * Aux Cache: hidden states of tokens whose KV is absent from the next layer's cache).
  * d_positions: device int32[n] original token positions of sequence `seq`; d_hidden_out:
- * device [n, d_model] in the context's dtype.  The entries stay in the cache.  Synchronises
- * the stream; a position not held there gives LAZY_E_NOT_IN_AUX (rows of found positions are
- * still written). */
+ * device [n, d_model] in the context's dtype.  This is a NON-CONSUMING read for inspection and
+ * for callers that drive their own decode loop: the entries stay in the cache.  lazy_decode_step
+ * does not go through this call; it revives inside its own kernels (same look-up, same rows) and
+ * there an entry leaves the Aux Cache the moment its token gets K/V in the next layer.
+ * Synchronises the stream; a position not held there gives LAZY_E_NOT_IN_AUX (rows of found
+ * positions are still written). */
 int aux_cache_revive(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq,
                      const int32_t *d_positions, int32_t n, void *d_hidden_out);
 
@@ -148,7 +153,7 @@ int lazy_get_kept(lazy_ctx *ctx, void *stream, int32_t layer_entered, int32_t se
  * token attended at that layer, itself last). */
 int lazy_get_scores(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, float *d_scores,
                     int32_t *h_count);
-/* Test hook: the NEXT prefill (decode step) takes this kept set (positions, ascending, device
+/* Test hook (no counterpart in the paper): the NEXT prefill (decode step) takes this kept set (positions, ascending, device
  * int32[n]; the last token is kept regardless) at the schedule point instead of selecting by
  * score.  n = 0 clears the hook for that point.  The array must stay valid until that call
  * has run. */
@@ -175,6 +180,11 @@ int lazy_get_aux(lazy_ctx *ctx, void *stream, int32_t layer, int32_t seq, int32_
 int lazy_get_revived(lazy_ctx *ctx, void *stream, int32_t layer_entered, int32_t seq, int32_t *d_pos,
                      int32_t *h_count);
 int lazy_get_stats(lazy_ctx *ctx, lazy_stats *out);
+/* Rows kept at a schedule point (Section 3.2, top-percentile selection as a count): ceil(keep_bp / 10000 *
+ * n_total) in integer arithmetic, clamped to [1, n_present]; n_total = tokens of the sequence the
+ * percentage refers to, n_present = rows still present before the cut.  The same function sizes every
+ * buffer inside the library; 0 on bad arguments. */
+int32_t lazy_keep_count(int32_t n_total, uint32_t keep_bp, int32_t n_present);
 /* Per-step device times.  With timing on, every kernel launch of lazy_prefill_run is bracketed by
  * CUDA events on the caller's stream; lazy_get_kernel_times synchronises the stream and returns,
  * per kind of step, the summed event time of the latest run together with the ALGORITHMIC work of
@@ -195,6 +205,12 @@ typedef struct {
 } lazy_kernel_times;
 int lazy_set_kernel_timing(lazy_ctx *ctx, int32_t on);
 int lazy_get_kernel_times(lazy_ctx *ctx, void *stream, lazy_kernel_times *out);
+/* The same measurements launch by launch, in launch order: kind, device time and algorithmic work of
+ * every timed launch of the latest run (host arrays with room for `cap` entries; *count receives the
+ * number of timed launches, which may exceed cap).  Lets a caller see how a kind's rate depends on the
+ * number of surviving rows (the row count follows from the work: flops / flops per row). */
+int lazy_get_kernel_events(lazy_ctx *ctx, void *stream, int32_t cap, int32_t *kinds, float *ms, double *flops,
+                           double *bytes, int32_t *count);
 /* Where the scoring layer is cut (Section 3.2, Aux Cache paragraph).  after_layer = 0 (default): between
  * the layer's attention half and its MLP, so that MLP already runs on the kept rows, the Aux Cache holds
  * post-attention hidden states and a revived token first gets that layer's MLP.  after_layer = 1: after
@@ -204,10 +220,25 @@ int lazy_get_kernel_times(lazy_ctx *ctx, void *stream, lazy_kernel_times *out);
  * setting invalidates the caches of an earlier prefill (decode then returns LAZY_E_STATE). */
 int lazy_set_aux_point(lazy_ctx *ctx, int32_t after_layer);
 /* Synchronises `stream` and returns the first device-side error recorded since the last call
- * of this function (LAZY_OK if none), clearing it. */
+ * of this function (LAZY_OK if none), clearing it.  Plumbing: no counterpart in the paper.  After a
+ * LAZY_E_TIMEOUT the context stays usable: the next lazy_prefill_run / lazy_decode_step starts by
+ * clearing the arrival counters an aborted GEMM may have left behind. */
 int lazy_sync_status(lazy_ctx *ctx, void *stream);
 /* Same, for the context-free calls below. */
 int lazy_device_status(void *stream);
+/* Where the latest non-OK device status taken by this process came from: *where = code of the wait or
+ * check that failed (1..4 GEMM roles, 5 gather index, 6 Aux look-up, 7 token id, 8 selection, 9 decode
+ * planning, 10 RoPE position, 11..13 attention roles, 14 split-wave counter wait, 15 wait self-test),
+ * *a / *b two integers of context (CTA and parity for a wait, row and value for a check).  Any pointer
+ * may be NULL.  Plumbing: no counterpart in the paper. */
+int lazy_status_detail(int32_t *where, int32_t *a, int32_t *b);
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  Enqueues a one-warp kernel
+ * that waits, for at most limit_us microseconds (1..100000), on something that is never signalled:
+ * which = 0 an mbarrier phase (the wait every tensor-core role uses), which = 1 the arrival counter of
+ * the split last GEMM wave.  No copy, MMA or tensor-memory allocation is in flight, so the wait simply
+ * runs out: the kernel records LAZY_E_TIMEOUT in the status word and returns, and the device stays
+ * usable.  The status surfaces through lazy_device_status(). */
+int lazy_k_wait_selftest(void *stream, int32_t which, uint32_t limit_us);
 void lazy_destroy(lazy_ctx *ctx);
 const char *lazy_strerror(int status);
 
@@ -240,7 +271,8 @@ int lazy_prune_op(void *stream, int32_t dtype, int32_t n, int32_t d_model, int32
 /* y[r,:] = x[r,:] * rsqrt(mean(x[r,:]^2) + eps) * g  (Llama-2 pre-norm). x, y [n, d]. */
 int lazy_k_rmsnorm(void *stream, int32_t dtype, const void *x, const void *g, void *y, int32_t n,
                    int32_t d, float eps);
-/* C[M,N] = A[M,K] * B[N,K]^T (+ R[M,N] if R != NULL). bf16: tcgen05 tensor cores, TMA-fed;
+/* C[M,N] = A[M,K] * B[N,K]^T (+ R[M,N] if R != NULL): the dense products of the layers of
+ * Section 3.1 / 3.2. bf16: tcgen05 tensor cores, TMA-fed;
  * fp32: CUDA cores. lda = K, ldc = N (dense).  K and N multiples of 8.  impl: 0 = the
  * dtype's production kernel (bf16: weight streaming for M <= 4; tensor cores above, with one CTA
  * per 128x256 tile or a CTA pair per 256x256 tile, whichever measured faster for the shape),
@@ -253,7 +285,8 @@ int lazy_k_gemm(void *stream, int32_t dtype, int32_t impl, const void *A, const 
  * arrival counters).  The scratch must be zero before its first use, is left zero by every call,
  * and must not be shared by calls running at the same time.  Results do not depend on it being
  * given (the parts of a tile are added in a fixed order).  The paper has no counterpart: this is
- * scheduling of the dense products of Section 3.2's layers.  NULL scratch = lazy_k_gemm. */
+ * scheduling of the dense products of Section 3.2's layers.  NULL scratch = lazy_k_gemm.  If a call
+ * ended in LAZY_E_TIMEOUT, zero the first 2048 bytes of the scratch before using it again. */
 size_t lazy_k_gemm_scratch_bytes(void);
 int lazy_k_gemm_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *B,
                    const void *R, void *C, int32_t M, int32_t N, int32_t K, void *d_scratch,
@@ -290,7 +323,9 @@ int lazy_k_score(void *stream, int32_t dtype, const void *q, int32_t ldq, const 
  * GPU loading it holds until exit (about 1.04 MB).  Limits: n_heads * n_total <= 262144 and
  * 2 * n_heads * n_seqs <= 4096; anything larger returns LAZY_E_CAPACITY and runs nothing.  The
  * call allocates and frees nothing.  The first call on each device looks up the array's device
- * address (a synchronous runtime query), so make that first call outside any stream capture.
+ * address (a synchronous runtime query), so make that first call outside any stream capture; the
+ * address is remembered per device for the life of the process, so do not call this on a device
+ * after a cudaDeviceReset of it.
  * All calls share the one array, which simply keeps what the last call left there (nothing needs
  * clearing: every value read is written earlier by the same call); two calls whose kernels may
  * overlap on the GPU (different streams, different threads) race on it, so serialise them. */

@@ -86,6 +86,8 @@ _SIGNATURES = {
     "lazy_get_stats": (_I, [_P, C.POINTER(lazy_stats)]),
     "lazy_set_kernel_timing": (_I, [_P, _I]),
     "lazy_get_kernel_times": (_I, [_P, _P, C.POINTER(lazy_kernel_times)]),
+    "lazy_get_kernel_events": (_I, [_P, _P, _I, C.POINTER(_I), C.POINTER(C.c_float), C.POINTER(C.c_double),
+                                    C.POINTER(C.c_double), C.POINTER(_I)]),
     "lazy_sync_status": (_I, [_P, _P]),
     "lazy_device_status": (_I, [_P]),
     "lazy_destroy": (None, [_P]),
@@ -108,6 +110,9 @@ _SIGNATURES = {
     "lazy_k_select": (_I, [_P, _P, _P, _P, _I, _P, _P]),
     "lazy_k_select_threshold": (_I, [_P, _P, _P, _I, C.c_uint32, _P, _P, _P]),
     "lazy_k_gather_rows": (_I, [_P, _P, _P, _P, _I, _I, _I]),
+    "lazy_keep_count": (_I, [_I, _U, _I]),
+    "lazy_status_detail": (_I, [C.POINTER(_I), C.POINTER(_I), C.POINTER(_I)]),
+    "lazy_k_wait_selftest": (_I, [_P, _I, _U]),
 }
 
 _lib = None
@@ -312,6 +317,15 @@ class LazyPrefill:
         return {name: {"ms": t.ms[i], "launches": t.launches[i], "flops": t.flops[i], "bytes": t.bytes[i]}
                 for i, name in enumerate(KERNEL_KINDS)}
 
+    def lazy_get_kernel_events(self) -> List[Tuple[str, float, float, float]]:
+        """(kind, ms, flops, bytes) of every timed launch of the latest run, in launch order."""
+        cap = 4096
+        kinds, ms = (C.c_int32 * cap)(), (C.c_float * cap)()
+        fl, by, cnt = (C.c_double * cap)(), (C.c_double * cap)(), C.c_int32()
+        _check("lazy_get_kernel_events", lib().lazy_get_kernel_events(self.ctx, _stream(), cap, kinds, ms, fl, by,
+                                                                      C.byref(cnt)))
+        return [(KERNEL_KINDS[kinds[i]], ms[i], fl[i], by[i]) for i in range(min(cnt.value, cap))]
+
     def lazy_sync_status(self) -> None:
         _check("lazy_sync_status", lib().lazy_sync_status(self.ctx, _stream()))
 
@@ -319,6 +333,21 @@ class LazyPrefill:
 # ------------------------------------------------------------------------------- context-free calls
 def lazy_device_status() -> None:
     _check("lazy_device_status", lib().lazy_device_status(_stream()))
+
+
+def lazy_status_detail() -> Tuple[int, int, int]:
+    """(where, a, b) of the latest non-OK device status this process took."""
+    w, a, b = C.c_int32(), C.c_int32(), C.c_int32()
+    _check("lazy_status_detail", lib().lazy_status_detail(C.byref(w), C.byref(a), C.byref(b)))
+    return w.value, a.value, b.value
+
+
+def lazy_k_wait_selftest(which: int, limit_us: int) -> None:
+    _check("lazy_k_wait_selftest", lib().lazy_k_wait_selftest(_stream(), which, limit_us))
+
+
+def lazy_keep_count(n_total: int, keep_bp: int, n_present: int) -> int:
+    return int(lib().lazy_keep_count(n_total, keep_bp, n_present))
 
 
 def lazy_k_rmsnorm(x: torch.Tensor, g: torch.Tensor, eps: float) -> torch.Tensor:
@@ -452,7 +481,7 @@ def lazy_prune_op(x: torch.Tensor, pos: torch.Tensor, w_qkv: torch.Tensor, w_o: 
     if forced_keep_idx is not None:
         n_keep = forced_keep_idx.numel()
     else:
-        n_keep = max(1, min(n, (n * keep_bp + 9999) // 10000))
+        n_keep = lazy_keep_count(n, keep_bp, n)
     n_drop = n - n_keep
     nbytes = lib().lazy_prune_op_workspace_bytes(n, d, n_heads, head_dim, dt, max_pos)
     if workspace is None:

@@ -30,10 +30,8 @@ int lazy_k_gemm_ws(void *stream, int32_t dtype, int32_t impl, const void *A, con
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, B, nullptr, R, C, M, N, K, 0);
-  gemm_force_kernel(impl == 2 ? 1 : (impl == 3 ? 2 : 0));
-  const int rc = launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status, d_scratch, scratch_bytes);
-  gemm_force_kernel(0);
-  return rc;
+  return launch_gemm((cudaStream_t)stream, dtype, A, B, R, C, M, N, K, status, d_scratch, scratch_bytes,
+                     impl == 2 ? 1 : (impl == 3 ? 2 : 0));
 }
 
 int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
@@ -50,11 +48,8 @@ int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void 
   DevStatus *status = dev_status_ptr();
   if (!status) return LAZY_E_CUDA;
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  gemm_force_kernel(impl == 2 ? 1 : (impl == 3 ? 2 : 0));
-  const int rc = launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status, d_scratch,
-                                    scratch_bytes);
-  gemm_force_kernel(0);
-  return rc;
+  return launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status, d_scratch, scratch_bytes,
+                            impl == 2 ? 1 : (impl == 3 ? 2 : 0));
 }
 
 int lazy_k_rope_kv(void *stream, int32_t dtype, void *qkv, const int32_t *pos, float *rope_table,

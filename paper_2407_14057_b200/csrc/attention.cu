@@ -343,12 +343,7 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
 }  // namespace
 
 bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv) {
-  static int veto = -1;  // LAZY_ATTN=mma keeps the warp-level kernel (A/B timing, debugging)
-  if (veto < 0) {
-    const char *e = getenv("LAZY_ATTN");
-    veto = (e && e[0] == 'm') ? 1 : 0;
-  }
-  return !veto && dtype == LAZY_BF16 && head_dim == 128 && (ldq % 8) == 0 && (ldkv % 8) == 0;
+  return dtype == LAZY_BF16 && head_dim == 128 && (ldq % 8) == 0 && (ldkv % 8) == 0;
 }
 
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,

@@ -49,7 +49,11 @@ struct __align__(8) AttBarriers {
   unsigned long long s_full;   // S_j computed (phase j)
   unsigned long long s_free;   // S_j loaded into registers by all four softmax warps (phase j)
   unsigned long long p_full[2];
-  unsigned long long pv_done;
+  // P_j V_j retired; one barrier per P buffer (tile parity), phase index j >> 1.  A parity wait can
+  // only tell a phase from the one before it, so a waiter must never lag two phases: tile j+2 cannot
+  // retire on pv_done[j & 1] before P_{j+2} exists, and the softmax threads await P_j V_j before they
+  // write P_{j+2}, so every wait below is for the barrier's current or just-completed phase.
+  unsigned long long pv_done[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -120,7 +124,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     mbar_init(smem_u32(&bars->s_full), 1);
     mbar_init(smem_u32(&bars->s_free), 4);       // one arrival per softmax warp
     for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->p_full[b]), 4);
-    mbar_init(smem_u32(&bars->pv_done), 1);
+    for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars->pv_done[b]), 1);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     tma_prefetch_desc(&map_q);
@@ -221,7 +225,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           umma_bf16_a_tmem(tmem_o, tmem_p + (uint32_t)(k * 8), vd, idesc_pv, (j | k) != 0 ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars->v_empty[st]));  // V_j is free once these MMAs retire
-        umma_commit(smem_u32(&bars->pv_done));
+        umma_commit(smem_u32(&bars->pv_done[st]));
       }
     }
   } else {
@@ -281,7 +285,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         if (__any_sync(0xffffffffu, need)) {
           // O must be at rest: the previous P V has to retire before it is rescaled in place
-          ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+          ok = mbar_wait(smem_u32(&bars->pv_done[(j - 1) & 1]), (uint32_t)((j - 1) >> 1) & 1u, abort_flag, status,
+                         W_ATTN_SOFTMAX);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -331,10 +336,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       }
       // P_j goes where P_{j-2} was.  P_{j-2} V_{j-2} is issued by another thread than the S MMAs, so S_j's
-      // arrival says nothing about it; P_{j-1} V_{j-1} having retired does (same thread, issued in order), and
-      // that phase cannot be overtaken before P_j exists.
+      // arrival says nothing about it: its own barrier does (phase (j-2) >> 1 of pv_done[b]).
       if (j >= 2) {
-        ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(j - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+        ok = mbar_wait(smem_u32(&bars->pv_done[b]), (uint32_t)((j - 2) >> 1) & 1u, abort_flag, status,
+                       W_ATTN_SOFTMAX);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
       }
@@ -344,15 +349,15 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->p_full[b]));
     }
-    // A parity wait can only tell the current phase from the one before it.  After the last P
-    // is handed over, P V of the tile before may still be in flight, so the two remaining phases
-    // are awaited one after the other.
+    // The last two P V products (one per barrier) may still be in flight.
     if (ok && n_kt >= 2) {
-      ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 2) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = mbar_wait(smem_u32(&bars->pv_done[(n_kt - 2) & 1]), (uint32_t)((n_kt - 2) >> 1) & 1u, abort_flag, status,
+                     W_ATTN_SOFTMAX);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok) {
-      ok = mbar_wait(smem_u32(&bars->pv_done), (uint32_t)(n_kt - 1) & 1u, abort_flag, status, W_ATTN_SOFTMAX);
+      ok = mbar_wait(smem_u32(&bars->pv_done[(n_kt - 1) & 1]), (uint32_t)((n_kt - 1) >> 1) & 1u, abort_flag, status,
+                     W_ATTN_SOFTMAX);
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok && score_row) {

@@ -33,6 +33,7 @@ enum DevWhere {
   W_ATTN_MMA = 12,
   W_ATTN_SOFTMAX = 13,
   W_GEMM_TAIL = 14,
+  W_WAIT_SELFTEST = 15,
 };
 
 __device__ __forceinline__ void dev_fail(DevStatus *st, int code, int where, int a = 0, int b = 0) {
@@ -45,8 +46,10 @@ __device__ __forceinline__ void dev_fail(DevStatus *st, int code, int where, int
 
 // Address of this device's status word (a __device__ global of the library); NULL on failure.
 DevStatus *dev_status_ptr();
-// Synchronises the stream, returns and clears the status word.
+// Synchronises the stream, returns and clears the status word.  The detail fields of the latest
+// non-OK status taken by this process stay readable through last_status_detail().
 int sync_and_take_status(cudaStream_t stream, int *where_out);
+void last_status_detail(int *where, int *a, int *b);
 
 // ---- storage types --------------------------------------------------------------------------
 typedef __nv_bfloat16 bf16;
@@ -186,11 +189,16 @@ int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, co
 // scratch (gemm_scratch_bytes() bytes, zeroed once, private to the stream) lets the tensor-core kernels
 // split the last partial wave of tiles along K; without it they run a plain tile loop.
 size_t gemm_scratch_bytes();
+// force_kernel (cross-checks): 0 = chosen by shape, 1 = one CTA per tile, 2 = CTA pairs.
+// b_const: the caller guarantees that B (the weights) is not written by earlier work still in flight on
+// the stream; only then may the weight-streaming kernel (M <= 4) start fetching B while the kernel before
+// it drains.
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
-                int M, int N, int K, DevStatus *status, void *scratch = nullptr, size_t scratch_bytes = 0);
+                int M, int N, int K, DevStatus *status, void *scratch = nullptr, size_t scratch_bytes = 0,
+                int force_kernel = 0, bool b_const = false);
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
                        void *C, int M, int F, int K, DevStatus *status, void *scratch = nullptr,
-                       size_t scratch_bytes = 0);
+                       size_t scratch_bytes = 0, int force_kernel = 0, bool b_const = false);
 // QKV projection with the rotary embedding and the K/V cache write in its epilogue (bf16,
 // head_dim 128, d_model a multiple of 256): qkv [M, 3d] receives the rotated q (its k and v thirds
 // are left untouched), rotated k and v go to cache rows kv_row[r] (or r) with their position tag.
@@ -199,13 +207,14 @@ int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
                          void *scratch = nullptr, size_t scratch_bytes = 0);
-void gemm_force_kernel(int which);
 // Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
 // rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).
 bool gemv_small_m_eligible(int dtype, int M, int K);
+// b_const: B is not being written by earlier work on the stream, so the launch may be a programmatic
+// dependent whose first weight loads are issued before the preceding kernel has completed.
 int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
                         void *C, int M, int N, int K, int swiglu, const void *gain = nullptr,
-                        float eps = 0.f, int c_f32 = 0);
+                        float eps = 0.f, int c_f32 = 0, bool b_const = false);
 int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
                          const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
@@ -237,7 +246,7 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
 size_t attn_score_scratch_floats(int n_seqs, int n_heads, int max_tiles);
 int launch_score_from_attention(cudaStream_t st, const float *scratch, const int32_t *cu_q, int n_seqs,
                                 int n_total, int n_heads, int max_tiles, float *scores);
-// True when the tensor-core prefill attention applies (and LAZY_ATTN=mma does not veto it).
+// True when the tensor-core prefill attention applies.
 bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
@@ -282,7 +291,7 @@ int launch_gather_rows(cudaStream_t st, const void *src, const int32_t *idx, voi
                        int row_bytes, int src_rows, DevStatus *status);
 int launch_gather_i32(cudaStream_t st, const int32_t *src, const int32_t *idx, int32_t *dst, int n);
 int launch_lm_head(cudaStream_t st, int dtype, const void *h, const void *w, float *logits,
-                   int n_rows, int d, int vocab);
+                   int n_rows, int d, int vocab, bool w_const = false);
 int launch_argmax(cudaStream_t st, const float *logits, int32_t *out, int n_rows, int vocab);
 int launch_fill_i32(cudaStream_t st, int32_t *p, int32_t v, size_t n);
 int launch_iota_pos(cudaStream_t st, int32_t *pos, const int32_t *cu, int n_seqs, int n_total);

@@ -352,11 +352,11 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     } else {
       if (gemv_small_m_eligible(dt, M, d)) {
         LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, 3 * d, d, 0, c->g_attn[l],
-                                     c->cfg.rms_eps, 0));
+                                     c->cfg.rms_eps, 0, true));
       } else {
         LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
         LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status, c->gemm_scratch,
-                             c->gemm_scratch_bytes));
+                             c->gemm_scratch_bytes, 0, true));
       }
       LAZY_TRY(launch_rope_kv(st, dt, c->qkv, xpos, c->rope_table, kc, vc, kvp, kv_row_new, M, c->H, c->dh,
                               c->max_pos, status));
@@ -387,21 +387,22 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
       LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
                                n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
     }
-    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status, c->gemm_scratch, c->gemm_scratch_bytes));
+    LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status, c->gemm_scratch, c->gemm_scratch_bytes, 0,
+                         true));
 
     const int pt = c->point_at[l + 1];
     // The layer's MLP on the rows in flight (revived rows included, under the default cut point).
     auto run_mlp = [&]() -> int {
       if (gemv_small_m_eligible(dt, M, d)) {
         LAZY_TRY(launch_gemv_small_m(st, x, c->w_gate[l], c->w_up[l], nullptr, c->act, M, c->F, d, 1, c->g_mlp[l],
-                                     c->cfg.rms_eps, 0));
+                                     c->cfg.rms_eps, 0, true));
       } else {
         LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, M, d, c->cfg.rms_eps));
         LAZY_TRY(launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, M, c->F, d, status,
-                                    c->gemm_scratch, c->gemm_scratch_bytes));
+                                    c->gemm_scratch, c->gemm_scratch_bytes, 0, true));
       }
       LAZY_TRY(launch_gemm(st, dt, c->act, c->w_down[l], x, x, M, d, c->F, status, c->gemm_scratch,
-                           c->gemm_scratch_bytes));
+                           c->gemm_scratch_bytes, 0, true));
       return LAZY_OK;
     };
     // cut after the whole layer: the MLP runs before the re-selection, and rows revived from the Aux Cache
@@ -511,7 +512,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
   for (int s = 0; s < S; ++s) tab(T_LAST)[s] = tab(T_CU_X)[s + 1] - 1;
   LAZY_TRY(upload(T_LAST));
   LAZY_TRY(launch_rmsnorm_rows(st, dt, x, dtab(T_LAST), c->g_final, c->h_last, S, d, c->cfg.rms_eps));
-  LAZY_TRY(launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, S, d, c->V));
+  LAZY_TRY(launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, S, d, c->V, true));
   if (d_next_ids) LAZY_TRY(launch_argmax(st, d_logits, d_next_ids, S, c->V));
   xmap_kernel<<<cdiv(M, 256), 256, 0, st>>>(dtab(T_CU_X), dtab(T_BASE), xpos, S, M, xmap, 0);
   KLAUNCH_OK();

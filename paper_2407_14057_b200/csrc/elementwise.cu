@@ -33,6 +33,13 @@ DevStatus *dev_status_ptr() {
   return ptrs[dev];
 }
 
+static DevStatus g_last_bad_status = {0, 0, 0, 0};
+void last_status_detail(int *where, int *a, int *b) {
+  if (where) *where = g_last_bad_status.where;
+  if (a) *a = g_last_bad_status.a;
+  if (b) *b = g_last_bad_status.b;
+}
+
 int sync_and_take_status(cudaStream_t stream, int *where_out) {
   DevStatus *p = dev_status_ptr();
   if (!p) return LAZY_E_CUDA;
@@ -40,6 +47,7 @@ int sync_and_take_status(cudaStream_t stream, int *where_out) {
   DevStatus h;
   if (cudaMemcpy(&h, p, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return LAZY_E_CUDA;
   if (h.code != 0) {
+    g_last_bad_status = h;
     if (cudaMemset(p, 0, sizeof(DevStatus)) != cudaSuccess) return LAZY_E_CUDA;
   }
   if (where_out) *where_out = h.where;
@@ -345,13 +353,13 @@ __global__ void lm_head_kernel(const T *__restrict__ h, const T *__restrict__ w,
 }
 
 int launch_lm_head(cudaStream_t st, int dtype, const void *h, const void *w, float *logits,
-                   int n_rows, int d, int vocab) {
+                   int n_rows, int d, int vocab, bool w_const) {
   if (n_rows == 0) return LAZY_OK;
   if (gemv_small_m_eligible(dtype, 4, d)) {  // up to four rows per pass over the matrix
     for (int s0 = 0; s0 < n_rows; s0 += 4) {
       const int m = n_rows - s0 < 4 ? n_rows - s0 : 4;
       LAZY_TRY(launch_gemv_small_m(st, (const bf16 *)h + (size_t)s0 * d, w, nullptr, nullptr,
-                                   logits + (size_t)s0 * vocab, m, vocab, d, 0, nullptr, 0.f, 1));
+                                   logits + (size_t)s0 * vocab, m, vocab, d, 0, nullptr, 0.f, 1, w_const));
     }
     return LAZY_OK;
   }

@@ -185,7 +185,7 @@ __device__ __forceinline__ void gemm_fixup_row(uint32_t taddr, const float *slot
 
 // Warp-level, bounded wait until *flag >= target.  False (and the abort flag set) on expiry.
 __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned target, volatile int *abort_flag,
-                                               DevStatus *status) {
+                                               DevStatus *status, unsigned long long limit_ns = WAIT_LIMIT_NS) {
   int ok = 1;
   if ((threadIdx.x & 31) == 0) {
     const unsigned long long t0 = global_timer_ns();
@@ -196,7 +196,7 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
       if (v >= target) break;
       if ((++spins & 63u) == 0) {
         if (*abort_flag) { ok = 0; break; }
-        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (global_timer_ns() - t0 > limit_ns) {
           *abort_flag = 1;
           dev_fail(status, LAZY_E_TIMEOUT, W_GEMM_TAIL, (int)blockIdx.x, (int)v);
           ok = 0;

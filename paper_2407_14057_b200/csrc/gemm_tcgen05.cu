@@ -233,20 +233,17 @@ int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_row
 // how the row count pads to 128 / 256, how many waves that makes, what the split last wave recovers, and the
 // pair kernel's measured ~6 % shorter wave on the plain / residual / QKV epilogues (none on SwiGLU, whose
 // epilogue dominates the difference).  Measured against both kernels at 1013-23112 rows of the 7B widths the
-// estimate picks the faster one except within ~2 %.  LAZY_GEMM=single / pair overrides (A/B timing).
-int g_force_kernel = 0;  // 1: one CTA per tile, 2: CTA pairs (cross-check entry points)
-bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_bytes) {
-  static int mode = -1;  // 0 auto, 1 always single, 2 always pair
-  static int max_pairs = 0;
-  if (mode < 0) {
-    const char *e = getenv("LAZY_GEMM");
-    mode = !e ? 0 : (strcmp(e, "single") == 0 ? 1 : (strcmp(e, "pair") == 0 ? 2 : 0));
-    max_pairs = gemm_pair_max_clusters();
-    if (max_pairs > sm_count() / 2) max_pairs = sm_count() / 2;
+// estimate picks the faster one except within ~2 %.  force: 1 = one CTA per tile, 2 = CTA pairs (the
+// cross-check entry points), 0 = by the estimate.
+bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_bytes, int force) {
+  static int max_pairs = -1;
+  if (max_pairs < 0) {
+    int n = gemm_pair_max_clusters();
+    if (n > sm_count() / 2) n = sm_count() / 2;
+    max_pairs = n < 0 ? 0 : n;
   }
-  if (M <= BM || g_force_kernel == 1 || max_pairs < 1) return false;
-  if (g_force_kernel == 2) return true;
-  if (mode != 0) return mode == 2;
+  if (M <= BM || force == 1 || max_pairs < 1) return false;
+  if (force == 2) return true;
   const int tile_n = epi == EPI_SWIGLU ? BN / 2 : BN, extra = epi == EPI_SWIGLU ? 8 : 0, num_kb = cdiv(K, BK);
   double w_one = 0, w_pair = 0;
   plan_tail(cdiv(M, BM) * cdiv(N, tile_n), num_kb, sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K, extra,
@@ -260,12 +257,12 @@ bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_b
 template <int EPI>
 int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C,
               int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
-              size_t scratch_bytes) {
+              size_t scratch_bytes, int force_kernel) {
   // TMA needs 16-byte aligned bases and row pitches; the epilogue stores 8 columns at a time.
   if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
-  if (gemm_use_pair(EPI, M, N, K, scratch, scratch_bytes))
+  if (gemm_use_pair(EPI, M, N, K, scratch, scratch_bytes, force_kernel))
     return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
   CUtensorMap ma, mb0, mb1;
   LAZY_TRY(make_map(&ma, A, M, K, BM));
@@ -295,16 +292,18 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
 // more SMs than that the kernels fall back to the plain tile loop.
 size_t gemm_scratch_bytes() { return gemm_tail_scratch_bytes(GEMM_TAIL_MAX_CTAS); }
 
-// Cross-check switch of the context-free entry points: 0 = by shape, 1 = one CTA per tile, 2 = CTA pairs.
-void gemm_force_kernel(int which) { g_force_kernel = which; }
-
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
-                int M, int N, int K, DevStatus *status, void *scratch, size_t scratch_bytes) {
+                int M, int N, int K, DevStatus *status, void *scratch, size_t scratch_bytes, int force_kernel,
+                bool b_const) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, B, nullptr, R, C, M, N, K, 0);
-  if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, B, nullptr, R, C, M, N, K, 0);
-  if (R) return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes);
-  return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes);
+  if (gemv_small_m_eligible(dtype, M, K))
+    return launch_gemv_small_m(st, A, B, nullptr, R, C, M, N, K, 0, nullptr, 0.f, 0, b_const);
+  if (R)
+    return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes,
+                                   force_kernel);
+  return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes,
+                              force_kernel);
 }
 
 bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {
@@ -326,15 +325,18 @@ int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void
   r.d_model = d_model;
   r.max_pos = max_pos;
   return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, 3 * d_model, d_model, status, r, scratch,
-                                 scratch_bytes);
+                                 scratch_bytes, 0);
 }
 
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
-                       void *C, int M, int F, int K, DevStatus *status, void *scratch, size_t scratch_bytes) {
+                       void *C, int M, int F, int K, DevStatus *status, void *scratch, size_t scratch_bytes,
+                       int force_kernel, bool b_const) {
   if (M == 0) return LAZY_OK;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  if (gemv_small_m_eligible(dtype, M, K)) return launch_gemv_small_m(st, A, Bg, Bu, nullptr, C, M, F, K, 1);
-  return launch_tc<EPI_SWIGLU>(st, A, Bg, Bu, nullptr, C, M, F, K, status, RopeArgs(), scratch, scratch_bytes);
+  if (gemv_small_m_eligible(dtype, M, K))
+    return launch_gemv_small_m(st, A, Bg, Bu, nullptr, C, M, F, K, 1, nullptr, 0.f, 0, b_const);
+  return launch_tc<EPI_SWIGLU>(st, A, Bg, Bu, nullptr, C, M, F, K, status, RopeArgs(), scratch, scratch_bytes,
+                               force_kernel);
 }
 
 }  // namespace lazy

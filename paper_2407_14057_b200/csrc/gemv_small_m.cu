@@ -63,10 +63,11 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   __shared__ float gv_red[M_ROWS][GV_THREADS / 32];
   const int kvec = K >> 3;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // Weights do not depend on the kernel before this one: the first batch of this warp's first column is
-  // requested before waiting for that kernel (the launch allows this grid to start while it drains), and
-  // the kernel after this one is released to do the same.  Activations, gains and residuals are touched
-  // only after the wait.
+  // When launched as a programmatic dependent (the caller vouches that the weights are not being written
+  // by earlier work on the stream), this grid starts while the kernel before it drains: the first batch of
+  // this warp's first column is requested before waiting for that kernel, and the kernel after this one is
+  // released to do the same.  Activations, gains and residuals are touched only after the wait.  Launched
+  // the ordinary way the grid starts after that kernel has completed and the two instructions do nothing.
   constexpr int U = SWIGLU ? 4 : 8;  // weight vectors per lane in flight (x2 matrices for SwiGLU)
   const int n_first = blockIdx.x * (GV_THREADS / 32) + warp;
   uint4 wr[U], ur[SWIGLU ? U : 1];  // the batch in flight
@@ -214,14 +215,14 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
 
 template <int M_ROWS, int MODE>
 int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C, int N,
-               int K, const void *gain, float eps, int c_f32, const GemvRope &rope = GemvRope()) {
+               int K, const void *gain, float eps, int c_f32, bool pdl, const GemvRope &rope = GemvRope()) {
   const size_t smem = (size_t)M_ROWS * K * 2;
   auto kfn = gemv_small_m_kernel<M_ROWS, MODE>;
   LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   int blocks = cdiv(N, GV_THREADS / 32);
   const int cap = sm_count() * 4;
   if (blocks > cap) blocks = cap;
-  // programmatic dependent launch: this grid may start while the kernel before it in the stream drains
+  // programmatic dependent launch (pdl): this grid may start while the kernel before it in the stream drains
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(blocks, 1, 1);
   cfg.blockDim = dim3(GV_THREADS, 1, 1);
@@ -231,7 +232,7 @@ int launch_one(cudaStream_t st, const void *A, const void *B0, const void *B1, c
   attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl ? 1 : 0;
   LAZY_CUDA_OK(cudaLaunchKernelEx(&cfg, kfn, (const bf16 *)A, (const bf16 *)B0, (const bf16 *)B1, (const bf16 *)R, C,
                                   N, K, (const bf16 *)gain, eps, c_f32, rope));
   LAZY_COUNT_LAUNCH();
@@ -247,13 +248,14 @@ bool gemv_small_m_eligible(int dtype, int M, int K) {
 // gain != NULL: the rows of A are RMS-normalised (gain, eps) before the product, with the rounding a
 // separate normalisation kernel writing bf16 would have had.  c_f32: C holds fp32 instead of bf16.
 int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
-                        void *C, int M, int N, int K, int swiglu, const void *gain, float eps, int c_f32) {
+                        void *C, int M, int N, int K, int swiglu, const void *gain, float eps, int c_f32,
+                        bool b_const) {
   if (((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) || ((uintptr_t)gain & 15))
     return LAZY_E_BADARG;
 #define GV_CASE(m)                                                                            \
   case m:                                                                                     \
-    return swiglu ? launch_one<m, GV_SWIGLU>(st, A, B0, B1, nullptr, C, N, K, gain, eps, c_f32) \
-                  : launch_one<m, GV_PLAIN>(st, A, B0, nullptr, R, C, N, K, gain, eps, c_f32);
+    return swiglu ? launch_one<m, GV_SWIGLU>(st, A, B0, B1, nullptr, C, N, K, gain, eps, c_f32, b_const) \
+                  : launch_one<m, GV_PLAIN>(st, A, B0, nullptr, R, C, N, K, gain, eps, c_f32, b_const);
   switch (M) {
     GV_CASE(1)
     GV_CASE(2)
@@ -266,7 +268,8 @@ int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const vo
 
 // QKV projection of one to four rows (optionally RMS-normalised first) with the rotary embedding and the
 // K/V cache write in its epilogue: qkv [M, 3d] receives the rotated q (its k and v thirds are left
-// untouched), rotated k and v go to cache rows kv_row[m] with their position tag.  head_dim 128.
+// untouched), rotated k and v go to cache rows kv_row[m] with their position tag.  head_dim 128.  Only the
+// decode step calls this, with the context's own (constant) weights: always a programmatic dependent.
 int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
                          const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status) {
@@ -285,7 +288,7 @@ int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void
   r.status = status;
   const int tasks = 3 * d_model / 2;
 #define GV_CASE(m) \
-  case m: return launch_one<m, GV_QKV_ROPE>(st, x, w_qkv, nullptr, nullptr, qkv, tasks, d_model, gain, eps, 0, r);
+  case m: return launch_one<m, GV_QKV_ROPE>(st, x, w_qkv, nullptr, nullptr, qkv, tasks, d_model, gain, eps, 0, true, r);
   switch (M) {
     GV_CASE(1)
     GV_CASE(2)

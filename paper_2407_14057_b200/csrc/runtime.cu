@@ -3,6 +3,7 @@
 
 #include <new>
 
+#include "gemm_epilogue.cuh"
 #include "runtime.cuh"
 
 namespace lazy {
@@ -208,6 +209,14 @@ static void fill_shape(lazy_ctx *c, const lazy_model_cfg *cfg, const lazy_schedu
   c->max_pos = cfg->max_prompt_tokens + cfg->max_new_tokens;
 }
 
+// The split-wave GEMMs leave their arrival counters at zero, except when a bounded wait ran out in the
+// middle of a launch.  A run that follows such a failure must not inherit the stale counts, so every run
+// starts by clearing the 2 KiB counter block (one tiny memset in a 27 ms prefill / 3 ms decode step).
+static int reset_gemm_counters(lazy_ctx *c, cudaStream_t st) {
+  if (!c->gemm_scratch) return LAZY_OK;
+  return cudaMemsetAsync(c->gemm_scratch, 0, GEMM_TAIL_COUNTER_BYTES, st) == cudaSuccess ? LAZY_OK : LAZY_E_CUDA;
+}
+
 }  // namespace lazy
 
 using namespace lazy;
@@ -226,6 +235,8 @@ int lazy_ctx::time_begin(cudaStream_t st, int kind, double flops, double bytes) 
     ev_pool.push_back(e);
   }
   ev_kind.push_back(kind);
+  ev_flops.push_back(flops);
+  ev_bytes.push_back(bytes);
   cudaEventRecord(ev_pool[2 * slot], st);
   return slot;
 }
@@ -318,6 +329,11 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
   return LAZY_OK;
 }
 
+int32_t lazy_keep_count(int32_t n_total, uint32_t keep_bp, int32_t n_present) {
+  if (n_total < 1 || keep_bp < 1 || keep_bp > 10000 || n_present < 1) return 0;
+  return keep_count(n_total, keep_bp, n_present);
+}
+
 int lazy_set_aux_point(lazy_ctx *c, int32_t after_layer) {
   if (!c || (after_layer != 0 && after_layer != 1)) return LAZY_E_BADARG;
   if (c->aux_after_layer != (after_layer != 0)) {
@@ -381,7 +397,10 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   const long long launches0 = g_launches;
   const int P = c->P, L = c->L, d = c->d, dt = c->dtype;
   const size_t rb = c->row_bytes();
+  LAZY_TRY(reset_gemm_counters(c, st));
   c->ev_kind.clear();
+  c->ev_flops.clear();
+  c->ev_bytes.clear();
   for (int i = 0; i < LAZY_N_KERNEL_KINDS; ++i) c->k_flops[i] = c->k_bytes[i] = 0.0;
 
   // ---- host bookkeeping: every row count follows from the lengths and the schedule
@@ -575,7 +594,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   TIMED(LAZY_K_RMSNORM, 0, 2.0 * n_seqs * rb,
         launch_rmsnorm_rows(st, dt, x, d_last, c->g_final, c->h_last, n_seqs, d, c->cfg.rms_eps));
   TIMED(LAZY_K_LM_HEAD, 0, (double)c->V * rb,
-        launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, n_seqs, d, c->V));
+        launch_lm_head(st, dt, c->h_last, c->w_lm_head, d_logits, n_seqs, d, c->V, true));
   // the residual stream may live in either ping-pong buffer; decode does not need it
   c->forced.clear();
   c->have_prefill = true;
@@ -618,6 +637,7 @@ int lazy_decode_step(lazy_ctx *c, void *stream, const int32_t *d_new_ids, float 
                      int32_t *d_next_ids) {
   if (!c || !d_new_ids || !d_logits) return LAZY_E_BADARG;
   if (!c->have_prefill) return LAZY_E_STATE;
+  LAZY_TRY(reset_gemm_counters(c, (cudaStream_t)stream));
   return decode_step_impl(c, (cudaStream_t)stream, d_new_ids, d_logits, d_next_ids);
 }
 
@@ -794,6 +814,22 @@ int lazy_get_kernel_times(lazy_ctx *c, void *stream, lazy_kernel_times *out) {
   for (int k = 0; k < LAZY_N_KERNEL_KINDS; ++k) {
     out->flops[k] = c->k_flops[k];
     out->bytes[k] = c->k_bytes[k];
+  }
+  return LAZY_OK;
+}
+
+int lazy_get_kernel_events(lazy_ctx *c, void *stream, int32_t cap, int32_t *kinds, float *ms, double *flops,
+                           double *bytes, int32_t *count) {
+  if (!c || !count || cap < 0 || (cap > 0 && (!kinds || !ms || !flops || !bytes))) return LAZY_E_BADARG;
+  LAZY_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  *count = (int32_t)c->ev_kind.size();
+  for (size_t i = 0; i < c->ev_kind.size() && (int32_t)i < cap; ++i) {
+    float t = 0.f;
+    LAZY_CUDA_OK(cudaEventElapsedTime(&t, c->ev_pool[2 * i], c->ev_pool[2 * i + 1]));
+    kinds[i] = c->ev_kind[i];
+    ms[i] = t;
+    flops[i] = c->ev_flops[i];
+    bytes[i] = c->ev_bytes[i];
   }
   return LAZY_OK;
 }

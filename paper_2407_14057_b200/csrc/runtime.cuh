@@ -79,6 +79,7 @@ struct lazy_ctx {
   uint32_t timing_mask = 0xffffffffu;  // kinds that get an event pair
   std::vector<cudaEvent_t> ev_pool;  // pairs: 2*i start, 2*i+1 stop
   std::vector<int> ev_kind;          // kind of each used pair
+  std::vector<double> ev_flops, ev_bytes;  // algorithmic work of the launch each pair brackets
   double k_flops[LAZY_N_KERNEL_KINDS], k_bytes[LAZY_N_KERNEL_KINDS];
   // Returns the index of a fresh event pair (or -1) after recording its start.
   int time_begin(cudaStream_t st, int kind, double flops, double bytes);

@@ -11,6 +11,8 @@
 // radix select over the fp32 bit patterns (the last row is given the maximal key so it always
 // survives); a final pass in index order emits kept and dropped row indices with ballot / popcount
 // prefix sums, taking ties at the threshold in ascending index order until n_keep is reached.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace lazy {
@@ -418,16 +420,19 @@ static __device__ __align__(256) float g_static_score_scratch[STATIC_SCORE_MAX_L
 
 // Device address of the array on the current device.  The array's name is only a host-side handle
 // here: the address a kernel can use comes from cudaGetSymbolAddress, asked once per device.
+// The per-device slots are atomic, so two host threads making their first call at once both store
+// the same address without a data race.  The slots outlive a cudaDeviceReset of their device: a
+// process that resets a device must not call this entry point on it afterwards.
 float *static_score_scratch_ptr() {
-  static float *ptrs[64] = {nullptr};
+  static std::atomic<float *> ptrs[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!ptrs[dev]) {
-    float *p = nullptr;
+  float *p = ptrs[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress((void **)&p, g_static_score_scratch) != cudaSuccess) return nullptr;
-    ptrs[dev] = p;
+    ptrs[dev].store(p, std::memory_order_release);
   }
-  return ptrs[dev];
+  return p;
 }
 }  // namespace
 

@@ -55,3 +55,23 @@ def test_null_arguments_are_rejected_without_touching_the_device(lib):
     assert lib.aux_cache_revive(None, None, 0, 0, None, 0, None) == -1
     assert lib.lazy_k_gemm(None, 0, 0, None, None, None, None, 1, 8, 8) == -1
     assert lib.lazy_prune_op_workspace_bytes(0, 256, 4, 64, 1, 16) == 0
+
+
+def test_keep_count_of_the_library_matches_the_worked_values(lib):
+    """Host arithmetic only: the count the library sizes every buffer with, against the hand-worked
+    fixture (Section 3.2, top-percentile selection as a count)."""
+    with open(os.path.join(ROOT, "tests", "golden", "keep_counts.txt")) as f:
+        rows = [l for l in f if l.strip() and not l.startswith("#")]
+    for line in rows:
+        N, bp, want = [int(t) for t in line.split("|")]
+        assert lib.lazy_keep_count(N, bp, N) == want
+    assert lib.lazy_keep_count(100, 7000, 50) == 50          # clamped to the rows present
+    assert lib.lazy_keep_count(100, 1, 100) == 1             # never below one row
+    assert lib.lazy_keep_count(0, 5000, 1) == 0 and lib.lazy_keep_count(10, 0, 10) == 0   # bad arguments
+    assert lib.lazy_keep_count(10, 10001, 10) == 0
+
+
+def test_wait_selftest_rejects_bad_arguments_without_a_device(lib):
+    assert lib.lazy_k_wait_selftest(None, 2, 1000) == -1
+    assert lib.lazy_k_wait_selftest(None, 0, 0) == -1
+    assert lib.lazy_k_wait_selftest(None, 0, 200000) == -1     # limits above 0.1 s are refused

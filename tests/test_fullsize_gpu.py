@@ -25,6 +25,14 @@ from helpers import rel_err, to_np, weights_to_np
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
+# End-to-end gates of the 32-layer run against the fp64 forced replay.  Measured: the residual stream's
+# error grows like a random walk of one-layer roundings, 1.1e-2 after layer 0, 2.8e-2 after layer 7,
+# 3.7e-2 after layer 15, 4.9e-2 after layer 23, 5.4e-2 after layer 31 (about 1.0e-2 x sqrt(layers)); logits
+# 5.1e-2; Eq. 1 scores within 1.6e-3 absolute at every depth; the GPU's greedy token is the oracle's
+# second-ranked token (logits of a random-init model are nearly flat) and the two top-10 sets coincide.
+E2E_DRIFT_GATE = 0.08
+E2E_LOGITS_GATE = 0.08
+E2E_SCORE_ABS_GATE = 3e-3
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -41,28 +49,47 @@ def model7b():
     torch.cuda.empty_cache()
 
 
-def _layer_inputs(eng, shape, emb, l, schedule, n):
+def _rows_entering(lengths, schedule, l):
+    """Rows of every sequence that enter layer l (counts follow from lengths and schedule alone)."""
+    rows = list(lengths)
+    for e, bp in schedule:
+        if e <= l:
+            rows = [O.keep_count(n, bp, r) for n, r in zip(lengths, rows)]
+    return rows
+
+
+def _member_rows(packed, lengths, schedule, l_entering, seq):
+    """Rows of sequence `seq` inside a packed [sum rows, d] tensor of the segment entering layer l_entering."""
+    rows = _rows_entering(lengths, schedule, l_entering)
+    a = sum(rows[:seq])
+    assert packed.shape[0] == sum(rows)
+    return packed[a:a + rows[seq]]
+
+
+def _layer_inputs(eng, shape, emb, l, schedule, n, seq=0, lengths=None):
     """Rows and positions that ENTER layer l on the GPU (its own previous output)."""
+    lengths = [n] if lengths is None else lengths
     pos = np.arange(n)
     for e, _ in schedule:
         if e <= l:
-            pos = to_np(eng.lazy_get_kept(e, 0)).astype(np.int64)
-    x = emb if l == 0 else to_np(eng.lazy_get_hidden(l - 1))
+            pos = to_np(eng.lazy_get_kept(e, seq)).astype(np.int64)
+    x = emb if l == 0 else to_np(_member_rows(eng.lazy_get_hidden(l - 1), lengths, schedule, l, seq))
     assert x.shape[0] == len(pos)
     return x, pos
 
 
-def _check_layer_against_oracle(eng, shape, lw, emb, l, schedule, n, rows=None):
+def _check_layer_against_oracle(eng, shape, lw, emb, l, schedule, n, seq=0, lengths=None):
     """Layer l of the GPU run against the oracle applied to the GPU's own input of that layer: the
     per-layer form of the parity bound (2e-2 per tensor, scores 1e-3), free of the drift that a deep
-    bf16 stack accumulates against an fp64 run."""
-    x_in, pos = _layer_inputs(eng, shape, emb, l, schedule, n)
+    bf16 stack accumulates against an fp64 run.  seq / lengths pick one member of a packed batch."""
+    lengths = [n] if lengths is None else lengths
+    x_in, pos = _layer_inputs(eng, shape, emb, l, schedule, n, seq, lengths)
     keep = None
     for e, _ in schedule:
         if e == l + 1:
-            keep = to_np(eng.lazy_get_kept(e, 0)).astype(np.int64)
+            keep = to_np(eng.lazy_get_kept(e, seq)).astype(np.int64)
     ref = O.layer_step(shape, lw, x_in, pos, keep_pos=keep)
-    sc = to_np(eng.lazy_get_scores(l, 0))
+    sc = to_np(eng.lazy_get_scores(l, seq))
     assert np.max(np.abs(sc - ref["scores"])) < 1e-3
     rel = np.abs(sc - ref["scores"]) / ref["scores"].clip(1e-30)
     assert np.max(rel) < 3e-2, (l, np.max(rel))       # same inputs on both sides: only one layer's rounding
@@ -74,12 +101,12 @@ def _check_layer_against_oracle(eng, shape, lw, emb, l, schedule, n, rows=None):
         s_of = dict(zip(pos.tolist(), ref["scores"].tolist()))
         for p in diff:
             assert abs(s_of[p] - tau) <= 3e-2 * tau and abs(s_of[p] - tau) <= 1e-3
-        apos, ahid = eng.lazy_get_aux(l, 0)
+        apos, ahid = eng.lazy_get_aux(l, seq)
         assert np.array_equal(to_np(apos), ref["aux_pos"])
         assert rel_err(to_np(ahid), ref["aux_rows"]) < TOL
-    got = to_np(eng.lazy_get_hidden(l))
+    got = to_np(_member_rows(eng.lazy_get_hidden(l), lengths, schedule, l + 1, seq))
     assert rel_err(got, ref["hidden_out"]) < TOL, (l, rel_err(got, ref["hidden_out"]))
-    kpos, kk, vv = eng.lazy_get_kv(l, 0)
+    kpos, kk, vv = eng.lazy_get_kv(l, seq)
     assert np.array_equal(to_np(kpos), pos)
     assert rel_err(to_np(kk), ref["k"].reshape(len(pos), -1)) < TOL
     assert rel_err(to_np(vv), ref["v"].reshape(len(pos), -1)) < TOL
@@ -172,6 +199,52 @@ def test_7b_full_depth_prefill_sampled_and_properties(model7b):
     eng.close()
 
 
+def test_7b_full_depth_forced_replay_end_to_end_drift(model7b):
+    """The whole 32-layer, 3376-token pruned prefill against the fp64 oracle replayed on the GPU's three
+    kept sets (a chain of `layer_step` calls, one layer's weights widened at a time: the same arithmetic as
+    `prefill` with forced sets).  Records the drift of the residual stream per layer, the error of the
+    first-token logits and whether the greedy token agrees.  The per-tensor 2e-2 bound is a one-layer
+    bound (see _check_layer_against_oracle); end to end the bf16 rounding of 32 layers accumulates, and the
+    gates below are what the measurement supports, with margin."""
+    shape, schedule, n = synth.LLAMA7B, synth.SCHEDULE_7B, 3376
+    ids = synth.make_prompt(shape.vocab, n, 100)
+    eng = B.LazyPrefill(shape, model7b, schedule, torch.bfloat16, 1, n, debug_capture=True)
+    logits = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+    eng.lazy_prefill_run(ids.cuda(), [0, n], logits)
+    eng.lazy_sync_status()
+    kept = {e: to_np(eng.lazy_get_kept(e, 0)).astype(np.int64) for e, _ in schedule}
+    x = to_np(model7b["tok_embed"][ids.long().cuda()]).astype(np.float64)
+    pos = np.arange(n)
+    drift, score_abs, score_rel = [], [], []
+    for l in range(shape.n_layers):
+        lw = {k: to_np(v) for k, v in model7b["layers"][l].items()}
+        ref = O.layer_step(shape, lw, x, pos, keep_pos=kept.get(l + 1))
+        drift.append(rel_err(to_np(eng.lazy_get_hidden(l)), ref["hidden_out"]))
+        sc = to_np(eng.lazy_get_scores(l, 0))
+        score_abs.append(float(np.max(np.abs(sc - ref["scores"]))))
+        score_rel.append(float(np.max(np.abs(sc - ref["scores"]) / ref["scores"].clip(1e-30))))
+        x, pos = ref["hidden_out"], ref["pos_out"]
+    ref_logits = O.lm_head(shape, {"g_final": to_np(model7b["g_final"]), "w_lm_head": to_np(model7b["w_lm_head"])},
+                           x[-1])
+    got = to_np(logits[0]).astype(np.float64)
+    lerr = rel_err(got, ref_logits)
+    order = np.argsort(-ref_logits)
+    rank_of_gpu_argmax = int(np.nonzero(order == int(np.argmax(got)))[0][0])
+    top10 = len(set(order[:10].tolist()) & set(np.argsort(-got)[:10].tolist()))
+    print("e2e drift per layer:", " ".join(f"{d:.4f}" for d in drift))
+    print(f"e2e logits rel err {lerr:.4f}; greedy token equal: {rank_of_gpu_argmax == 0} "
+          f"(GPU argmax is the oracle's rank {rank_of_gpu_argmax}); top-10 overlap {top10}/10; "
+          f"scores: max abs {max(score_abs):.2e}, max rel {max(score_rel):.3f}")
+    assert drift[0] < TOL and drift[1] < TOL                   # no accumulation yet: the one-layer bound
+    print("e2e score abs err per layer:", " ".join(f"{a:.1e}" for a in score_abs))
+    assert max(score_abs[:8]) < 1e-3                           # Eq. 1 scores before the first cut: the one-layer bound
+    assert max(score_abs) < E2E_SCORE_ABS_GATE                 # deeper: inputs have drifted, see the gates above
+    assert all(d < 1.6e-2 * (l + 1) ** 0.5 + 4e-3 for l, d in enumerate(drift))   # random-walk growth, not linear
+    assert max(drift) < E2E_DRIFT_GATE and lerr < E2E_LOGITS_GATE
+    assert rank_of_gpu_argmax < 3 and top10 >= 8
+    eng.close()
+
+
 def test_7b_prefill_4096_then_32_decode_steps_properties(model7b):
     shape, schedule, n, steps = synth.LLAMA7B, synth.SCHEDULE_7B, 4096, 32
     ids = synth.make_prompt(shape.vocab, n, 101)
@@ -218,11 +291,11 @@ def test_7b_prefill_4096_then_32_decode_steps_properties(model7b):
     eng.close()
 
 
-def test_7b_varlen_batch_of_8_equals_sequences_run_alone(model7b):
+def test_7b_varlen_batch_of_8_vs_oracle_and_vs_sequences_run_alone(model7b):
     shape, schedule = synth.LLAMA7B, synth.SCHEDULE_7B
     lengths = synth.make_varlen_lengths(8, 1024, 4096, seed=4)
     ids, cu = synth.make_varlen_batch(shape.vocab, lengths, seed=5)
-    eng = B.LazyPrefill(shape, model7b, schedule, torch.bfloat16, 8, sum(lengths))
+    eng = B.LazyPrefill(shape, model7b, schedule, torch.bfloat16, 8, sum(lengths), debug_capture=True)
     logits = torch.empty((8, shape.vocab), dtype=torch.float32, device="cuda")
     d_ids = ids.cuda()
     eng.lazy_prefill_run(d_ids, cu, logits)
@@ -232,23 +305,59 @@ def test_7b_varlen_batch_of_8_equals_sequences_run_alone(model7b):
     for s in range(8):
         _check_selection_properties(eng, lengths[s], schedule, s, shape.n_layers)
         kept_batch.append([to_np(eng.lazy_get_kept(e, s)) for e, _ in schedule])
+    # one member of the packed batch against the ORACLE, element by element, on the GPU's own layer inputs:
+    # the first layer, the layer that holds the first cut and the one after it (a member in the middle of
+    # the packing, so that its rows start inside a GEMM tile and an attention launch of their own)
+    m = 3
+    emb = to_np(model7b["tok_embed"][d_ids[cu[m]:cu[m + 1]].long()])
+    for l in (0, 7, 8):
+        lw = {k: to_np(v) for k, v in model7b["layers"][l].items()}
+        _check_layer_against_oracle(eng, shape, lw, emb, l, schedule, lengths[m], seq=m, lengths=lengths)
+    h_last = to_np(_member_rows(eng.lazy_get_hidden(31), lengths, schedule, 32, m))[-1]
+    ref_logits = O.lm_head(shape, {"g_final": to_np(model7b["g_final"]), "w_lm_head": to_np(model7b["w_lm_head"])},
+                           h_last)
+    assert rel_err(to_np(logits[m]), ref_logits) < TOL
+    score_batch = {s: [to_np(eng.lazy_get_scores(e - 1, s)) for e, _ in schedule] for s in (0, 3, 7)}
     eng.close()
     del eng
     torch.cuda.empty_cache()
+    # Sequences are independent, so a member run alone must reproduce the batch.  Not bit for bit: which
+    # output tiles of a GEMM get their K loop split across SMs depends on the total row count, and a split
+    # tile adds its fp32 partial sums in another order.  The comparison is therefore made cut by cut on EQUAL
+    # inputs: the solo run is handed the batch's kept sets for the earlier cuts and selects freely at cut i;
+    # the two sets may then differ only in tokens whose score lies within 3 % of the threshold (the band of
+    # the oracle tests), and with all three sets handed over the logits agree to the one-tensor tolerance.
     solo = B.LazyPrefill(shape, model7b, schedule, torch.bfloat16, 1, max(lengths))
     lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
     for s in (0, 3, 7):
-        solo.lazy_prefill_run(d_ids[cu[s]:cu[s + 1]].contiguous(), [0, lengths[s]], lg)
-        solo.lazy_sync_status()
-        # Sequences are independent.  Not bit-identical, though: which output tiles of a GEMM get their K
-        # loop split across SMs depends on the total row count, and a split tile adds its fp32 partial
-        # sums in another order.  So: the same kept sets up to near-ties at the threshold, the same logits
-        # to bf16 noise.
+        p_ids = d_ids[cu[s]:cu[s + 1]].contiguous()
         for i, (e, _) in enumerate(schedule):
+            for j in range(i):
+                solo.lazy_set_forced_keep(schedule[j][0], 0, torch.tensor(kept_batch[s][j], dtype=torch.int32).cuda())
+            solo.lazy_prefill_run(p_ids, [0, lengths[s]], lg)
+            solo.lazy_sync_status()
             a, b = to_np(solo.lazy_get_kept(e, 0)), kept_batch[s][i]
             assert len(a) == len(b)
-            # (random-init attention is nearly flat, so rounding noise moves a few per cent of the ranks
-            # next to the threshold by the third cut)
-            assert len(np.intersect1d(a, b)) >= 0.93 * len(a)
-        assert rel_err(to_np(lg[0]), to_np(logits[s]).astype(np.float64)) < 2 * TOL
+            cand = np.arange(lengths[s]) if i == 0 else kept_batch[s][i - 1]
+            sc = score_batch[s][i]
+            assert sc.shape == cand.shape
+            tau = np.sort(sc[:-1])[::-1][len(b) - 2]
+            s_of = dict(zip(cand.tolist(), sc.tolist()))
+            diff = set(a.tolist()) ^ set(b.tolist())
+            for p in diff:
+                assert abs(s_of[p] - tau) <= 3e-2 * tau, (s, e, p, s_of[p], tau)
+            print(f"seq {s} cut entering layer {e}: {len(diff) // 2} of {len(b)} tokens differ (near-ties)")
+        for j, (e, _) in enumerate(schedule):
+            solo.lazy_set_forced_keep(e, 0, torch.tensor(kept_batch[s][j], dtype=torch.int32).cuda())
+        solo.lazy_prefill_run(p_ids, [0, lengths[s]], lg)
+        solo.lazy_sync_status()
+        assert rel_err(to_np(lg[0]), to_np(logits[s]).astype(np.float64)) < TOL
+        # free-running, for the record: rounding noise moves ranks next to the threshold, and a different
+        # set at one cut changes every later score a little
+        solo.lazy_prefill_run(p_ids, [0, lengths[s]], lg)
+        solo.lazy_sync_status()
+        ov = [len(np.intersect1d(to_np(solo.lazy_get_kept(e, 0)), kept_batch[s][i])) / len(kept_batch[s][i])
+              for i, (e, _) in enumerate(schedule)]
+        print(f"seq {s} free-running kept-set overlap with the batch run per cut: {[round(o, 4) for o in ov]}")
+        assert ov[0] >= 0.99 and min(ov) >= 0.90
     solo.close()

@@ -267,6 +267,19 @@ def test_attention_and_score(dtype, H, dh, lengths):
         assert abs(s[a:b].sum() - 1) < 1e-4
 
 
+def test_attention_beyond_4096_keys():
+    """One sequence longer than 4096 tokens (more than 64 key tiles per query tile, several waves of query
+    tiles) next to a short one, against the explicit n x n oracle: long prompts are timed at 8k-32k tokens,
+    so the kernel is also checked element by element past 4096 keys."""
+    o, o_ref, s, s_ref, cu = _attention_case(torch.bfloat16, 2, 128, [4500, 300], 60)
+    assert rel_err(o, o_ref) < BF16_STEP_TOL
+    assert np.max(np.abs(s - s_ref)) < 1e-3
+    assert np.max(np.abs(s - s_ref) / s_ref.clip(1e-12)) < 2e-2
+    # rows near the end of the long sequence individually (a max over the whole tensor is set by early rows)
+    for r in (4096, 4223, 4499):
+        assert rel_err(o[r], o_ref[r]) < BF16_STEP_TOL
+
+
 def test_attention_running_max_rescale_path():
     """Logits that keep growing with the key index force the streaming softmax to raise its running
     maximum late (the tensor-core kernel then rescales the accumulator it keeps in tensor memory)."""
@@ -336,3 +349,25 @@ def test_gather_rows_reports_a_bad_index_instead_of_reading_it():
         B.lazy_device_status()
     assert e.value.status == -1
     B.lazy_device_status()                                          # cleared
+
+
+# ----------------------------------------------------------------------------- bounded waits
+@pytest.mark.parametrize("which,where", [(0, 15), (1, 14)])
+def test_bounded_wait_runs_out_and_reports_timeout(which, where):
+    """Every device-side wait of the tensor-core kernels is bounded.  A one-warp kernel waits, for at most
+    one millisecond, on an mbarrier phase (which = 0) or on a split-wave arrival counter (which = 1) that
+    nothing ever signals; no copy or MMA is in flight.  The wait must give up, LAZY_E_TIMEOUT with the
+    waiting site's code must come back through the status word, and the device must serve the next call."""
+    B.lazy_device_status()                                   # start from a clean status word
+    B.lazy_k_wait_selftest(which, 1000)
+    with pytest.raises(B.LazyError) as e:
+        B.lazy_device_status()
+    assert e.value.status == -5                              # LAZY_E_TIMEOUT
+    assert B.lazy_status_detail()[0] == where
+    B.lazy_device_status()                                   # cleared by the read
+    x = torch.randn((64, 256)).to(torch.bfloat16).cuda()
+    w = torch.randn((128, 256)).to(torch.bfloat16).cuda()
+    got = B.lazy_k_gemm(x, w)                                # the device still answers, results still right
+    B.lazy_device_status()
+    ref = x.double().cpu().numpy() @ w.double().cpu().numpy().T
+    assert rel_err(to_np(got), ref) < 1e-2

@@ -404,6 +404,24 @@ def test_decode_invariants_with_pruning():
     frac = O.tokens_computed_fraction(st, 40)
     assert frac[0] == 1.0 and all(0 < f <= 1.0 for f in frac)
     assert all(frac[l + 1] <= frac[l] for l in range(shape.n_layers - 1))
+    # exact values, counted independently from the caches: prompt positions are 0..39, generated
+    # tokens (positions >= 40) must not count, position 39 must
+    for l, c in enumerate(st.layers):
+        assert frac[l] == len(set(c.kv.keys()) & set(range(40))) / 40.0
+
+
+def test_tokens_computed_fraction_hand_worked():
+    """Right after a prefill of 10 tokens with keep 70 % entering layer 1 and 30 % entering layer 2, the
+    fractions are 10/10, 7/10, 3/10 by the keep counts alone; a decode step adds position 10, which is
+    not a prompt token, and revives prompt tokens only into layers that already count them or not."""
+    shape = MINI
+    W = weights_to_np(mini_weights(seed=23))
+    ids = to_np(synth.make_prompt(shape.vocab, 10, seed=23))
+    st = O.prefill(shape, W, ids, ((1, 7000), (2, 3000)))
+    assert O.tokens_computed_fraction(st, 10) == [1.0, 0.7, 0.3] + [0.3] * (shape.n_layers - 3)
+    # a boundary case of the prompt/generated split: with n_prompt = 9, position 9 is not counted
+    assert O.tokens_computed_fraction(st, 9)[0] == 1.0
+    assert O.tokens_computed_fraction(st, 11)[0] == 10.0 / 11.0
 
 
 def test_decode_revived_row_feeds_deferred_mlp():

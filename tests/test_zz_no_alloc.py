@@ -6,7 +6,8 @@ the whole device, or late in a process that has already given its memory away.  
 `lazy_k_score_static` keeps its scratch in a fixed array inside the library.  This test calls it
 through the C ABI, twice in a row on different inputs (the array is shared and keeps whatever the
 previous call left behind), and checks each result against the ordinary entry point, whose
-scratch the caller provides.  It also checks that oversized requests are refused.
+scratch the caller provides, and against the CPU oracle's Eq. 1.  It also checks that oversized
+requests are refused.
 
 The file sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+import lazyllm_oracle as O
 from paper_2407_14057_b200 import binding as B
 from paper_2407_14057_b200 import build
 
@@ -46,6 +48,15 @@ def test_static_scratch_score_matches_caller_scratch_score_twice_in_a_row():
         assert torch.max(torch.abs(got - want)).item() < 1e-3            # the tolerance of the score tests
         assert torch.equal(got, want)                                      # same kernels: same bits
         assert abs(got[: lengths[0]].sum().item() - 1.0) < 1e-4
+        # and against the definition itself (Eq. 1 written out on the CPU), sequence by sequence
+        qn = q.float().cpu().numpy().reshape(n, H, dh)
+        kn = k.float().cpu().numpy().reshape(n, H, dh)
+        a = 0
+        for ln in lengths:
+            pos = np.arange(ln)
+            _, s_ref = O.attend(qn[a:a + ln], kn[a:a + ln], np.zeros((ln, H, dh)), pos, pos, -1)
+            assert np.max(np.abs(got[a:a + ln].cpu().numpy() - s_ref)) < 1e-3
+            a += ln
 
 
 def test_static_scratch_score_refuses_sizes_beyond_its_array():
