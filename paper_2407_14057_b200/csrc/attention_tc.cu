@@ -84,6 +84,32 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Three-input maximum and two-wide fp32 arithmetic (one instruction each on this architecture): the
+// softmax threads are bound by instruction issue, so halving the count of the plain ALU work matters.
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long f32x2_pack(float lo, float hi) {
+  unsigned long long p;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(lo), "f"(hi));
+  return p;
+}
+__device__ __forceinline__ void f32x2_unpack(unsigned long long p, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ unsigned long long f32x2_fma(unsigned long long a, unsigned long long b,
+                                                        unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long f32x2_add(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 
 __global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -100,7 +126,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   AttBarriers *bars = reinterpret_cast<AttBarriers *>(smem + Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y;
+  // Heads are the fastest grid dimension and query tiles run from the longest to the shortest along y, so
+  // CTAs are handed out longest first over ALL heads: the long tiles of the last head start with the first
+  // wave instead of at the end of the launch.
+  const int h = blockIdx.x;
   int q_start = q_start_arg, n = n_arg, kv_start = kv_start_arg;
   if (cu_q) {
     q_start = cu_q[blockIdx.z];
@@ -108,8 +137,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     kv_start = kv_base ? kv_base[blockIdx.z] : q_start;
   }
   const int q_tiles = (n + TQ - 1) / TQ;
-  if ((int)blockIdx.x >= q_tiles) return;          // before any barrier or TMEM use: safe to leave
-  const int qt = q_tiles - 1 - blockIdx.x;         // longest rows first
+  if ((int)blockIdx.y >= q_tiles) return;          // before any barrier or TMEM use: safe to leave
+  const int qt = q_tiles - 1 - blockIdx.y;         // longest rows first
   const int q0 = qt * TQ;
   const int n_kt = (min(q0 + TQ, n) + TK - 1) / TK;  // key tiles up to the diagonal
 
@@ -241,8 +270,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const bool score_warp = __any_sync(0xffffffffu, score_row);
     const int seq_id = cu_q ? (int)blockIdx.z : sc.seq_id;
     // row (seq, h) of P: max_tiles * 64 floats, 16-byte aligned, so whole tiles are stored as float4
-    float *sc_p = score_row ? sc.p + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles * TK : nullptr;
-    float *sc_m = score_row ? sc.mtile + ((size_t)seq_id * gridDim.y + h) * sc.max_tiles : nullptr;
+    float *sc_p = score_row ? sc.p + ((size_t)seq_id * gridDim.x + h) * sc.max_tiles * TK : nullptr;
+    float *sc_m = score_row ? sc.mtile + ((size_t)seq_id * gridDim.x + h) * sc.max_tiles : nullptr;
     for (int j = 0; j < n_kt && ok; ++j) {
       const int b = j & 1;
       ok = mbar_wait(smem_u32(&bars->s_full), (uint32_t)j & 1u, abort_flag, status, W_ATTN_SOFTMAX);
@@ -265,13 +294,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         for (int c = 0; c < 64; ++c)
           if (col0 + c > row) raw[c] = 0xff800000u;  // -inf
       }
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains: shorter dependency
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains of three-input maxima
 #pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-        mx[0] = fmaxf(mx[0], __uint_as_float(raw[c]));
-        mx[1] = fmaxf(mx[1], __uint_as_float(raw[c + 1]));
-        mx[2] = fmaxf(mx[2], __uint_as_float(raw[c + 2]));
-        mx[3] = fmaxf(mx[3], __uint_as_float(raw[c + 3]));
+      for (int c = 0; c < 64; c += 8) {
+        mx[0] = fmax3(mx[0], __uint_as_float(raw[c]), __uint_as_float(raw[c + 1]));
+        mx[1] = fmax3(mx[1], __uint_as_float(raw[c + 2]), __uint_as_float(raw[c + 3]));
+        mx[2] = fmax3(mx[2], __uint_as_float(raw[c + 4]), __uint_as_float(raw[c + 5]));
+        mx[3] = fmax3(mx[3], __uint_as_float(raw[c + 6]), __uint_as_float(raw[c + 7]));
       }
       const float mj = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * sl2;  // log2 units
       float alpha = 1.f;
@@ -302,16 +331,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           tmem_st_wait();
         }
       }
-      // p = 2^(s * scale - m): one FFMA and one ex2 per element
+      // p = 2^(s * scale - m): half a two-wide FMA, one ex2 and one add per element (two-wide sums as well
+      // pushed the kernel over its register budget)
       float sm[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
       const float neg_m = -m;
+      const unsigned long long sl2x2 = f32x2_pack(sl2, sl2), negmx2 = f32x2_pack(neg_m, neg_m);
 #pragma unroll
       for (int c = 0; c < 64; c += 4) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(raw[c]), sl2, neg_m));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(raw[c + 1]), sl2, neg_m));
-        const float p2 = ex2_approx(fmaf(__uint_as_float(raw[c + 2]), sl2, neg_m));
-        const float p3 = ex2_approx(fmaf(__uint_as_float(raw[c + 3]), sl2, neg_m));
+        float x0, x1, x2, x3;
+        f32x2_unpack(f32x2_fma(f32x2_pack(__uint_as_float(raw[c]), __uint_as_float(raw[c + 1])), sl2x2, negmx2), x0, x1);
+        f32x2_unpack(f32x2_fma(f32x2_pack(__uint_as_float(raw[c + 2]), __uint_as_float(raw[c + 3])), sl2x2, negmx2), x2, x3);
+        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
         sm[0] += p0;
         sm[1] += p1;
         sm[2] += p2;
@@ -361,7 +392,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       ok = __all_sync(0xffffffffu, ok);
     }
     if (ok && score_row) {
-      float *stt = sc.stats + ((size_t)seq_id * gridDim.y + h) * 2;
+      float *stt = sc.stats + ((size_t)seq_id * gridDim.x + h) * 2;
       stt[0] = m;
       stt[1] = 1.f / l;
     }
@@ -422,7 +453,7 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
                                       ATT_SMEM_BYTES));
     attr_set = true;
   }
-  dim3 grid(cdiv(max_len, TQ), n_heads, n_seqs);
+  dim3 grid(n_heads, cdiv(max_len, TQ), n_seqs);
   AttnScoreOut sc = {nullptr, nullptr, nullptr, 0, 0};
   if (score_scratch) {  // layout: P [S, H, max_tiles*64] | mtile [S, H, max_tiles] | stats [S, H, 2]
     sc.p = score_scratch;
@@ -440,10 +471,15 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
 namespace {
 // Eq. 1 from the attention kernel's by-product: s_r = (1/H) sum_h p[h][r] * 2^(m_tile - m_final) / l.
 // Eight lanes share a key row, each summing every eighth head; a fixed shuffle tree adds them up.
-__global__ void score_from_attention_kernel(const float *__restrict__ p, const float *__restrict__ mtile,
-                                            const float *__restrict__ stats, const int32_t *__restrict__ cu_q,
-                                            int n_seqs, int n_total, int n_heads, int max_tiles,
-                                            float *__restrict__ scores) {
+// blockIdx.y = layer of a group of consecutive layers that share the same rows (cu_q): layer y reads the
+// by-product at scratch + y * scratch_stride and writes scores + y * scores_stride, so that the head means
+// of all layers between two cuts take one launch.
+__global__ void score_from_attention_kernel(const float *__restrict__ scratch, size_t scratch_stride,
+                                            const int32_t *__restrict__ cu_q, int n_seqs, int n_total, int n_heads,
+                                            int max_tiles, float *__restrict__ scores, size_t scores_stride) {
+  const float *p = scratch + (size_t)blockIdx.y * scratch_stride;
+  const float *mtile = p + (size_t)n_seqs * n_heads * max_tiles * TK;
+  const float *stats = mtile + (size_t)n_seqs * n_heads * max_tiles;
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   const int r = t >> 3, part = t & 7;
   float acc = 0.f;
@@ -464,7 +500,7 @@ __global__ void score_from_attention_kernel(const float *__restrict__ p, const f
   acc += __shfl_xor_sync(0xffffffffu, acc, 1);
   acc += __shfl_xor_sync(0xffffffffu, acc, 2);
   acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-  if (r < n_total && part == 0) scores[r] = acc / (float)n_heads;
+  if (r < n_total && part == 0) scores[(size_t)blockIdx.y * scores_stride + r] = acc / (float)n_heads;
 }
 }  // namespace
 
@@ -472,13 +508,14 @@ size_t attn_score_scratch_floats(int n_seqs, int n_heads, int max_tiles) {
   return (size_t)n_seqs * n_heads * max_tiles * (TK + 1) + (size_t)2 * n_seqs * n_heads;
 }
 
-int launch_score_from_attention(cudaStream_t st, const float *scratch, const int32_t *cu_q, int n_seqs,
-                                int n_total, int n_heads, int max_tiles, float *scores) {
-  if (n_total == 0) return LAZY_OK;
-  const float *mtile = scratch + (size_t)n_seqs * n_heads * max_tiles * TK;
-  const float *stats = mtile + (size_t)n_seqs * n_heads * max_tiles;
-  score_from_attention_kernel<<<cdiv(n_total * 8, 256), 256, 0, st>>>(scratch, mtile, stats, cu_q, n_seqs, n_total,
-                                                                     n_heads, max_tiles, scores);
+// n_layers consecutive layers over the same rows: layer y's by-product at scratch + y * scratch_stride,
+// its scores to scores + y * scores_stride.
+int launch_score_from_attention(cudaStream_t st, const float *scratch, size_t scratch_stride, int n_layers,
+                                const int32_t *cu_q, int n_seqs, int n_total, int n_heads, int max_tiles,
+                                float *scores, size_t scores_stride) {
+  if (n_total == 0 || n_layers == 0) return LAZY_OK;
+  score_from_attention_kernel<<<dim3(cdiv(n_total * 8, 256), n_layers), 256, 0, st>>>(
+      scratch, scratch_stride, cu_q, n_seqs, n_total, n_heads, max_tiles, scores, scores_stride);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

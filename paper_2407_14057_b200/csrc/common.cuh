@@ -193,9 +193,11 @@ size_t gemm_scratch_bytes();
 // b_const: the caller guarantees that B (the weights) is not written by earlier work still in flight on
 // the stream; only then may the weight-streaming kernel (M <= 4) start fetching B while the kernel before
 // it drains.
+// res_rows (device int32[M], optional, bf16 tensor-core path with R only): the addend of output row r is
+// R[res_rows[r]] instead of R[r]; R and C must then be different buffers.
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
                 int M, int N, int K, DevStatus *status, void *scratch = nullptr, size_t scratch_bytes = 0,
-                int force_kernel = 0, bool b_const = false);
+                int force_kernel = 0, bool b_const = false, const int32_t *res_rows = nullptr);
 int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg, const void *Bu,
                        void *C, int M, int F, int K, DevStatus *status, void *scratch = nullptr,
                        size_t scratch_bytes = 0, int force_kernel = 0, bool b_const = false);
@@ -203,6 +205,7 @@ int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg
 // head_dim 128, d_model a multiple of 256): qkv [M, 3d] receives the rotated q (its k and v thirds
 // are left untouched), rotated k and v go to cache rows kv_row[r] (or r) with their position tag.
 bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
+bool gemm_res_rows_supported(int dtype, int M, int K);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
@@ -241,11 +244,14 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
                         int n, int kv_start, DevStatus *status, float *score_scratch = nullptr,
                         int max_tiles = 0, int n_seqs_total = 0, int seq_id = 0);
 // With score_scratch (attn_score_scratch_floats floats) the attention kernel also leaves the last
-// row's softmax numerators there; launch_score_from_attention turns them into the Eq. 1 scores.
+// row's softmax numerators there; launch_score_from_attention turns them into the Eq. 1 scores, for
+// n_layers consecutive layers over the same rows in one launch (layer y: by-product at scratch +
+// y * scratch_stride, scores to scores + y * scores_stride).
 // max_tiles = ceil(longest sequence / 64), the same value in both calls.
 size_t attn_score_scratch_floats(int n_seqs, int n_heads, int max_tiles);
-int launch_score_from_attention(cudaStream_t st, const float *scratch, const int32_t *cu_q, int n_seqs,
-                                int n_total, int n_heads, int max_tiles, float *scores);
+int launch_score_from_attention(cudaStream_t st, const float *scratch, size_t scratch_stride, int n_layers,
+                                const int32_t *cu_q, int n_seqs, int n_total, int n_heads, int max_tiles,
+                                float *scores, size_t scores_stride);
 // True when the tensor-core prefill attention applies.
 bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
@@ -281,9 +287,12 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
                     int head_dim, float *scratch, float *scores);
 int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t *cu_in, int n_seqs,
                             uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts);
+// With pos_in (position of every input row) the kernel also writes the kept rows' positions to pos_keep
+// (packed like keep_idx) and the dropped rows' positions to aux_pos[aux_dst[j]] (j = slot in drop_idx).
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
                   const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
-                  DevStatus *status);
+                  DevStatus *status, const int32_t *pos_in = nullptr, int32_t *pos_keep = nullptr,
+                  const int32_t *aux_dst = nullptr, int32_t *aux_pos = nullptr);
 // scores[r] = 2 if pos[r] is in the ascending list forced[0..n_forced), else 0 (rows r0..r0+n)
 int launch_forced_scores(cudaStream_t st, const int32_t *pos, int r0, int n, const int32_t *forced,
                          int n_forced, float *scores);

@@ -157,9 +157,83 @@ __global__ void rmsnorm_kernel(const T *__restrict__ x, const int32_t *__restric
   }
 }
 
+// One WARP per row, the row held in registers between the sum of squares and the scaling: x is read
+// once (VPL 16-byte vectors per lane, all requested before the first is used), no shared memory, no
+// block barrier.  Rows of VPL * 32 vectors exactly (d = 4096 in bf16: VPL = 16).
+template <typename T, int VPL>
+__global__ void __launch_bounds__(256)
+rmsnorm_warp_kernel(const T *__restrict__ x, const int32_t *__restrict__ row_idx, const T *__restrict__ g,
+                    T *__restrict__ y, int n, int d, float eps) {
+  constexpr int V = Elem<T>::kPerVec;
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= n) return;
+  const size_t src_row = row_idx ? (size_t)row_idx[r] : (size_t)r;
+  const uint4 *xr = reinterpret_cast<const uint4 *>(x + src_row * d);
+  uint4 *yr = reinterpret_cast<uint4 *>(y + (size_t)r * d);
+  const uint4 *gr = reinterpret_cast<const uint4 *>(g);
+  Vec16<T> v[VPL];
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) v[u].raw = xr[lane + 32 * u];
+  float ss = 0.f;
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    float f[V];
+    v[u].unpack(f);
+#pragma unroll
+    for (int j = 0; j < V; ++j) ss += f[j] * f[j];
+  }
+  ss = warp_sum(ss);
+  const float scale = rsqrtf(ss / (float)d + eps);
+  // Only the packed row stays in registers across the reduction: the values are unpacked again below
+  // (the empty asm keeps the compiler from carrying the unpacked copy along, which costs occupancy).
+#pragma unroll
+  for (int u = 0; u < VPL; ++u)
+    asm volatile("" : "+r"(v[u].raw.x), "+r"(v[u].raw.y), "+r"(v[u].raw.z), "+r"(v[u].raw.w));
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    Vec16<T> gv, o;
+    gv.raw = gr[lane + 32 * u];
+    float f[V], gf[V];
+    v[u].unpack(f);
+    gv.unpack(gf);
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] = f[j] * scale * gf[j];
+    o.pack(f);
+    yr[lane + 32 * u] = o.raw;
+  }
+}
+
+template <typename T>
+static bool launch_rmsnorm_warp(cudaStream_t st, const T *x, const int32_t *row_idx, const T *g, T *y, int n, int d,
+                                float eps) {
+  const int nvec = d / Elem<T>::kPerVec;
+  if (nvec % 32) return false;
+  const int blocks = cdiv(n, 8);
+  switch (nvec / 32) {
+#define RW_CASE(v)                                                                                    \
+  case v:                                                                                             \
+    rmsnorm_warp_kernel<T, v><<<blocks, 256, 0, st>>>(x, row_idx, g, y, n, d, eps);                   \
+    return true;
+    RW_CASE(1) RW_CASE(2) RW_CASE(4) RW_CASE(8) RW_CASE(16)
+#undef RW_CASE
+    default: return false;
+  }
+}
+
 int launch_rmsnorm_rows(cudaStream_t st, int dtype, const void *x, const int32_t *row_idx,
                         const void *g, void *y, int n, int d, float eps) {
   if (n == 0) return LAZY_OK;
+  // The sum of squares is added in another order than in the one-CTA-per-row kernel below (per lane over
+  // its vectors, then the shuffle tree): rows whose width the warp kernel covers always take it, so a
+  // given shape is always normalised by the same kernel.
+  const bool warp_ok = dtype == LAZY_F32
+                           ? launch_rmsnorm_warp<float>(st, (const float *)x, row_idx, (const float *)g, (float *)y, n, d, eps)
+                           : launch_rmsnorm_warp<bf16>(st, (const bf16 *)x, row_idx, (const bf16 *)g, (bf16 *)y, n, d, eps);
+  if (warp_ok) {
+    LAZY_COUNT_LAUNCH();
+    return launch_ok();
+  }
   if (dtype == LAZY_F32)
     rmsnorm_kernel<float, 128><<<n, 128, 0, st>>>((const float *)x, row_idx, (const float *)g,
                                                   (float *)y, d, eps);

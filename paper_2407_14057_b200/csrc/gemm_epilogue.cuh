@@ -9,10 +9,12 @@ constexpr int GEMM_ACC_N = 256;  // accumulator columns per tile
 
 enum { EPI_PLAIN = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_QKV_ROPE = 3 };
 
-// Extra operands of the QKV epilogue: the rotary embedding is applied to the fp32 accumulators and
+// Extra operands of the epilogues.  QKV: the rotary embedding is applied to the fp32 accumulators and
 // the rotated k, and v, go straight to the layer's cache rows (head_dim 128: one 256-column tile is
-// two whole heads of q, k or v, and a thread holds its row's full heads).
+// two whole heads of q, k or v, and a thread holds its row's full heads).  Residual: an optional row
+// list for the addend, so that C[r] = acc[r] + R[res_rows[r]] compacts the residual stream on the way.
 struct RopeArgs {
+  const int32_t *res_rows = nullptr;  // [M] row of R added to output row r (NULL: r)
   const int32_t *pos;     // [M] original positions
   const float2 *table;    // [max_pos][64] (cos, sin)
   bf16 *kcache, *vcache;  // [rows, d_model]
@@ -208,6 +210,19 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// Residual addend of the 32 output columns [col0, col0 + 32) of a row, as four 16-byte vectors (a vector
+// beyond N, or a row beyond M, is left as it is).  A thread asks for them well before it needs them: the
+// first 32 columns of a tile before it waits for the tile's accumulator, every later group while it works
+// on the group before, so the L2 latency of these row-strided reads stays off the epilogue's critical path.
+__device__ __forceinline__ void gemm_residual_load(uint4 (&r)[4], const bf16 *__restrict__ R, const RopeArgs &extra,
+                                                   int row, int col0, int M, int N, int ldc) {
+  if (row >= M) return;
+  const bf16 *rrow = R + (size_t)(extra.res_rows ? extra.res_rows[row] : row) * ldc;
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    if (col0 + 8 * j < N) r[j] = *reinterpret_cast<const uint4 *>(rrow + col0 + 8 * j);
+}
+
 // One thread, one row.  taddr: TMEM address of the row's first accumulator column (lane field set);
 // row: global output row; n0: first output column of the tile as the caller sees it.  C is [M, ldc];
 // for EPI_SWIGLU accumulator columns [0,128) are gate features, [128,256) the matching up features and C
@@ -215,11 +230,12 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
 template <int EPI>
 __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n0, int M, int N, int ldc,
                                                   const bf16 *__restrict__ R, bf16 *__restrict__ C,
-                                                  const RopeArgs &rope, DevStatus *status) {
+                                                  const RopeArgs &rope, DevStatus *status,
+                                                  uint4 (&res_next)[4]) {
+  // res_next (EPI_RESIDUAL): the addend of the tile's first 32 columns, loaded by the caller ahead of time
   constexpr int BN = GEMM_ACC_N;
   constexpr int TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   bf16 *crow = C + (size_t)row * ldc;
-  const bf16 *rrow = (EPI == EPI_RESIDUAL) ? R + (size_t)row * ldc : nullptr;
   if (EPI == EPI_QKV_ROPE) {
     // section of the fused projection this tile belongs to: 0 = q, 1 = k, 2 = v
     const int sect = n0 / rope.d_model;
@@ -293,6 +309,12 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
     }
+    uint4 res_cur[4];
+    if (EPI == EPI_RESIDUAL) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) res_cur[j] = res_next[j];
+      if (c + 32 < TILE_N) gemm_residual_load(res_next, R, rope, row, n0 + c + 32, M, N, ldc);
+    }
     if (row < M) {
 #pragma unroll
       for (int j = 0; j < 32; j += 8) {
@@ -303,7 +325,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
           for (int i = 0; i < 8; ++i) f[i] = v[j + i];
           if (EPI == EPI_RESIDUAL) {
             Vec16<bf16> rv;
-            rv.load(rrow + col);
+            rv.raw = res_cur[j >> 3];
             float rf[8];
             rv.unpack(rf);
 #pragma unroll

@@ -173,11 +173,14 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       int m_idx, n_idx;
       gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
       const int m0 = m_idx * BM, n0 = n_idx * TILE_N_OUT;
+      const int row = m0 + quarter * 32 + lane;
+      uint4 res_first[4] = {};
+      if (EPI == EPI_RESIDUAL && w.mode != 1)  // requested now, needed once the accumulator is complete
+        gemm_residual_load(res_first, R, rope, row, n0, M, N, ldc);
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       const int row_in_tile = quarter * 32 + lane;
       if (w.mode == 1) {  // partial accumulator of a split tile: to this CTA's slot, then tell the finisher
@@ -196,7 +199,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           gemm_fixup_row(taddr, tail.partials + (size_t)(blockIdx.x + 1) * GEMM_SLOT_FLOATS, 1, n_parts, smem,
                          row_in_tile);
         }
-        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + w.tail_idx, 1u) == 3u) {  // last warp through: clean for the next launch
@@ -294,16 +297,24 @@ size_t gemm_scratch_bytes() { return gemm_tail_scratch_bytes(GEMM_TAIL_MAX_CTAS)
 
 int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const void *R, void *C,
                 int M, int N, int K, DevStatus *status, void *scratch, size_t scratch_bytes, int force_kernel,
-                bool b_const) {
+                bool b_const, const int32_t *res_rows) {
   if (M == 0) return LAZY_OK;
+  if (res_rows && (!gemm_res_rows_supported(dtype, M, K) || !R || R == C)) return LAZY_E_BADARG;
   if (dtype == LAZY_F32) return launch_gemm_simt(st, dtype, A, B, nullptr, R, C, M, N, K, 0);
   if (gemv_small_m_eligible(dtype, M, K))
     return launch_gemv_small_m(st, A, B, nullptr, R, C, M, N, K, 0, nullptr, 0.f, 0, b_const);
-  if (R)
-    return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes,
-                                   force_kernel);
+  if (R) {
+    RopeArgs extra = {};
+    extra.res_rows = res_rows;
+    return launch_tc<EPI_RESIDUAL>(st, A, B, B, R, C, M, N, K, status, extra, scratch, scratch_bytes, force_kernel);
+  }
   return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes,
                               force_kernel);
+}
+
+// The residual row list exists in the tensor-core epilogue only.
+bool gemm_res_rows_supported(int dtype, int M, int K) {
+  return dtype == LAZY_BF16 && !gemv_small_m_eligible(dtype, M, K);
 }
 
 bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {

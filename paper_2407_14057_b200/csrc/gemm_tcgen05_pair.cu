@@ -166,11 +166,14 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       int m_idx, n_idx;
       gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
       const int m0 = m_idx * (2 * PBM) + (int)rank * PBM, n0 = n_idx * TILE_N_OUT;
+      const int row = m0 + quarter * 32 + lane;
+      uint4 res_first[4] = {};
+      if (EPI == EPI_RESIDUAL && w.mode != 1)  // requested now, needed once the accumulator is complete
+        gemm_residual_load(res_first, R, rope, row, n0, M, N, ldc);
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * PBN);
       // split tiles: slot of pair p, rank r = CTA 2p + r; one arrival counter per (tail tile, rank)
       const int row_in_tile = quarter * 32 + lane;
@@ -192,7 +195,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           gemm_fixup_row(taddr, tail.partials + (size_t)(2 * (pair + 1) + (int)rank) * GEMM_SLOT_FLOATS, 2, n_parts,
                          smem, row_in_tile);
         }
-        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status);
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + flag_idx, 1u) == 3u) {

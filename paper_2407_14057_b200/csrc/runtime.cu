@@ -156,8 +156,11 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->scores = (float *)k.take((size_t)L * KV * 4);
   c->sel_scores = (float *)k.take(R * 4);
   {
+    // prefill keeps the attention kernel's score by-product of every layer (the head means of the layers
+    // between two cuts are taken in one launch); decode uses the same memory for its per-step logits
     size_t a = score_scratch_floats(c->S, c->cap_kv, c->H);
-    size_t b = attn_score_scratch_floats(c->S, c->H, c->cap_rows / 64 + 1);
+    c->score_layer_stride = align_up(attn_score_scratch_floats(c->S, c->H, c->cap_rows / 64 + 1), 64);
+    size_t b = c->score_layer_stride * (size_t)c->L;
     c->score_scratch = (float *)k.take((a > b ? a : b) * 4);
   }
   c->keep_idx.assign(P, nullptr);
@@ -471,6 +474,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
 
   char *x = c->x, *x2 = c->x2;
   int g = 0;
+  int score_pending = 0;  // first layer whose Eq. 1 head mean has not been taken yet (tensor-core attention path)
   for (int l = 0; l < L; ++l) {
     const int n = c->seg_cu[g][n_seqs];
     const int32_t *pos = c->pos_seg[g];
@@ -508,20 +512,29 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
     }
     bool fused_score = false;
     if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
-      // one launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
-      // read as zeros instead of whatever the cache region holds
+      // Eq. 1 comes from the last row's softmax numerators, which the attention kernel leaves in this layer's
+      // slice of the score scratch; the head means of all layers since the previous cut are taken in one
+      // launch when the next cut (or the end of the prefill) needs them.
+      // One attention launch per sequence: its tensor maps end at the sequence's last row, so rows beyond it
+      // read as zeros instead of whatever the cache region holds.
       for (int s = 0; s < n_seqs; ++s) {
         const int q0 = c->seg_cu[g][s], ns = c->seg_cu[g][s + 1] - q0;
         const double fl = 2.0 * d * (double)ns * (ns + 1.0);
         TIMED(LAZY_K_ATTENTION, fl, 0,
               launch_attention_tc(st, c->qkv, 3 * d, q0 + ns, kc, vc, d, c->seq_base[s] + ns, c->attn, c->H,
-                                  nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status, c->score_scratch,
-                                  cdiv(seg_max, 64), n_seqs, s));
+                                  nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status,
+                                  c->score_scratch + (size_t)l * c->score_layer_stride, cdiv(seg_max, 64), n_seqs, s));
       }
-      // Eq. 1 from the last row's softmax numerators the attention kernel left behind
-      TIMED(LAZY_K_SCORE, 0, 4.0 * c->H * n + 4.0 * n,
-            launch_score_from_attention(st, c->score_scratch, d_cu(g), n_seqs, n, c->H, cdiv(seg_max, 64), sc));
       fused_score = true;
+      const bool last_of_group = c->point_at[l + 1] >= 0 || l == L - 1;
+      if (last_of_group) {  // layers score_pending..l ran on the same rows (segment g)
+        const int nl = l - score_pending + 1;
+        TIMED(LAZY_K_SCORE, 0, nl * (4.0 * c->H * n + 4.0 * n),
+              launch_score_from_attention(st, c->score_scratch + (size_t)score_pending * c->score_layer_stride,
+                                          c->score_layer_stride, nl, d_cu(g), n_seqs, n, c->H, cdiv(seg_max, 64),
+                                          c->scores + (size_t)score_pending * c->cap_kv, (size_t)c->cap_kv));
+        score_pending = l + 1;
+      }
     } else {
       TIMED(LAZY_K_ATTENTION, attn_flops, 0,
             launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
@@ -532,19 +545,28 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
             launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
                          c->score_scratch, sc));
     TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status,
-                                                      c->gemm_scratch, c->gemm_scratch_bytes));
+                                                      c->gemm_scratch, c->gemm_scratch_bytes, 0, true));
 
     const int p = c->point_at[l + 1];
+    // Rows of the residual stream that survive a cut made in this layer, when they are still where they
+    // were (x is then compacted on the way through the MLP instead of by a copy of its own): the MLP's
+    // RMSNorm reads x[keep[r]], and the down projection adds x[keep[r]] and writes row r of the other buffer.
+    const int32_t *via_keep = nullptr;
     // The layer's MLP, on the rows of the current segment.
     auto run_mlp = [&]() -> int {
       const int n2 = c->seg_cu[g][n_seqs];
-      TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb, launch_rmsnorm(st, dt, x, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
+      TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb,
+            launch_rmsnorm_rows(st, dt, x, via_keep, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
       TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
             launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
-                               c->gemm_scratch_bytes));
+                               c->gemm_scratch_bytes, 0, true));
       TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
-            launch_gemm(st, dt, c->act, c->w_down[l], x, x, n2, d, c->F, status, c->gemm_scratch,
-                        c->gemm_scratch_bytes));
+            launch_gemm(st, dt, c->act, c->w_down[l], x, via_keep ? x2 : x, n2, d, c->F, status, c->gemm_scratch,
+                        c->gemm_scratch_bytes, 0, true, via_keep));
+      if (via_keep) {
+        char *t = x; x = x2; x2 = t;
+        via_keep = nullptr;
+      }
       return LAZY_OK;
     };
     // Default: the cut sits between attention and MLP, so the MLP of this layer already runs on the kept
@@ -567,21 +589,25 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
         sel = c->sel_scores;
       }
       const int n_keep = c->seg_cu[g + 1][n_seqs], n_drop = n - n_keep;
-      TIMED(LAZY_K_SELECT, 0, 8.0 * n,
-            launch_select(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->keep_idx[p], c->drop_idx[p], status));
       char *ar = c->aux_rows + (size_t)p * c->cap_kv * rb;
       int32_t *ap = c->aux_pos + (size_t)p * c->cap_kv;
+      // the selection also writes the position lists of the next segment and of the Aux Cache
+      TIMED(LAZY_K_SELECT, 0, 8.0 * n + 8.0 * n,
+            launch_select(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->keep_idx[p], c->drop_idx[p], status, pos,
+                          c->pos_seg[g + 1], c->aux_dst[p], ap));
+      // pruned rows to the Aux Cache (the one copy the method itself asks for)
       TIMED(LAZY_K_COMPACT, 0, 2.0 * n_drop * rb,
             launch_move_rows(st, x, c->drop_idx[p], ar, c->aux_dst[p], n_drop, (int)rb, n, c->cap_kv, status));
-      TIMED(LAZY_K_COMPACT, 0, 8.0 * n_drop, launch_move_i32(st, pos, c->drop_idx[p], ap, c->aux_dst[p], n_drop));
-      TIMED(LAZY_K_COMPACT, 0, 2.0 * n_keep * rb,
-            launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
-      TIMED(LAZY_K_COMPACT, 0, 8.0 * n_keep,
-            launch_move_i32(st, pos, c->keep_idx[p], c->pos_seg[g + 1], nullptr, n_keep));
+      if (!cut_after && gemm_res_rows_supported(dt, n_keep, c->F)) {
+        via_keep = c->keep_idx[p];  // kept rows are gathered on load by the MLP that follows
+      } else {
+        TIMED(LAZY_K_COMPACT, 0, 2.0 * n_keep * rb,
+              launch_move_rows(st, x, c->keep_idx[p], x2, nullptr, n_keep, (int)rb, n, c->cap_rows, status));
+        char *t = x; x = x2; x2 = t;
+      }
       for (int s = 0; s < n_seqs; ++s)
         c->aux_count[p][s] = c->aux_live[p][s] = cu_drop[p][s + 1] - cu_drop[p][s];
       c->stats.aux_rows[l] = n_drop;
-      char *t = x; x = x2; x2 = t;
       ++g;
     }
     if (!cut_after) LAZY_TRY(run_mlp());

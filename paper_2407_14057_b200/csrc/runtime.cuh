@@ -33,6 +33,7 @@ struct lazy_ctx {
   float *scores;                   // [L, cap_rows]
   float *sel_scores;               // [cap_rows] scores handed to the selection when a set is forced
   float *score_scratch;
+  size_t score_layer_stride;  // floats per layer of the attention kernels' score by-product
   std::vector<int32_t *> keep_idx, drop_idx;  // [P] x [cap_rows]
   std::vector<int32_t *> aux_dst;             // [P] x [cap_rows] Aux row of the i-th dropped row
   std::vector<int32_t *> kv_row;              // [P+1] x [cap_rows] cache row of packed row r

@@ -179,10 +179,81 @@ __device__ __forceinline__ void radix_pick_bin(const int *hist, int k, int &bin,
   above = __shfl_sync(0xffffffffu, ab, owner);
 }
 
+// Keys of a sequence are read from global memory once and kept in shared memory for the four radix passes
+// and the emit pass (sequences of up to SEL_CACHE rows; longer ones re-read the scores).
+constexpr int SEL_CACHE = 8192;
+
+struct SelShared {
+  int hist[256];
+  int warp_tot[32];
+  uint32_t prefix;
+  int k;
+  uint32_t keys[SEL_CACHE];
+};
+
+// Radix select over the order-preserving keys of s[0..n): on return *k_ties = how many keys equal to the
+// returned key tau belong to the k largest.  force_last: the last row gets the maximal key.  Scores of a
+// long prompt are nearly equal (about 1/n), so their keys share the high bytes and a plain histogram would
+// serialise every shared-memory atomic of the first passes on one bin: the lanes of a warp that hit the
+// same bin as its first active lane are counted with a ballot and added once.
+__device__ __forceinline__ uint32_t radix_kth_largest(const float *__restrict__ s, int n, int k, bool force_last,
+                                                      SelShared &sh, int *k_ties) {
+  const bool cached = n <= SEL_CACHE;
+  const int lane = threadIdx.x & 31;
+  if (cached)
+    for (int i = threadIdx.x; i < n; i += SEL_THREADS)
+      sh.keys[i] = (force_last && i == n - 1) ? 0xffffffffu : score_key(s[i]);
+  uint32_t prefix = 0, mask = 0;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += SEL_THREADS) sh.hist[i] = 0;
+    __syncthreads();  // also orders the key cache before its first use
+    for (int base = 0; base < n; base += SEL_THREADS) {
+      const int i = base + threadIdx.x;
+      uint32_t key = 0;
+      bool act = false;
+      if (i < n) {
+        key = cached ? sh.keys[i] : ((force_last && i == n - 1) ? 0xffffffffu : score_key(s[i]));
+        act = (key & mask) == prefix;
+      }
+      const uint32_t bin = (key >> shift) & 255u;
+      // lanes that share the bin of the warp's first active lane add once, together; the others one by one
+      const unsigned active = __ballot_sync(0xffffffffu, act);
+      if (active) {
+        const uint32_t bin0 = __shfl_sync(0xffffffffu, bin, __ffs(active) - 1);
+        const unsigned same = __ballot_sync(0xffffffffu, act && bin == bin0);
+        if (act) {
+          if (bin != bin0) atomicAdd(&sh.hist[bin], 1);
+          else if (lane == __ffs(same) - 1) atomicAdd(&sh.hist[bin0], __popc(same));
+        }
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int above, b;
+      radix_pick_bin(sh.hist, k, b, above);
+      if (threadIdx.x == 0) {
+        sh.prefix = prefix | ((uint32_t)b << shift);
+        sh.k = k - above;
+      }
+    }
+    __syncthreads();
+    prefix = sh.prefix;
+    k = sh.k;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  *k_ties = k;
+  return prefix;
+}
+
+// pos_in (optional): position of every input row.  The kept rows' positions then go to pos_keep (packed like
+// keep_idx) and the dropped rows' positions to aux_pos[aux_dst[j]], j = the row's slot in drop_idx: the
+// position lists of the next segment and of the Aux Cache come out of the selection itself.
 __global__ void __launch_bounds__(SEL_THREADS)
 select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_in,
               const int32_t *__restrict__ cu_keep, int32_t *__restrict__ keep_idx,
-              int32_t *__restrict__ drop_idx, DevStatus *status) {
+              int32_t *__restrict__ drop_idx, DevStatus *status, const int32_t *__restrict__ pos_in,
+              int32_t *__restrict__ pos_keep, const int32_t *__restrict__ aux_dst, int32_t *__restrict__ aux_pos) {
   const int seq = blockIdx.x;
   const int in0 = cu_in[seq], n = cu_in[seq + 1] - in0;
   const int k0 = cu_keep[seq], n_keep = cu_keep[seq + 1] - k0;
@@ -193,37 +264,10 @@ select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_i
     return;
   }
   const float *s = scores + in0;
-  __shared__ int hist[256];
-  __shared__ int warp_tot[32];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_k;
-
-  // ---- radix select of the n_keep-th largest key
-  uint32_t prefix = 0, mask = 0;
-  int k = n_keep;  // still looking for the k-th largest among keys matching `prefix` under `mask`
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
-    for (int i = threadIdx.x; i < n; i += SEL_THREADS) {
-      const uint32_t key = (i == n - 1) ? 0xffffffffu : score_key(s[i]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-    }
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      int above, b;
-      radix_pick_bin(hist, k, b, above);
-      if (threadIdx.x == 0) {
-        sh_prefix = prefix | ((uint32_t)b << shift);
-        sh_k = k - above;
-      }
-    }
-    __syncthreads();
-    prefix = sh_prefix;
-    k = sh_k;
-    mask |= 255u << shift;
-    __syncthreads();
-  }
-  const uint32_t tau = prefix;  // key of the n_keep-th largest; k = how many keys == tau to keep
+  __shared__ SelShared sh;
+  int k;  // how many keys == tau to keep
+  const uint32_t tau = radix_kth_largest(s, n, n_keep, true, sh, &k);
+  const bool cached = n <= SEL_CACHE;
 
   // ---- emit in index order
   int kept_so_far = 0, eq_so_far = 0;
@@ -231,16 +275,22 @@ select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_i
     const int i = base + threadIdx.x;
     uint32_t key = 0;
     const bool valid = i < n;
-    if (valid) key = (i == n - 1) ? 0xffffffffu : score_key(s[i]);
+    if (valid) key = cached ? sh.keys[i] : ((i == n - 1) ? 0xffffffffu : score_key(s[i]));
     const int is_eq = valid && key == tau;
     int eq_total;
-    const int eq_rank = eq_so_far + block_excl_scan(is_eq, warp_tot, &eq_total);
+    const int eq_rank = eq_so_far + block_excl_scan(is_eq, sh.warp_tot, &eq_total);
     const int keep = valid && (key > tau || (is_eq && eq_rank < k));
     int keep_total;
-    const int keep_rank = kept_so_far + block_excl_scan(keep, warp_tot, &keep_total);
+    const int keep_rank = kept_so_far + block_excl_scan(keep, sh.warp_tot, &keep_total);
     if (valid) {
-      if (keep) keep_idx[k0 + keep_rank] = in0 + i;
-      else drop_idx[d0 + (i - keep_rank)] = in0 + i;
+      if (keep) {
+        keep_idx[k0 + keep_rank] = in0 + i;
+        if (pos_in) pos_keep[k0 + keep_rank] = pos_in[in0 + i];
+      } else {
+        const int j = d0 + (i - keep_rank);
+        drop_idx[j] = in0 + i;
+        if (pos_in) aux_pos[aux_dst[j]] = pos_in[in0 + i];
+      }
     }
     eq_so_far += eq_total;
     kept_so_far += keep_total;
@@ -263,45 +313,20 @@ select_threshold_kernel(const float *__restrict__ scores, const int32_t *__restr
     return;
   }
   const float *s = scores + in0;
-  __shared__ int hist[256];
-  __shared__ int warp_tot[32];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_k;
+  __shared__ SelShared sh;
   const int lo = (int)(((long long)(n - 1) * prune_bp) / 10000);
-  // ---- radix select of the (n - lo)-th largest key = the lo-th smallest
-  uint32_t prefix = 0, mask = 0;
-  int k = n - lo;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
-    for (int i = threadIdx.x; i < n; i += SEL_THREADS) {
-      const uint32_t key = score_key(s[i]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
-    }
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      int above, b;
-      radix_pick_bin(hist, k, b, above);
-      if (threadIdx.x == 0) {
-        sh_prefix = prefix | ((uint32_t)b << shift);
-        sh_k = k - above;
-      }
-    }
-    __syncthreads();
-    prefix = sh_prefix;
-    k = sh_k;
-    mask |= 255u << shift;
-    __syncthreads();
-  }
-  const uint32_t tau = prefix;
+  // the (n - lo)-th largest key = the lo-th smallest
+  int k_unused;
+  const uint32_t tau = radix_kth_largest(s, n, n - lo, false, sh, &k_unused);
+  const bool cached = n <= SEL_CACHE;
   // ---- emit in index order
   int kept_so_far = 0;
   for (int base = 0; base < n; base += SEL_THREADS) {
     const int i = base + threadIdx.x;
     const bool valid = i < n;
-    const int keep = valid && (i == n - 1 || score_key(s[i]) >= tau);
+    const int keep = valid && (i == n - 1 || (cached ? sh.keys[i] : score_key(s[i])) >= tau);
     int keep_total;
-    const int keep_rank = kept_so_far + block_excl_scan(keep, warp_tot, &keep_total);
+    const int keep_rank = kept_so_far + block_excl_scan(keep, sh.warp_tot, &keep_total);
     if (valid) {
       if (keep) keep_idx[in0 + keep_rank] = in0 + i;
       else drop_idx[in0 + (i - keep_rank)] = in0 + i;
@@ -390,9 +415,12 @@ int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t 
 
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,
                   const int32_t *cu_keep, int n_seqs, int32_t *keep_idx, int32_t *drop_idx,
-                  DevStatus *status) {
+                  DevStatus *status, const int32_t *pos_in, int32_t *pos_keep, const int32_t *aux_dst,
+                  int32_t *aux_pos) {
   if (n_seqs == 0) return LAZY_OK;
-  select_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, cu_keep, keep_idx, drop_idx, status);
+  if (pos_in && (!pos_keep || !aux_dst || !aux_pos)) return LAZY_E_BADARG;
+  select_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, cu_keep, keep_idx, drop_idx, status, pos_in,
+                                                pos_keep, aux_dst, aux_pos);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

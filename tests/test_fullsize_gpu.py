@@ -323,10 +323,15 @@ def test_7b_varlen_batch_of_8_vs_oracle_and_vs_sequences_run_alone(model7b):
     torch.cuda.empty_cache()
     # Sequences are independent, so a member run alone must reproduce the batch.  Not bit for bit: which
     # output tiles of a GEMM get their K loop split across SMs depends on the total row count, and a split
-    # tile adds its fp32 partial sums in another order.  The comparison is therefore made cut by cut on EQUAL
-    # inputs: the solo run is handed the batch's kept sets for the earlier cuts and selects freely at cut i;
-    # the two sets may then differ only in tokens whose score lies within 3 % of the threshold (the band of
-    # the oracle tests), and with all three sets handed over the logits agree to the one-tensor tolerance.
+    # tile adds its fp32 partial sums in another order.  The comparison is therefore made cut by cut on the same
+    # token sets: the solo run is handed the batch's kept sets for the earlier cuts and selects freely at cut i.
+    # The bf16 roundings of every layer fall differently in the two runs, so the two score vectors agree to a
+    # few per cent, less well the deeper the cut (measured: differing tokens lie within 1.5 % / 3.1 % / 8.0 % of
+    # the threshold at the cuts entering layers 8 / 16 / 24, and 0.3 % / 0.8 % / 1.7 % of the kept tokens differ).
+    # The two sets may therefore differ only in tokens whose score lies within 4 % / 8 % / 16 % of the
+    # threshold, and in at most 4 % of the tokens.  With all three sets handed over, the logits are those of two
+    # bf16 runs of 32 layers whose roundings differ in places: each lies about 5e-2 from exact arithmetic (see
+    # E2E_LOGITS_GATE), they lie 3.0e-2 from each other (measured), and are held to twice the one-tensor bound.
     solo = B.LazyPrefill(shape, model7b, schedule, torch.bfloat16, 1, max(lengths))
     lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
     for s in (0, 3, 7):
@@ -344,14 +349,17 @@ def test_7b_varlen_batch_of_8_vs_oracle_and_vs_sequences_run_alone(model7b):
             tau = np.sort(sc[:-1])[::-1][len(b) - 2]
             s_of = dict(zip(cand.tolist(), sc.tolist()))
             diff = set(a.tolist()) ^ set(b.tolist())
-            for p in diff:
-                assert abs(s_of[p] - tau) <= 3e-2 * tau, (s, e, p, s_of[p], tau)
-            print(f"seq {s} cut entering layer {e}: {len(diff) // 2} of {len(b)} tokens differ (near-ties)")
+            worst = max([abs(s_of[p] - tau) / tau for p in diff], default=0.0)
+            print(f"seq {s} cut entering layer {e}: {len(diff) // 2} of {len(b)} tokens differ, all within "
+                  f"{100 * worst:.2f} % of the threshold")
+            assert worst <= (4e-2, 8e-2, 16e-2)[i] and len(diff) // 2 <= 0.04 * len(b), (s, e, worst, len(diff))
         for j, (e, _) in enumerate(schedule):
             solo.lazy_set_forced_keep(e, 0, torch.tensor(kept_batch[s][j], dtype=torch.int32).cuda())
         solo.lazy_prefill_run(p_ids, [0, lengths[s]], lg)
         solo.lazy_sync_status()
-        assert rel_err(to_np(lg[0]), to_np(logits[s]).astype(np.float64)) < TOL
+        both = rel_err(to_np(lg[0]), to_np(logits[s]).astype(np.float64))
+        print(f"seq {s} logits, batch member vs run alone on the same kept sets: {both:.4f}")
+        assert both < 2 * TOL
         # free-running, for the record: rounding noise moves ranks next to the threshold, and a different
         # set at one cut changes every later score a little
         solo.lazy_prefill_run(p_ids, [0, lengths[s]], lg)
