@@ -13,8 +13,8 @@ blocking, fusion or reordering: every attention matrix is formed explicitly.
 Readings of points the paper leaves open (all listed in the design document):
   * Eq. 1: query = the last token, key = token i, i.e. the LAST ROW of the usual
     [query, key] probability matrix, averaged over heads.
-  * The score of layer e-1 selects the set that enters layer e (Section 3.2:
-    "pruned at layer l+1" by s^l); the cut sits between attention (+ output
+  * The score of layer e-1 selects the set that enters layer e (Section 3.2: the
+    score s^l decides what the following layer still sees); the cut sits between attention (+ output
     projection + residual) and the MLP of layer e-1, so that MLP already runs on
     the kept rows only and the Aux Cache of layer e-1 holds post-attention,
     pre-MLP hidden states.  The literal alternative (cut after the whole layer, Aux
@@ -128,6 +128,41 @@ def select_top(scores: np.ndarray, n_keep: int, forced: int) -> Tuple[np.ndarray
     return np.asarray(kept, dtype=np.int64), np.asarray(dropped, dtype=np.int64)
 
 
+def select_ties_kept(scores: np.ndarray, n_keep: int, forced: int) -> Tuple[np.ndarray, np.ndarray]:
+    """The selection of Section 3.2 read as a THRESHOLD at the same percentile the count form uses.
+
+    tau = the n_keep-th largest score among the candidates, the forced candidate (the token being predicted
+    from) counting as larger than everything.  A token is pruned iff its score is smaller than tau; scores
+    equal to tau are not smaller, so every tie at the threshold is kept and the number of kept tokens
+    (>= n_keep) depends on the data.  Without ties at tau this is exactly `select_top`.
+    Returns (kept ascending, dropped ascending).
+    """
+    s = np.asarray(scores)
+    n = s.shape[0]
+    if forced < 0:
+        forced += n
+    assert 1 <= n_keep <= n
+    others = sorted((float(s[i]) for i in range(n) if i != forced), reverse=True)
+    if n_keep == 1:
+        kept = [forced]
+    else:
+        tau = others[n_keep - 2]                      # the forced token takes the first of the n_keep places
+        kept = [i for i in range(n) if i == forced or float(s[i]) >= tau]
+    drop = [i for i in range(n) if i not in set(kept)]
+    return np.asarray(kept, dtype=np.int64), np.asarray(drop, dtype=np.int64)
+
+
+SELECTIONS = ("count", "threshold")
+
+
+def _select(selection: str, scores, n_keep: int, forced: int):
+    if selection == "count":
+        return select_top(scores, n_keep, forced)
+    if selection == "threshold":
+        return select_ties_kept(scores, n_keep, forced)
+    raise ValueError(f"selection must be one of {SELECTIONS}")
+
+
 # --------------------------------------------------------------------------- model pieces
 def select_threshold(scores: np.ndarray, prune_bp: int) -> Tuple[np.ndarray, np.ndarray]:
     """The selection of Section 3.2 read as a threshold: a token is pruned if its score is smaller than
@@ -210,11 +245,14 @@ class LayerCache:
 class LazyState:
     """Everything one sequence carries from prefill into decode, plus per-call records."""
 
-    def __init__(self, cfg, schedule, aux_point: str = "pre_mlp"):
+    def __init__(self, cfg, schedule, aux_point: str = "pre_mlp", selection: str = "count"):
         if aux_point not in AUX_POINTS:
             raise ValueError(f"aux_point must be one of {AUX_POINTS}")
+        if selection not in SELECTIONS:
+            raise ValueError(f"selection must be one of {SELECTIONS}")
         self.cfg = cfg
         self.aux_point = aux_point
+        self.selection = selection
         self.schedule = {int(e): int(bp) for e, bp in schedule}
         self.layers = [LayerCache() for _ in range(cfg.n_layers)]
         self.n_tokens = 0                      # tokens seen so far (prompt + generated)
@@ -253,16 +291,19 @@ def validate_schedule(cfg, schedule) -> None:
 
 # --------------------------------------------------------------------------- prefill
 def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]]] = None,
-            keep_records: bool = True, aux_point: str = "pre_mlp") -> LazyState:
+            keep_records: bool = True, aux_point: str = "pre_mlp", selection: str = "count") -> LazyState:
     """Token-pruned prefill of one prompt (Sections 3.1 and 3.2).
 
     ids: [N] token ids.  schedule: iterable of (layer_entered, cumulative keep in basis
     points of N); layer 0 always sees the whole prompt.  forced_keep: optional
     {layer_entered: kept positions} that replaces the score-based selection at that
     point (used to replay another implementation's kept sets).  aux_point: see AUX_POINTS.
+    selection: "count" keeps exactly the scheduled number of tokens (ties to the lower position);
+    "threshold" prunes a token iff its score is smaller than the score at that rank, so ties at the
+    threshold all survive and later layers may see more rows than scheduled.
     """
     validate_schedule(cfg, schedule)
-    st = LazyState(cfg, schedule, aux_point)
+    st = LazyState(cfg, schedule, aux_point, selection)
     ids = np.asarray(ids).astype(np.int64)
     N = ids.shape[0]
     st.n_tokens = N
@@ -290,7 +331,7 @@ def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]
                 keep = np.asarray([r for r in range(n) if int(pos[r]) in want], dtype=np.int64)
                 drop = np.asarray([r for r in range(n) if int(pos[r]) not in want], dtype=np.int64)
             else:
-                keep, drop = select_top(s, keep_count(N, st.schedule[l + 1], n), n - 1)
+                keep, drop = _select(selection, s, keep_count(N, st.schedule[l + 1], n), n - 1)
             st.kept_pos[l + 1] = pos[keep].copy()
             st.dropped_pos[l + 1] = pos[drop].copy()
         if cut and aux_point == "pre_mlp":
@@ -396,7 +437,7 @@ def decode_step(cfg, W, st: LazyState, token_id: int,
                 keep = np.asarray([i for i in range(len(ctx)) if int(ctx[i]) in want], dtype=np.int64)
             else:
                 n_keep = keep_count(p + 1, st.schedule[l + 1], len(ctx))
-                keep, _ = select_top(s, n_keep, len(ctx) - 1)
+                keep, _ = _select(st.selection, s, n_keep, len(ctx) - 1)
             sel = ctx[keep]                           # includes p
             sel_set = set(int(t) for t in sel)
             for r in list(X.keys()):                  # in flight but not selected any more

@@ -517,3 +517,75 @@ def test_prune_op_agrees_with_prefill_first_layer():
     assert np.array_equal(r["hidden_attn"], st.hidden_after_attn[0])
     assert sorted(st.layers[0].aux.keys()) == r["aux_pos"].tolist()
     assert np.array_equal(r["k_kept"][0], st.layers[0].kv[int(r["pos_kept"][0])][0])
+
+
+# ----------------------------------------------------------------------------- threshold reading, ties kept
+def test_select_ties_kept_hand_worked():
+    """Worked by hand from the definition: tau = the n_keep-th largest score with the forced (last) token
+    counted as the largest; pruned iff score < tau."""
+    s = np.array([0.30, 0.10, 0.10, 0.05, 0.10, 0.02], dtype=np.float32)   # forced = index 5
+    # n_keep = 3: places go to {5 (forced), 0.30, 0.10}; tau = 0.10; the three 0.10s all survive
+    keep, drop = O.select_ties_kept(s, 3, 5)
+    assert keep.tolist() == [0, 1, 2, 4, 5] and drop.tolist() == [3]
+    # the count form keeps exactly three, the tie going to the lower index
+    k2, d2 = O.select_top(s, 3, 5)
+    assert k2.tolist() == [0, 1, 5] and d2.tolist() == [2, 3, 4]
+    # n_keep = 2: tau = 0.30, no tie: both forms agree
+    assert O.select_ties_kept(s, 2, 5)[0].tolist() == O.select_top(s, 2, 5)[0].tolist() == [0, 5]
+    # n_keep = 1: only the forced token
+    assert O.select_ties_kept(s, 1, 5)[0].tolist() == [5]
+    # everything equal: nothing is smaller than tau, nothing is pruned
+    u = np.full(7, 1.0 / 7, dtype=np.float32)
+    assert O.select_ties_kept(u, 3, 6)[0].tolist() == list(range(7))
+    # the forced token's own score does not move the threshold (here it would be the largest)
+    t = np.array([0.1, 0.2, 0.3, 0.9], dtype=np.float32)
+    assert O.select_ties_kept(t, 2, 3)[0].tolist() == [2, 3]
+
+
+def test_select_ties_kept_equals_count_form_without_ties_and_brute_force_with():
+    rng = np.random.default_rng(31)
+    for n in (1, 2, 5, 64, 257):
+        s = rng.permutation(n).astype(np.float32)          # all distinct
+        for n_keep in sorted({1, max(1, n // 3), n}):
+            a = O.select_ties_kept(s, n_keep, n - 1)
+            b = O.select_top(s, n_keep, n - 1)
+            assert a[0].tolist() == b[0].tolist() and a[1].tolist() == b[1].tolist()
+    for _ in range(50):                                     # few levels: ties everywhere
+        n = int(rng.integers(2, 40))
+        s = rng.integers(0, 4, n).astype(np.float32)
+        n_keep = int(rng.integers(1, n + 1))
+        keep, drop = O.select_ties_kept(s, n_keep, n - 1)
+        k_top, _ = O.select_top(s, n_keep, n - 1)
+        assert set(k_top.tolist()) <= set(keep.tolist()) and len(keep) >= n_keep     # a superset of the count form
+        if len(drop):
+            tau = min(float(s[i]) for i in keep if i != n - 1) if len(keep) > 1 else np.inf
+            assert all(float(s[i]) < tau for i in drop)                              # pruned iff strictly smaller
+        assert sorted(keep.tolist() + drop.tolist()) == list(range(n))
+
+
+def test_threshold_prefill_equals_count_prefill_without_ties_and_keeps_all_ties():
+    """Generic inputs have no ties: both readings give the same run.  A layer whose query projection is zero
+    attends uniformly (closed form s_j = 1/n), every score ties, and the threshold reading prunes nothing
+    there while the count reading prunes down to the schedule."""
+    shape = MINI
+    W = weights_to_np(mini_weights(seed=29))
+    ids = to_np(synth.make_prompt(shape.vocab, 30, seed=29))
+    sched = ((1, 6000), (2, 3000))
+    a = O.prefill(shape, W, ids, sched, selection="count")
+    b = O.prefill(shape, W, ids, sched, selection="threshold")
+    assert all(np.array_equal(a.kept_pos[e], b.kept_pos[e]) for e, _ in sched)
+    assert np.array_equal(a.logits, b.logits)
+    d = shape.d_model
+    W["layers"][0] = dict(W["layers"][0])
+    wq = np.array(W["layers"][0]["w_qkv"], copy=True)
+    wq[:d] = 0.0                                           # q = 0 in layer 0: uniform attention rows
+    W["layers"][0]["w_qkv"] = wq
+    c = O.prefill(shape, W, ids, sched, selection="count")
+    t = O.prefill(shape, W, ids, sched, selection="threshold")
+    assert np.allclose(t.scores[0], 1.0 / 30) and len(np.unique(t.scores[0])) == 1
+    assert len(c.kept_pos[1]) == 18 and len(t.kept_pos[1]) == 30          # nothing is smaller than tau
+    assert len(t.kept_pos[2]) == O.keep_count(30, 3000, 30) == 9           # the next cut has no ties again
+    assert len(t.layers[0].aux) == 0 and len(c.layers[0].aux) == 12
+    # decode keeps using the state's reading
+    assert t.selection == "threshold"
+    O.decode_step(shape, W, t, O.greedy(t.logits))
