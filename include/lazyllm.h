@@ -211,6 +211,15 @@ int lazy_get_kernel_times(lazy_ctx *ctx, void *stream, lazy_kernel_times *out);
  * number of surviving rows (the row count follows from the work: flops / flops per row). */
 int lazy_get_kernel_events(lazy_ctx *ctx, void *stream, int32_t cap, int32_t *kinds, float *ms, double *flops,
                            double *bytes, int32_t *count);
+/* How the scheduled percentile selects (Section 3.2, token pruning).  mode 0 (default): as a count, exactly
+ * lazy_keep_count() tokens survive a point, ties going to the lower position, so every row count follows
+ * from lengths and schedule and lazy_prefill_run never synchronises.  mode 1: as a threshold, a token is
+ * pruned iff its score is smaller than the score at that rank (the last token counting as the largest), so
+ * tokens tied with the threshold all survive and later layers may see more rows than scheduled; the kept
+ * count of every sequence is then read back from the device at each point (one stream synchronisation per
+ * point in lazy_prefill_run, one more per point in lazy_decode_step).  Without ties both modes select the
+ * same sets.  Takes effect with the next lazy_prefill_run / lazy_decode_step. */
+int lazy_set_selection(lazy_ctx *ctx, int32_t mode);
 /* Where the scoring layer is cut (Section 3.2, Aux Cache paragraph).  after_layer = 0 (default): between
  * the layer's attention half and its MLP, so that MLP already runs on the kept rows, the Aux Cache holds
  * post-attention hidden states and a revived token first gets that layer's MLP.  after_layer = 1: after

@@ -99,6 +99,7 @@ _SIGNATURES = {
     "lazy_k_gemm": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
     "lazy_k_gemm_swiglu": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
     "lazy_set_aux_point": (_I, [_P, _I]),
+    "lazy_set_selection": (_I, [_P, _I]),
     "lazy_k_gemm_scratch_bytes": (_Z, []),
     "lazy_k_gemm_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
     "lazy_k_gemm_swiglu_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
@@ -262,6 +263,9 @@ class LazyPrefill:
 
     def lazy_set_aux_point(self, after_layer: bool) -> None:
         _check("lazy_set_aux_point", lib().lazy_set_aux_point(self.ctx, 1 if after_layer else 0))
+
+    def lazy_set_selection(self, threshold: bool) -> None:
+        _check("lazy_set_selection", lib().lazy_set_selection(self.ctx, 1 if threshold else 0))
 
     def lazy_get_hidden(self, layer: int) -> torch.Tensor:
         rows = C.c_int32()

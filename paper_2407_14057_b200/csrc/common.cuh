@@ -287,6 +287,10 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
                     int head_dim, float *scratch, float *scores);
 int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t *cu_in, int n_seqs,
                             uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts);
+// counts[s] = rows of sequence s whose score is not smaller than its (cu_keep[s+1] - cu_keep[s])-th largest
+// score, the last row counting as the largest: the kept count of the threshold reading (ties all kept).
+int launch_select_tie_count(cudaStream_t st, const float *scores, const int32_t *cu_in, const int32_t *cu_keep,
+                            int n_seqs, int32_t *counts, DevStatus *status);
 // With pos_in (position of every input row) the kernel also writes the kept rows' positions to pos_keep
 // (packed like keep_idx) and the dropped rows' positions to aux_pos[aux_dst[j]] (j = slot in drop_idx).
 int launch_select(cudaStream_t st, const float *scores, const int32_t *cu_in,

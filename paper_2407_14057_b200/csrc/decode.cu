@@ -434,6 +434,19 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
         }
         sel = scores_sel;
       }
+      if (c->select_threshold) {
+        // threshold reading: ties at the scheduled rank all survive; the counts come back from the device
+        // (one more stream synchronisation at this boundary)
+        LAZY_TRY(launch_select_tie_count(st, sel, dtab(T_CU_CTX), dtab(T_CU_KEEP), S, dtab(T_COUNTS), status));
+        LAZY_CUDA_OK(cudaMemcpyAsync(tab(T_COUNTS), dtab(T_COUNTS), (size_t)S * 4, cudaMemcpyDeviceToHost, st));
+        LAZY_CUDA_OK(cudaStreamSynchronize(st));
+        for (int s = 0; s < S; ++s) {
+          const int keep = tab(T_COUNTS)[s];
+          if (keep < 1 || keep > ctx_n[s]) return LAZY_E_STATE;
+          tab(T_CU_KEEP)[s + 1] = tab(T_CU_KEEP)[s] + keep;
+        }
+        LAZY_TRY(upload(T_CU_KEEP));
+      }
       LAZY_TRY(launch_select(st, sel, dtab(T_CU_CTX), dtab(T_CU_KEEP), S, keep_idx, drop_idx, status));
       const int n_keep = tab(T_CU_KEEP)[S];
       LAZY_TRY(launch_move_i32(st, ctx_pos, keep_idx, ctx_pos2, nullptr, n_keep));

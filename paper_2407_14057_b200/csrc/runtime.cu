@@ -337,6 +337,12 @@ int32_t lazy_keep_count(int32_t n_total, uint32_t keep_bp, int32_t n_present) {
   return keep_count(n_total, keep_bp, n_present);
 }
 
+int lazy_set_selection(lazy_ctx *c, int32_t mode) {
+  if (!c || (mode != 0 && mode != 1)) return LAZY_E_BADARG;
+  c->select_threshold = mode == 1;
+  return LAZY_OK;
+}
+
 int lazy_set_aux_point(lazy_ctx *c, int32_t after_layer) {
   if (!c || (after_layer != 0 && after_layer != 1)) return LAZY_E_BADARG;
   if (c->aux_after_layer != (after_layer != 0)) {
@@ -424,19 +430,25 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   c->seg_cu.assign(P + 1, std::vector<int>(n_seqs + 1, 0));
   for (int s = 0; s <= n_seqs; ++s) c->seg_cu[0][s] = h_cu_seqlens[s];
   std::vector<std::vector<int>> cu_drop(P, std::vector<int>(n_seqs + 1, 0));
-  for (int p = 0; p < P; ++p) {
-    for (int s = 0; s < n_seqs; ++s) {
-      const int present = c->seg_cu[p][s + 1] - c->seg_cu[p][s];
-      int keep = keep_count(c->prompt_len[s], c->sched_bp[p], present);
-      auto it = c->forced.find(std::make_pair(p, s));
-      if (it != c->forced.end()) {
-        keep = it->second.second;
-        if (keep < 1 || keep > present) return LAZY_E_BADARG;
+  // Rows kept at points p_from.. from the rows present at p_from (count form: the scheduled count; under the
+  // threshold reading these are the counts before ties, corrected point by point once the scores exist).
+  auto plan_from = [&](int p_from) -> int {
+    for (int p = p_from; p < P; ++p) {
+      for (int s = 0; s < n_seqs; ++s) {
+        const int present = c->seg_cu[p][s + 1] - c->seg_cu[p][s];
+        int keep = keep_count(c->prompt_len[s], c->sched_bp[p], present);
+        auto it = c->forced.find(std::make_pair(p, s));
+        if (it != c->forced.end()) {
+          keep = it->second.second;
+          if (keep < 1 || keep > present) return LAZY_E_BADARG;
+        }
+        c->seg_cu[p + 1][s + 1] = c->seg_cu[p + 1][s] + keep;
+        cu_drop[p][s + 1] = cu_drop[p][s] + (present - keep);
       }
-      c->seg_cu[p + 1][s + 1] = c->seg_cu[p + 1][s] + keep;
-      cu_drop[p][s + 1] = cu_drop[p][s] + (present - keep);
     }
-  }
+    return LAZY_OK;
+  };
+  LAZY_TRY(plan_from(0));
   c->kv_count.assign(L, std::vector<int>(n_seqs, 0));
   c->aux_count.assign(P, std::vector<int>(n_seqs, 0));
   c->aux_live.assign(P, std::vector<int>(n_seqs, 0));
@@ -449,24 +461,29 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   const int W = c->S + 1;
   std::vector<int32_t> ints((size_t)(2 * P + 8) * W, 0);
   auto tab = [&](int i) { return ints.data() + (size_t)i * W; };
-  for (int g = 0; g <= P; ++g)
-    for (int s = 0; s <= n_seqs; ++s) tab(g)[s] = c->seg_cu[g][s];
-  for (int p = 0; p < P; ++p)
-    for (int s = 0; s <= n_seqs; ++s) tab(P + 1 + p)[s] = cu_drop[p][s];
-  for (int s = 0; s < n_seqs; ++s) {
-    tab(2 * P + 1)[s] = c->seq_base[s];
-    tab(2 * P + 2)[s] = c->seg_cu[P][s + 1] - 1;  // last row of the sequence in the final segment
-  }
-  LAZY_CUDA_OK(cudaMemcpyAsync(c->d_ints, ints.data(), ints.size() * 4, cudaMemcpyHostToDevice, st));
   auto d_cu = [&](int g) { return c->d_ints + (size_t)g * W; };
   auto d_cu_drop = [&](int p) { return c->d_ints + (size_t)(P + 1 + p) * W; };
   const int32_t *d_base = c->d_ints + (size_t)(2 * P + 1) * W;
   const int32_t *d_last = c->d_ints + (size_t)(2 * P + 2) * W;
-
-  for (int g = 0; g <= P; ++g)
-    LAZY_TRY(launch_seg_rows(st, d_cu(g), d_base, n_seqs, c->seg_cu[g][n_seqs], c->kv_row[g]));
-  for (int p = 0; p < P; ++p)
-    LAZY_TRY(launch_seg_rows(st, d_cu_drop(p), d_base, n_seqs, cu_drop[p][n_seqs], c->aux_dst[p]));
+  // Uploads the tables and rebuilds the cache-row lists of segments g_from.. and the Aux-row lists of
+  // points p_from.. (everything, at the start of a run; the tail, after a cut whose count was read back).
+  auto upload_tables = [&](int g_from, int p_from) -> int {
+    for (int g = 0; g <= P; ++g)
+      for (int s = 0; s <= n_seqs; ++s) tab(g)[s] = c->seg_cu[g][s];
+    for (int p = 0; p < P; ++p)
+      for (int s = 0; s <= n_seqs; ++s) tab(P + 1 + p)[s] = cu_drop[p][s];
+    for (int s = 0; s < n_seqs; ++s) {
+      tab(2 * P + 1)[s] = c->seq_base[s];
+      tab(2 * P + 2)[s] = c->seg_cu[P][s + 1] - 1;  // last row of the sequence in the final segment
+    }
+    LAZY_CUDA_OK(cudaMemcpyAsync(c->d_ints, ints.data(), ints.size() * 4, cudaMemcpyHostToDevice, st));
+    for (int g = g_from; g <= P; ++g)
+      LAZY_TRY(launch_seg_rows(st, d_cu(g), d_base, n_seqs, c->seg_cu[g][n_seqs], c->kv_row[g]));
+    for (int p = p_from; p < P; ++p)
+      LAZY_TRY(launch_seg_rows(st, d_cu_drop(p), d_base, n_seqs, cu_drop[p][n_seqs], c->aux_dst[p]));
+    return LAZY_OK;
+  };
+  LAZY_TRY(upload_tables(0, 0));
 
   // ---- embedding, positions
   TIMED(LAZY_K_EMBED, 0, 2.0 * N * rb, launch_embed(st, dt, c->tok_embed, d_prompt_ids, c->x, N, d, c->V, status));
@@ -587,6 +604,28 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
                                         it->second.first, it->second.second, c->sel_scores));
         }
         sel = c->sel_scores;
+      }
+      if (c->select_threshold) {
+        // Threshold reading: a row is pruned iff its score is smaller than the score at the scheduled rank, so
+        // ties at that rank all survive and the count depends on the data.  One count per sequence is read
+        // back here (a stream synchronisation per cut); every later row count is re-planned from it.
+        std::vector<int32_t> h_counts((size_t)n_seqs, 0);
+        LAZY_TRY(launch_select_tie_count(st, sel, d_cu(g), d_cu(g + 1), n_seqs, c->d_found, status));
+        LAZY_CUDA_OK(cudaMemcpyAsync(h_counts.data(), c->d_found, (size_t)n_seqs * 4, cudaMemcpyDeviceToHost, st));
+        LAZY_CUDA_OK(cudaStreamSynchronize(st));
+        bool changed = false;
+        for (int s = 0; s < n_seqs; ++s) {
+          const int present = c->seg_cu[g][s + 1] - c->seg_cu[g][s];
+          const int keep = h_counts[s];
+          if (keep < 1 || keep > present) return LAZY_E_STATE;
+          if (keep != c->seg_cu[g + 1][s + 1] - c->seg_cu[g + 1][s]) changed = true;
+          c->seg_cu[g + 1][s + 1] = c->seg_cu[g + 1][s] + keep;
+          cu_drop[p][s + 1] = cu_drop[p][s] + (present - keep);
+        }
+        if (changed) {
+          LAZY_TRY(plan_from(p + 1));
+          LAZY_TRY(upload_tables(g + 1, p));
+        }
       }
       const int n_keep = c->seg_cu[g + 1][n_seqs], n_drop = n - n_keep;
       char *ar = c->aux_rows + (size_t)p * c->cap_kv * rb;

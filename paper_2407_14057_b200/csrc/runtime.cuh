@@ -52,6 +52,7 @@ struct lazy_ctx {
                                        // position if it came from the Aux Cache, else -1
   int32_t *dec_i32;  // integer scratch of the decode step
   float *dec_f32;
+  bool select_threshold = false;  // threshold reading of the selection: ties at the scheduled rank all survive
   bool aux_after_layer = false;  // cut after the whole scoring layer (Aux rows = layer output) instead of before its MLP
   void *gemm_scratch;  // split-wave partials and counters of the tensor-core GEMMs (bf16 only)
   size_t gemm_scratch_bytes;

@@ -298,6 +298,46 @@ select_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_i
   if (threadIdx.x == 0 && kept_so_far != n_keep) dev_fail(status, LAZY_E_STATE, W_SELECT, seq, kept_so_far);
 }
 
+// Threshold reading at the scheduled rank: tau = the n_keep-th largest key of the sequence (the last row
+// counting as the largest), and every row whose score is not smaller than tau survives.  The kernel only
+// COUNTS the survivors: counts[seq] = n_keep + (keys equal to tau beyond the ones the count form would
+// keep).  With that count the ordinary selection keeps exactly the rows with score >= tau (no tie is cut),
+// so the host reads the counts back and launches select_kernel with them.
+__global__ void __launch_bounds__(SEL_THREADS)
+select_tie_count_kernel(const float *__restrict__ scores, const int32_t *__restrict__ cu_in,
+                        const int32_t *__restrict__ cu_keep, int32_t *__restrict__ counts, DevStatus *status) {
+  const int seq = blockIdx.x;
+  const int in0 = cu_in[seq], n = cu_in[seq + 1] - in0;
+  const int n_keep = cu_keep[seq + 1] - cu_keep[seq];
+  if (n == 0) {
+    if (threadIdx.x == 0) counts[seq] = 0;
+    return;
+  }
+  if (n_keep < 1 || n_keep > n) {
+    if (threadIdx.x == 0) {
+      dev_fail(status, LAZY_E_BADARG, W_SELECT, seq, n_keep);
+      counts[seq] = n_keep < 1 ? 1 : n;
+    }
+    return;
+  }
+  const float *s = scores + in0;
+  __shared__ SelShared sh;
+  int k_ties;
+  const uint32_t tau = radix_kth_largest(s, n, n_keep, true, sh, &k_ties);
+  const bool cached = n <= SEL_CACHE;
+  int eq_total = 0;
+  for (int base = 0; base < n; base += SEL_THREADS) {
+    const int i = base + threadIdx.x;
+    uint32_t key = 0;
+    const bool valid = i < n;
+    if (valid) key = cached ? sh.keys[i] : ((i == n - 1) ? 0xffffffffu : score_key(s[i]));
+    int t;
+    block_excl_scan(valid && key == tau, sh.warp_tot, &t);
+    eq_total += t;
+  }
+  if (threadIdx.x == 0) counts[seq] = n_keep - k_ties + eq_total;
+}
+
 // Threshold form of the selection: tau = the score at the prune_bp/10000 quantile of the sequence's n scores
 // (the order statistic with index floor((n-1) * prune_bp / 10000) from below), every row with score >= tau is
 // kept, and the last row always.  The count depends on the data (ties at tau are all kept), so kept / dropped
@@ -409,6 +449,14 @@ int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t 
                             uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts) {
   if (n_seqs == 0) return LAZY_OK;
   select_threshold_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, prune_bp, keep_idx, drop_idx, counts);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
+int launch_select_tie_count(cudaStream_t st, const float *scores, const int32_t *cu_in, const int32_t *cu_keep,
+                            int n_seqs, int32_t *counts, DevStatus *status) {
+  if (n_seqs == 0) return LAZY_OK;
+  select_tie_count_kernel<<<n_seqs, SEL_THREADS, 0, st>>>(scores, cu_in, cu_keep, counts, status);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

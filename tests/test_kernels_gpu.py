@@ -371,3 +371,13 @@ def test_bounded_wait_runs_out_and_reports_timeout(which, where):
     B.lazy_device_status()
     ref = x.double().cpu().numpy() @ w.double().cpu().numpy().T
     assert rel_err(to_np(got), ref) < 1e-2
+
+
+def test_select_kernel_writes_position_lists_and_handles_long_sequences():
+    """The selection at sizes on both sides of its shared-memory key cache (8192 rows), clustered scores (all
+    keys share their high bytes, the case the warp-combined histogram is for) included: bit-exact sets."""
+    for n, kind in ((8192, "uniform"), (8193, "lognormal"), (20000, "duplicates"), (3376, "uniform")):
+        s = synth.make_scores(n, kind, 77)
+        if kind == "uniform":
+            s = s + torch.arange(n, dtype=torch.float32) * 1e-12    # nearly equal, distinct in the low bits
+        _select_case([s], [max(1, (n * 3) // 10)])

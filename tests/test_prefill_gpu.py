@@ -276,3 +276,87 @@ def test_prune_op_full_size_bf16():
     """The single-layer pruning op at its full size: hidden [4096, 4096], 32 heads x 128, keep 60 %
     (2458 kept / 1638 to the Aux Cache)."""
     _prune_case(torch.bfloat16, 4096, 32, 128, 6000, seed=1)
+
+
+# ----------------------------------------------------------------------------- threshold reading end to end
+def _zero_query(W, layer, d):
+    """q = 0 in one layer: every attention row is uniform, every Eq. 1 score equals 1/n exactly."""
+    W["layers"][layer]["w_qkv"][:d] = 0
+
+
+def test_threshold_selection_prefill_and_decode_with_ties_fp32():
+    """The selection read as a threshold (pruned iff the score is smaller than the score at the scheduled rank):
+    ties at the threshold all survive, so row counts depend on the data and the library reads them back at
+    every point.  Layer 0 has a zero query projection, so all its scores tie: sequence by sequence the first
+    cut prunes NOTHING under this reading (the count reading would keep 60 %), the later cuts have no ties and
+    keep the scheduled counts.  Kept sets, hidden states, caches, Aux contents, logits and two decode steps
+    against the oracle run with the same reading."""
+    shape, schedule, lengths = synth.TINY.with_layers(3), ((1, 6000), (2, 3000)), [50, 9, 31]
+    W = synth.make_weights(shape, 21, bf16=False)
+    synth.perturb_gains(W, 121)
+    _zero_query(W, 0, shape.d_model)
+    Wn = weights_to_np(W)
+    ids, cu = synth.make_varlen_batch(shape.vocab, lengths, 22)
+    S = len(lengths)
+    eng = B.LazyPrefill(shape, _to_cuda(W), schedule, torch.float32, S, sum(lengths), max_new_tokens=2,
+                        debug_capture=True)
+    eng.lazy_set_selection(True)
+    logits = torch.empty((S, shape.vocab), dtype=torch.float32, device="cuda")
+    nxt = torch.empty(S, dtype=torch.int32, device="cuda")
+    eng.lazy_prefill_run(ids.cuda(), cu, logits)
+    eng.lazy_sync_status()
+    states = [O.prefill(shape, Wn, to_np(ids)[cu[s]:cu[s + 1]], schedule, selection="threshold") for s in range(S)]
+    st = eng.lazy_get_stats()
+    assert st.rows_computed[0] == sum(lengths) and st.rows_computed[1] == sum(lengths)     # nothing pruned at cut 1
+    assert st.rows_computed[2] == sum(O.keep_count(n, 3000, n) for n in lengths)
+    off = [0] * shape.n_layers
+    for s in range(S):
+        ref = states[s]
+        assert len(ref.kept_pos[1]) == lengths[s]                                          # the oracle agrees
+        for e, _ in schedule:
+            assert np.array_equal(to_np(eng.lazy_get_kept(e, s)), ref.kept_pos[e])
+        for l in range(shape.n_layers):
+            assert np.max(np.abs(to_np(eng.lazy_get_scores(l, s)) - ref.scores[l])) < 1e-5
+            n_l = ref.hidden_out[l].shape[0]
+            got = to_np(eng.lazy_get_hidden(l))[off[l]:off[l] + n_l]
+            off[l] += n_l
+            assert rel_err(got, ref.hidden_out[l]) < 1e-4
+            apos, _ = eng.lazy_get_aux(l, s)
+            assert to_np(apos).tolist() == sorted(ref.layers[l].aux.keys())
+        assert rel_err(to_np(logits[s]), ref.logits) < 1e-4
+    tok = [O.greedy(s_.logits) for s_ in states]
+    for step in range(2):
+        ref_logits = [O.decode_step(shape, Wn, states[s], tok[s]) for s in range(S)]
+        eng.lazy_decode_step(torch.tensor(tok, dtype=torch.int32).cuda(), logits, nxt)
+        eng.lazy_sync_status()
+        for s in range(S):
+            assert rel_err(to_np(logits[s]), ref_logits[s]) < 1e-4, (step, s)
+            for e, _ in schedule:
+                assert np.array_equal(to_np(eng.lazy_get_kept(e, s)), states[s].kept_pos[e]), (step, s, e)
+                assert sorted(to_np(eng.lazy_get_revived(e, s)).tolist()) == sorted(states[s].revived_pos[e].tolist())
+            assert int(nxt[s]) == O.greedy(ref_logits[s])
+        tok = [O.greedy(l) for l in ref_logits]
+    # the count reading on the same inputs prunes at the first cut
+    eng.lazy_set_selection(False)
+    eng.lazy_prefill_run(ids.cuda(), cu, logits)
+    eng.lazy_sync_status()
+    assert eng.lazy_get_stats().rows_computed[1] == sum(O.keep_count(n, 6000, n) for n in lengths)
+    eng.close()
+
+
+def test_threshold_selection_equals_count_selection_without_ties_bf16():
+    """Generic inputs have no ties at the threshold: both readings select the same sets and give the same bits."""
+    shape, schedule, n = synth.SMALL, ((1, 7000), (2, 5000), (3, 3000)), 333
+    W = _to_cuda(synth.make_weights(shape, 23, bf16=True))
+    ids = synth.make_prompt(shape.vocab, n, 24).cuda()
+    out = []
+    for thr in (False, True):
+        eng = B.LazyPrefill(shape, W, schedule, torch.bfloat16, 1, n)
+        eng.lazy_set_selection(thr)
+        lg = torch.empty((1, shape.vocab), dtype=torch.float32, device="cuda")
+        eng.lazy_prefill_run(ids, [0, n], lg)
+        eng.lazy_sync_status()
+        out.append((lg.clone(), [to_np(eng.lazy_get_kept(e, 0)) for e, _ in schedule]))
+        eng.close()
+    assert all(np.array_equal(a, b) for a, b in zip(out[0][1], out[1][1]))
+    assert torch.equal(out[0][0], out[1][0])
