@@ -343,9 +343,11 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
 
 // Splits the last partial wave along K when that pays: `units` persistent units of `cta_per_unit` CTAs,
 // m_tiles row tiles, M x K activations.  Costs are in K slices (one slice of MMAs ~ 0.4 us): a split tile
-// pays ~6 slices for its dump and ~10 for each part its finisher adds (measured; extra_cost more for a
-// heavy epilogue), so tiles are cut into at most four parts, and only when the wave then ends at least a
-// fifth earlier than a whole tile would.  The parts of
+// is charged 3 slices for its dump and 4 for each part its finisher adds (extra_cost more for a heavy
+// epilogue), tiles are cut into at most four parts, and only when the wave then ends earlier than 95 % of a
+// whole tile.  (Swept on the four projections at 1013-3376 rows: with the charges at 6 / 10 and the bar at
+// 80 % the output and down projections at 2364 rows ran whole waves and took 87 / 198 us instead of 78 /
+// 176 us.)  The parts of
 // the tiles of one column block run skewed in K, so the B rows of the tail must stay L2-resident (next to
 // A) or they are re-read from HBM.  scratch NULL or too small, or no gain: plain tile loop.
 inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit, int m_tiles, int m_band,
@@ -367,7 +369,7 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
   const long long a_rows = M < (long long)m_tiles * 256 ? M : (long long)m_tiles * 256;  // rows of the tail's band
   if (m_tiles > 2 && b_tail + a_rows * K * 2 > 96ll << 20) return t;  // one or two row tiles: B is read once anyway
   int best_units = 0;
-  long long best_cost = (long long)num_kb * 4 / 5;
+  long long best_cost = (long long)num_kb * 19 / 20;
   for (int parts = 2; parts <= 4; ++parts) {
     long long tu = (long long)rem * parts;
     if (tu > units) tu = units;
@@ -376,7 +378,7 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
     if (per_unit < GEMM_TAIL_MIN_KB) continue;
     const bool aligned = tu == (long long)rem * parts;  // ranges end on tile boundaries
     const long long pieces = aligned ? parts : (num_kb + per_unit - 1) / per_unit + 1;
-    const long long cost = per_unit + 6 + 10 * (pieces - 1) + extra_cost;
+    const long long cost = per_unit + 3 + 4 * (pieces - 1) + extra_cost;
     if (cost < best_cost) {
       best_cost = cost;
       best_units = (int)tu;
