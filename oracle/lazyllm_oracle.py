@@ -88,16 +88,21 @@ def attend(q: np.ndarray, k: np.ndarray, v: np.ndarray, qpos: np.ndarray, kpos: 
            score_row: int) -> Tuple[np.ndarray, np.ndarray]:
     """Multi-head attention output and the importance score of Eq. 1.
 
-    q: [nq, H, dh]; k, v: [nk, H, dh].  Returns (o [nq, H*dh], s [nk]) where
+    q: [nq, H, dh]; k, v: [nk, Hkv, dh] with Hkv dividing H.  With Hkv < H (grouped-query attention, the
+    layout of the 7B-class models with fewer key/value heads than query heads) query head h reads
+    key/value head h // (H // Hkv).  Returns (o [nq, H*dh], s [nk]) where
     s_j = (1/H) * sum_h A_h[score_row, j]: the probabilities with which the token whose
-    successor is being predicted attends to token j, averaged over the H heads.
+    successor is being predicted attends to token j, averaged over the H query heads.
     """
     nq, H, dh = q.shape
+    Hkv = k.shape[1]
+    assert H % Hkv == 0 and v.shape[1] == Hkv
+    group = H // Hkv
     o = np.zeros((nq, H, dh), dtype=F64)
     s = np.zeros(k.shape[0], dtype=F64)
     for h in range(H):
-        A = attention_probs(q[:, h, :], k[:, h, :], qpos, kpos)
-        o[:, h, :] = A @ f64(v[:, h, :])
+        A = attention_probs(q[:, h, :], k[:, h // group, :], qpos, kpos)
+        o[:, h, :] = A @ f64(v[:, h // group, :])
         s += A[score_row, :]
     return o.reshape(nq, H * dh), s / H
 
@@ -185,15 +190,23 @@ def select_threshold(scores: np.ndarray, prune_bp: int) -> Tuple[np.ndarray, np.
     return keep, drop
 
 
+def kv_heads(cfg) -> int:
+    """Key/value heads of the shape (grouped-query attention when fewer than the query heads)."""
+    return int(getattr(cfg, "n_kv_heads", 0) or cfg.n_heads)
+
+
 def _layer_qkv(cfg, lw, x, pos):
-    """Pre-norm, QKV projection, head split, RoPE on q and k."""
+    """Pre-norm, QKV projection, head split, RoPE on q and k.  w_qkv = [q rows | k rows | v rows] with
+    H*dh, Hkv*dh and Hkv*dh rows."""
     H, dh, d = cfg.n_heads, cfg.head_dim, cfg.d_model
+    Hkv = kv_heads(cfg)
+    dkv = Hkv * dh
     h = rmsnorm(x, lw["g_attn"], cfg.rms_eps)
     qkv = h @ f64(lw["w_qkv"]).T
     n = x.shape[0]
     q = rope(qkv[:, :d].reshape(n, H, dh), pos, cfg.rope_theta)
-    k = rope(qkv[:, d:2 * d].reshape(n, H, dh), pos, cfg.rope_theta)
-    v = qkv[:, 2 * d:].reshape(n, H, dh)
+    k = rope(qkv[:, d:d + dkv].reshape(n, Hkv, dh), pos, cfg.rope_theta)
+    v = qkv[:, d + dkv:].reshape(n, Hkv, dh)
     return q, k, v
 
 

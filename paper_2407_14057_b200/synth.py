@@ -32,6 +32,14 @@ class ModelShape:
     vocab: int
     rms_eps: float = 1e-6
     rope_theta: float = 1e4
+    n_kv_heads: int = 0          # key/value heads; 0 = as many as query heads (no grouping)
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_heads or self.n_heads
+
+    def with_kv_heads(self, n_kv_heads: int) -> "ModelShape":
+        return dataclasses.replace(self, n_kv_heads=n_kv_heads)
 
     def with_layers(self, n_layers: int) -> "ModelShape":
         return dataclasses.replace(self, n_layers=n_layers)
@@ -90,7 +98,7 @@ def make_weights(shape: ModelShape, seed: int, bf16: bool, device: str = "cpu",
     layers: List[Dict[str, torch.Tensor]] = []
     for _ in range(shape.n_layers):
         layers.append({
-            "w_qkv": _normal((3 * d, d), std, g, device, bf16),
+            "w_qkv": _normal((d + 2 * shape.kv_heads * shape.head_dim, d), std, g, device, bf16),
             "w_o": _normal((d, d), std, g, device, bf16),
             "w_gate": _normal((F, d), std, g, device, bf16),
             "w_up": _normal((F, d), std, g, device, bf16),

@@ -30,7 +30,7 @@ def _hf_model(shape, W):
     from transformers import LlamaConfig, LlamaForCausalLM
     cfg = LlamaConfig(vocab_size=shape.vocab, hidden_size=shape.d_model,
                       intermediate_size=shape.d_ffn, num_hidden_layers=shape.n_layers,
-                      num_attention_heads=shape.n_heads, num_key_value_heads=shape.n_heads,
+                      num_attention_heads=shape.n_heads, num_key_value_heads=shape.kv_heads,
                       head_dim=shape.head_dim, rms_norm_eps=shape.rms_eps,
                       rope_theta=shape.rope_theta, attention_bias=False, mlp_bias=False,
                       tie_word_embeddings=False, attn_implementation="eager",
@@ -42,8 +42,9 @@ def _hf_model(shape, W):
     for l, lw in enumerate(W["layers"]):
         p = f"model.layers.{l}."
         sd[p + "self_attn.q_proj.weight"] = lw["w_qkv"][:d]
-        sd[p + "self_attn.k_proj.weight"] = lw["w_qkv"][d:2 * d]
-        sd[p + "self_attn.v_proj.weight"] = lw["w_qkv"][2 * d:]
+        dkv = shape.kv_heads * shape.head_dim
+        sd[p + "self_attn.k_proj.weight"] = lw["w_qkv"][d:d + dkv]
+        sd[p + "self_attn.v_proj.weight"] = lw["w_qkv"][d + dkv:]
         sd[p + "self_attn.o_proj.weight"] = lw["w_o"]
         sd[p + "mlp.gate_proj.weight"] = lw["w_gate"]
         sd[p + "mlp.up_proj.weight"] = lw["w_up"]
@@ -71,6 +72,35 @@ def test_full_keep_matches_library_llama():
         assert np.max(np.abs(st.scores[l] - ref_s)) < 1e-6
         if l + 1 < MINI.n_layers:  # the library applies the final norm to its last entry
             assert rel_err(st.hidden_out[l], out.hidden_states[l + 1][0].numpy()) < 1e-5
+
+
+def test_grouped_query_attention_matches_library_llama():
+    """Fewer key/value heads than query heads (query head h reads key/value head h // group): logits, hidden
+    states, the head-mean last attention row and greedy decode against the library's Llama with
+    num_key_value_heads = 2 of 4 heads and 1 of 4 heads."""
+    for kvh in (2, 1):
+        shape = MINI.with_kv_heads(kvh)
+        W = mini_weights(seed=40 + kvh, shape=shape)
+        assert W["layers"][0]["w_qkv"].shape[0] == shape.d_model + 2 * kvh * shape.head_dim
+        ids = synth.make_prompt(shape.vocab, 29, seed=6)
+        m = _hf_model(shape, W)
+        with torch.no_grad():
+            out = m(ids.long()[None], output_attentions=True, output_hidden_states=True)
+            gen = m.generate(ids.long()[None], max_new_tokens=3, do_sample=False, use_cache=True)
+        Wn = weights_to_np(W)
+        st = O.prefill(shape, Wn, to_np(ids), schedule=())
+        assert rel_err(st.logits, out.logits[0, -1].numpy()) < 1e-5
+        for l in range(shape.n_layers):
+            ref_s = out.attentions[l][0, :, -1, :].mean(dim=0).numpy()
+            assert np.max(np.abs(st.scores[l] - ref_s)) < 1e-6
+            assert st.layers[l].kv[0][0].shape == (kvh, shape.head_dim)      # the cache holds kv heads only
+        got = [O.greedy(st.logits)]
+        for _ in range(2):
+            got.append(O.greedy(O.decode_step(shape, Wn, st, got[-1])))
+        assert got == gen[0, ids.shape[0]:].tolist()
+        # pruning on top: invariants of the pruned run hold with grouped heads as well
+        pr = O.prefill(shape, Wn, to_np(ids), ((1, 6000), (2, 3000)))
+        assert [len(pr.kept_pos[e]) for e in (1, 2)] == [18, 9] and abs(pr.scores[2].sum() - 1) < 1e-12
 
 
 def test_decode_full_keep_matches_library_greedy():
