@@ -53,13 +53,17 @@ typedef struct {
   int32_t max_seqs;          /* sequences per batch                                          */
   int32_t max_prompt_tokens; /* packed total over the batch                                  */
   int32_t max_new_tokens;    /* decode steps per sequence the caches leave room for          */
+  int32_t n_kv_heads;        /* key/value heads (grouped-query attention); 0 = n_heads.  Must divide
+                              * n_heads: query head h reads key/value head h / (n_heads / n_kv_heads) */
 } lazy_model_cfg;
 
 /* Weights, all device memory except the per-layer pointer arrays themselves (host arrays of
- * n_layers device pointers).  w_qkv = [3d, d] with the q rows first, then k, then v. */
+ * n_layers device pointers).  w_qkv = [d + 2 d_kv, d] with the d query rows first, then the d_kv key rows,
+ * then the d_kv value rows, d_kv = n_kv_heads * head_dim (= d without grouped-query attention).  K / V
+ * cache rows (lazy_get_kv) are d_kv wide. */
 typedef struct {
   const void *tok_embed;          /* [vocab, d]                */
-  const void *const *w_qkv;       /* n_layers x [3d, d]        */
+  const void *const *w_qkv;       /* n_layers x [d + 2 d_kv, d] */
   const void *const *w_o;         /* n_layers x [d, d]         */
   const void *const *w_gate;      /* n_layers x [d_ffn, d]     */
   const void *const *w_up;        /* n_layers x [d_ffn, d]     */

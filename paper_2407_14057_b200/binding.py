@@ -33,7 +33,7 @@ class lazy_model_cfg(C.Structure):
                 ("head_dim", C.c_int32), ("d_ffn", C.c_int32), ("vocab", C.c_int32),
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("dtype", C.c_int32),
                 ("max_seqs", C.c_int32), ("max_prompt_tokens", C.c_int32),
-                ("max_new_tokens", C.c_int32)]
+                ("max_new_tokens", C.c_int32), ("n_kv_heads", C.c_int32)]
 
 
 class lazy_weights(C.Structure):
@@ -182,7 +182,8 @@ class LazyPrefill:
         self.shape, self.dtype, self.schedule = shape, dtype, tuple(schedule)
         self.cfg = lazy_model_cfg(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim,
                                   shape.d_ffn, shape.vocab, shape.rms_eps, shape.rope_theta,
-                                  dtype_code(dtype), max_seqs, max_prompt_tokens, max_new_tokens)
+                                  dtype_code(dtype), max_seqs, max_prompt_tokens, max_new_tokens,
+                                  getattr(shape, "n_kv_heads", 0))
         self._sched, self._sched_keep = _make_schedule(schedule)
         nbytes = L.lazy_prefill_workspace_bytes_ex(C.byref(self.cfg), C.byref(self._sched),
                                                    1 if debug_capture else 0)
@@ -277,7 +278,7 @@ class LazyPrefill:
     def lazy_get_kv(self, layer: int, seq: int = 0):
         cnt = C.c_int32()
         _check("lazy_get_kv", lib().lazy_get_kv(self.ctx, _stream(), layer, seq, None, None, None, C.byref(cnt)))
-        d = self.shape.d_model
+        d = (getattr(self.shape, "n_kv_heads", 0) or self.shape.n_heads) * self.shape.head_dim
         pos = torch.empty(cnt.value, dtype=torch.int32, device="cuda")
         k = torch.empty((cnt.value, d), dtype=self.dtype, device="cuda")
         v = torch.empty((cnt.value, d), dtype=self.dtype, device="cuda")

@@ -26,11 +26,12 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
                                     const int32_t *__restrict__ cu_kv,
                                     const int32_t *__restrict__ kv_idx,
                                     const int32_t *__restrict__ q_kvlen, int n_seqs, int n_total,
-                                    int n_heads, int head_dim) {
+                                    int n_heads, int head_dim, int kv_group) {
   extern __shared__ float qs_all[];  // [warps][head_dim]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * (blockDim.x >> 5) + warp;
   const int h = blockIdx.y;
+  const int hk = h / kv_group;  // key/value head of this query head
   if (r >= n_total) return;
   int lo = 0, hi = n_seqs;
   while (hi - lo > 1) {
@@ -56,7 +57,7 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
     const int j = j0 + lane;
     float s = -INFINITY;
     if (j <= i) {
-      const T *kr = k + (kidx ? (size_t)kidx[j] : kbase + j) * ldkv + h * head_dim;
+      const T *kr = k + (kidx ? (size_t)kidx[j] : kbase + j) * ldkv + hk * head_dim;
       float dot = 0.f;
       for (int t = 0; t < head_dim; ++t) dot += qs[t] * Elem<T>::to_f(kr[t]);
       s = dot;
@@ -71,7 +72,7 @@ __global__ void attn_rowwarp_kernel(const T *__restrict__ q, int ldq, const T *_
     const int cnt = min(32, i - j0 + 1);
     for (int jj = 0; jj < cnt; ++jj) {
       const float pj = __shfl_sync(0xffffffffu, p, jj);
-      const T *vr = v + (kidx ? (size_t)kidx[j0 + jj] : kbase + j0 + jj) * ldkv + h * head_dim;
+      const T *vr = v + (kidx ? (size_t)kidx[j0 + jj] : kbase + j0 + jj) * ldkv + hk * head_dim;
 #pragma unroll
       for (int t = 0; t < 8; ++t)
         if (t < per_lane) acc[t] += pj * Elem<T>::to_f(vr[lane + 32 * t]);
@@ -143,7 +144,7 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
                 const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base,
                 const int32_t *__restrict__ cu_kv, const int32_t *__restrict__ kv_idx,
                 const int32_t *__restrict__ q_kvlen, int n_heads, int n_splits,
-                float *__restrict__ part_o, float *__restrict__ part_ml) {
+                float *__restrict__ part_o, float *__restrict__ part_ml, int kv_group) {
   extern __shared__ __align__(128) uint8_t fa_smem[];
   const int seq = blockIdx.z, h = blockIdx.y;
   const int q_start = cu_q[seq];
@@ -160,8 +161,8 @@ attn_mma_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__restrict__ k,
   const int n_kv = kv_idx ? cu_kv[seq + 1] - cu_kv[seq] : n;
   const size_t kb = kv_idx ? 0 : (kv_base ? (size_t)kv_base[seq] : (size_t)q_start);
   const bf16 *qg = q + (size_t)q_start * ldq + h * FA_D;
-  const bf16 *kg = k + kb * ldkv + h * FA_D;
-  const bf16 *vg = v + kb * ldkv + h * FA_D;
+  const bf16 *kg = k + kb * ldkv + (h / kv_group) * FA_D;
+  const bf16 *vg = v + kb * ldkv + (h / kv_group) * FA_D;
 
   const uint32_t sQ = smem_addr(fa_smem);
   const uint32_t sK = sQ + FA_TILE_BYTES;       // two buffers
@@ -348,9 +349,9 @@ bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv) {
 
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                      const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
-                     int n_seqs, int max_len, int n_total, int n_heads, int head_dim) {
+                     int n_seqs, int max_len, int n_total, int n_heads, int head_dim, int n_kv_heads) {
   return launch_attention_ex(st, dtype, q, ldq, k, v, ldkv, o, cu_q, kv_base, nullptr, nullptr, nullptr,
-                             n_seqs, max_len, n_total, n_heads, head_dim);
+                             n_seqs, max_len, n_total, n_heads, head_dim, n_kv_heads);
 }
 
 bool attention_list_split_eligible(int dtype, int head_dim) { return dtype == LAZY_BF16 && head_dim == FA_D; }
@@ -371,8 +372,10 @@ int attention_list_splits(int n_seqs, int max_rows, int n_heads, int max_ctx) {
 int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const void *k, const void *v, int ldkv,
                                 void *o, const int32_t *cu_q, const int32_t *cu_kv, const int32_t *kv_idx,
                                 const int32_t *q_kvlen, const int32_t *score_row, int n_seqs, int max_rows,
-                                int n_total, int n_heads, int n_splits, float *part, float *stats) {
+                                int n_total, int n_heads, int n_splits, float *part, float *stats, int n_kv_heads) {
   if (n_total == 0 || n_seqs == 0) return LAZY_OK;
+  const int kv_group = kv_group_of(n_heads, n_kv_heads);
+  if (kv_group < 1) return LAZY_E_BADARG;
   if (!part || !stats || !score_row || n_splits < 2 || (ldq % 8) || (ldkv % 8)) return LAZY_E_BADARG;
   static bool attr_set = false;
   if (!attr_set) {
@@ -384,7 +387,7 @@ int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const v
   dim3 grid(cdiv(max_rows, FA_BM) * n_splits, n_heads, n_seqs);
   attn_mma_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>((const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v,
                                                            ldkv, (bf16 *)o, cu_q, nullptr, cu_kv, kv_idx, q_kvlen,
-                                                           n_heads, n_splits, part_o, part_ml);
+                                                           n_heads, n_splits, part_o, part_ml, kv_group);
   LAZY_COUNT_LAUNCH();
   if (launch_ok() != LAZY_OK) return LAZY_E_CUDA;
   return launch_attention_combine(st, part_o, part_ml, n_splits, cu_q, score_row, n_seqs, n_total, n_heads, o,
@@ -394,8 +397,10 @@ int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const v
 int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                         const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                         const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
-                        int max_len, int n_total, int n_heads, int head_dim) {
+                        int max_len, int n_total, int n_heads, int head_dim, int n_kv_heads) {
   if (n_total == 0 || n_seqs == 0) return LAZY_OK;
+  const int kv_group = kv_group_of(n_heads, n_kv_heads);
+  if (kv_group < 1) return LAZY_E_BADARG;
   if (dtype == LAZY_BF16 && head_dim == FA_D && (ldq % 8) == 0 && (ldkv % 8) == 0) {
     static bool attr_set = false;
     if (!attr_set) {
@@ -407,7 +412,7 @@ int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, cons
     attn_mma_kernel<<<grid, FA_THREADS, FA_SMEM_BYTES, st>>>((const bf16 *)q, ldq, (const bf16 *)k,
                                                              (const bf16 *)v, ldkv, (bf16 *)o, cu_q,
                                                              kv_base, cu_kv, kv_idx, q_kvlen, n_heads, 1, nullptr,
-                                                             nullptr);
+                                                             nullptr, kv_group);
     LAZY_COUNT_LAUNCH();
     return launch_ok();
   }
@@ -419,12 +424,12 @@ int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, cons
     attn_rowwarp_kernel<float><<<grid, warps * 32, smem, st>>>((const float *)q, ldq, (const float *)k,
                                                               (const float *)v, ldkv, (float *)o, cu_q,
                                                               kv_base, cu_kv, kv_idx, q_kvlen, n_seqs, n_total,
-                                                              n_heads, head_dim);
+                                                              n_heads, head_dim, kv_group);
   else
     attn_rowwarp_kernel<bf16><<<grid, warps * 32, smem, st>>>((const bf16 *)q, ldq, (const bf16 *)k,
                                                              (const bf16 *)v, ldkv, (bf16 *)o, cu_q,
                                                              kv_base, cu_kv, kv_idx, q_kvlen, n_seqs, n_total,
-                                                             n_heads, head_dim);
+                                                             n_heads, head_dim, kv_group);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

@@ -43,7 +43,7 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
                            const int32_t *__restrict__ cu_ctx, const int32_t *__restrict__ ctx_rows,
                            const int32_t *__restrict__ q_kvlen, const int32_t *__restrict__ score_row,
                            int n_seqs, int n_ctx_total, float *__restrict__ part_o,
-                           float *__restrict__ part_ml, float *__restrict__ logits) {
+                           float *__restrict__ part_ml, float *__restrict__ logits, int kv_group) {
   __shared__ int32_t srow[DK_SPLIT];
   __shared__ float sl[DK_SPLIT];
   __shared__ float so[DK_THREADS / 16][DK_HD];
@@ -86,7 +86,7 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int row = srow[warp * 16 + i * 2 + half];
-      if (row >= 0) kv[i].load(k + (size_t)row * ldkv + h * DK_HD + sub * 8);
+      if (row >= 0) kv[i].load(k + (size_t)row * ldkv + (h / kv_group) * DK_HD + sub * 8);
       else kv[i].raw = make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
@@ -121,7 +121,7 @@ attn_decode_partial_kernel(const bf16 *__restrict__ q, int ldq, const bf16 *__re
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int row = srow[g * 8 + i];
-      if (row >= 0) vv[i].load(v + (size_t)row * ldkv + h * DK_HD + sub * 8);
+      if (row >= 0) vv[i].load(v + (size_t)row * ldkv + (h / kv_group) * DK_HD + sub * 8);
       else vv[i].raw = make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
@@ -251,8 +251,10 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
                             int ldkv, void *o, int ldo, const int32_t *cu_x, const int32_t *cu_ctx,
                             const int32_t *ctx_rows, const int32_t *q_kvlen, const int32_t *score_row,
                             int n_seqs, int n_rows, int n_ctx_total, int max_ctx, int n_heads,
-                            float *part, float *logits, float *stats) {
+                            float *part, float *logits, float *stats, int n_kv_heads) {
   if (n_rows == 0) return LAZY_OK;
+  const int kv_group = kv_group_of(n_heads, n_kv_heads);
+  if (kv_group < 1) return LAZY_E_BADARG;
   if (!q || !k || !v || !o || !cu_x || !cu_ctx || !ctx_rows || !q_kvlen || !score_row || !part ||
       !logits || !stats)
     return LAZY_E_BADARG;
@@ -263,7 +265,7 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
   float *part_ml = part + (size_t)n_rows * n_heads * n_splits * DK_HD;
   LAZY_TRY(launch_pdl(attn_decode_partial_kernel, dim3(n_splits, n_heads, n_rows), dim3(DK_THREADS), 0, st,
                       (const bf16 *)q, ldq, (const bf16 *)k, (const bf16 *)v, ldkv, cu_x, cu_ctx, ctx_rows, q_kvlen,
-                      score_row, n_seqs, n_ctx_total, part_o, part_ml, logits));
+                      score_row, n_seqs, n_ctx_total, part_o, part_ml, logits, kv_group));
   LAZY_COUNT_LAUNCH();
   LAZY_TRY(launch_pdl(attn_decode_combine_kernel, dim3(n_heads, n_rows), dim3(DK_CTHREADS), 0, st,
                       (const float *)part_o, (const float *)part_ml, n_splits, cu_x, score_row, n_seqs, (bf16 *)o,

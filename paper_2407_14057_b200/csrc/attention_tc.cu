@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 2)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, bf16 *__restrict__ o, int ldo,
                     const int32_t *__restrict__ cu_q, const int32_t *__restrict__ kv_base, int q_start_arg,
-                    int n_arg, int kv_start_arg, DevStatus *status, const AttnScoreOut sc) {
+                    int n_arg, int kv_start_arg, DevStatus *status, const AttnScoreOut sc, int kv_group) {
   extern __shared__ uint8_t att_smem_raw[];
   const uint32_t raw_addr = smem_u32(att_smem_raw);
   const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -82,6 +82,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   // CTAs are handed out longest first over ALL heads: the long tiles of the last head start with the first
   // wave instead of at the end of the launch.
   const int h = blockIdx.x;
+  const int hk = h / kv_group;  // key/value head this query head reads (grouped-query attention)
   int q_start = q_start_arg, n = n_arg, kv_start = kv_start_arg;
   if (cu_q) {
     q_start = cu_q[blockIdx.z];
@@ -142,8 +143,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t full = smem_u32(&bars->k_full[st]);
         mbar_expect_tx(full, KV_TILE_BYTES);
         const int row = kv_start + j * TK;
-        tma_load_2d(sK + st * KV_TILE_BYTES, &map_k, full, h * HD, row);
-        tma_load_2d(sK + st * KV_TILE_BYTES + KV_BLK, &map_k, full, h * HD + 64, row);
+        tma_load_2d(sK + st * KV_TILE_BYTES, &map_k, full, hk * HD, row);
+        tma_load_2d(sK + st * KV_TILE_BYTES + KV_BLK, &map_k, full, hk * HD + 64, row);
       }
     } else if (lane == 1) {
       for (int j = 0; j < n_kt; ++j) {
@@ -153,8 +154,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t full = smem_u32(&bars->v_full[st]);
         mbar_expect_tx(full, KV_TILE_BYTES);
         const int row = kv_start + j * TK;
-        tma_load_2d(sV + st * KV_TILE_BYTES, &map_v, full, h * HD, row);
-        tma_load_2d(sV + st * KV_TILE_BYTES + KV_BLK, &map_v, full, h * HD + 64, row);
+        tma_load_2d(sV + st * KV_TILE_BYTES, &map_v, full, hk * HD, row);
+        tma_load_2d(sV + st * KV_TILE_BYTES + KV_BLK, &map_v, full, hk * HD + 64, row);
       }
     }
   } else if (warp == 1) {
@@ -390,15 +391,17 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
                         const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
                         const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
                         int n, int kv_start, DevStatus *status, float *score_scratch, int max_tiles,
-                        int n_seqs_total, int seq_id) {
+                        int n_seqs_total, int seq_id, int n_kv_heads) {
   if (n_seqs == 0 || max_len == 0) return LAZY_OK;
+  const int kv_group = kv_group_of(n_heads, n_kv_heads);
+  if (kv_group < 1) return LAZY_E_BADARG;
   if ((ldq % 8) || (ldkv % 8) || ((uintptr_t)q & 15) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15) ||
       ((uintptr_t)o & 15))
     return LAZY_E_BADARG;
   CUtensorMap mq, mk, mv;
   LAZY_TRY(tma_map_2d_bf16(&mq, q, q_rows, n_heads * HD, ldq, 64, TQ));
-  LAZY_TRY(tma_map_2d_bf16(&mk, k, kv_rows, n_heads * HD, ldkv, 64, TK));
-  LAZY_TRY(tma_map_2d_bf16(&mv, v, kv_rows, n_heads * HD, ldkv, 64, TK));
+  LAZY_TRY(tma_map_2d_bf16(&mk, k, kv_rows, n_heads / kv_group * HD, ldkv, 64, TK));
+  LAZY_TRY(tma_map_2d_bf16(&mv, v, kv_rows, n_heads / kv_group * HD, ldkv, 64, TK));
   static bool attr_set = false;
   if (!attr_set) {
     LAZY_CUDA_OK(cudaFuncSetAttribute(attn_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -415,7 +418,7 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
     sc.seq_id = seq_id;
   }
   attn_tcgen05_kernel<<<grid, ATT_THREADS, ATT_SMEM_BYTES, st>>>(mq, mk, mv, (bf16 *)o, n_heads * HD, cu_q,
-                                                                 kv_base, q_start, n, kv_start, status, sc);
+                                                                 kv_base, q_start, n, kv_start, status, sc, kv_group);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }

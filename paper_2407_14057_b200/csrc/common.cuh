@@ -182,10 +182,13 @@ int launch_rmsnorm_rows(cudaStream_t st, int dtype, const void *x, const int32_t
                         const void *g, void *y, int n, int d, float eps);
 int launch_rope_table(cudaStream_t st, float *table, int max_pos, int head_dim, float theta);
 // q rotated in place inside qkv; rotated k and v written to the caches at row kv_row[r]
-// (or kv_row_offset + r if kv_row is NULL) together with the position tag.
+// (or r if kv_row is NULL) together with the position tag.  Grouped-query attention: n_kv_heads key/value
+// heads (0 = n_heads); a row of qkv is [q: n_heads*dh | k: n_kv_heads*dh | v: n_kv_heads*dh], a cache row
+// n_kv_heads*dh wide.  Every attention / score launcher below takes the same n_kv_heads: query head h reads
+// key/value head h / (n_heads / n_kv_heads).
 int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, const float *table,
                    void *kcache, void *vcache, int32_t *kv_pos, const int32_t *kv_row, int n,
-                   int n_heads, int head_dim, int max_pos, DevStatus *status);
+                   int n_heads, int head_dim, int max_pos, DevStatus *status, int n_kv_heads = 0);
 // scratch (gemm_scratch_bytes() bytes, zeroed once, private to the stream) lets the tensor-core kernels
 // split the last partial wave of tiles along K; without it they run a plain tile loop.
 size_t gemm_scratch_bytes();
@@ -204,12 +207,12 @@ int launch_gemm_swiglu(cudaStream_t st, int dtype, const void *A, const void *Bg
 // QKV projection with the rotary embedding and the K/V cache write in its epilogue (bf16,
 // head_dim 128, d_model a multiple of 256): qkv [M, 3d] receives the rotated q (its k and v thirds
 // are left untouched), rotated k and v go to cache rows kv_row[r] (or r) with their position tag.
-bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim);
+bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim, int d_kv = 0);
 bool gemm_res_rows_supported(int dtype, int M, int K);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
-                         void *scratch = nullptr, size_t scratch_bytes = 0);
+                         void *scratch = nullptr, size_t scratch_bytes = 0, int d_kv = 0);
 // Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
 // rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).
 bool gemv_small_m_eligible(int dtype, int M, int K);
@@ -220,21 +223,26 @@ int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const vo
                         float eps = 0.f, int c_f32 = 0, bool b_const = false);
 int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
                          const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
-                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status);
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status, int d_kv = 0);
 int launch_gemm_simt(cudaStream_t st, int dtype, const void *A, const void *B0, const void *B1,
                      const void *R, void *C, int M, int N, int K, int swiglu);
 // Attention over packed sequences. Sequence s: query rows [cu_q[s], cu_q[s+1]) of q, key rows
 // kv_base[s] + j of k/v (kv_base NULL: same rows as q). Query row i sees keys j <= i (prefill).
 int launch_attention(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                      const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
-                     int n_seqs, int max_len, int n_total, int n_heads, int head_dim);
+                     int n_seqs, int max_len, int n_total, int n_heads, int head_dim, int n_kv_heads = 0);
+// Query heads per key/value head (1 without grouping); 0 if n_kv_heads does not divide n_heads.
+inline int kv_group_of(int n_heads, int n_kv_heads) {
+  if (n_kv_heads <= 0) return 1;
+  return n_heads % n_kv_heads ? 0 : n_heads / n_kv_heads;
+}
 // General form (decode): sequence s has query rows [cu_q[s], cu_q[s+1]) and a key LIST
 // kv_idx[cu_kv[s] .. cu_kv[s+1]) of cache rows in ascending position order; query row r sees the
 // first q_kvlen[r] entries of its sequence's list.
 int launch_attention_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k,
                         const void *v, int ldkv, void *o, const int32_t *cu_q, const int32_t *kv_base,
                         const int32_t *cu_kv, const int32_t *kv_idx, const int32_t *q_kvlen, int n_seqs,
-                        int max_len, int n_total, int n_heads, int head_dim);
+                        int max_len, int n_total, int n_heads, int head_dim, int n_kv_heads = 0);
 // Prefill attention, bf16 / head_dim 128, on tcgen05 (see attention_tc.cu).  Sequences either come
 // from device arrays (cu_q, kv_base) or one sequence is given by scalars; q_rows / kv_rows bound
 // the tensor maps (reads beyond them give zeros).
@@ -242,7 +250,7 @@ int launch_attention_tc(cudaStream_t st, const void *q, int ldq, long long q_row
                         const void *v, int ldkv, long long kv_rows, void *o, int n_heads,
                         const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int max_len, int q_start,
                         int n, int kv_start, DevStatus *status, float *score_scratch = nullptr,
-                        int max_tiles = 0, int n_seqs_total = 0, int seq_id = 0);
+                        int max_tiles = 0, int n_seqs_total = 0, int seq_id = 0, int n_kv_heads = 0);
 // With score_scratch (attn_score_scratch_floats floats) the attention kernel also leaves the last
 // row's softmax numerators there; launch_score_from_attention turns them into the Eq. 1 scores, for
 // n_layers consecutive layers over the same rows in one launch (layer y: by-product at scratch +
@@ -257,7 +265,7 @@ bool attention_tc_eligible(int dtype, int head_dim, int ldq, int ldkv);
 size_t score_scratch_floats(int n_seqs, int n_total, int n_heads);
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                  const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
-                 int n_heads, int head_dim, float *scratch, float *scores);
+                 int n_heads, int head_dim, float *scratch, float *scores, int n_kv_heads = 0);
 // General form (decode): sequence s scores the key LIST key_rows[cu_q[s] .. cu_q[s+1]) (cache rows)
 // with the query in row q_rows[s].
 int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, const int32_t *cu_q,
@@ -270,7 +278,7 @@ int launch_attention_decode(cudaStream_t st, const void *q, int ldq, const void 
                             int ldkv, void *o, int ldo, const int32_t *cu_x, const int32_t *cu_ctx,
                             const int32_t *ctx_rows, const int32_t *q_kvlen, const int32_t *score_row,
                             int n_seqs, int n_rows, int n_ctx_total, int max_ctx, int n_heads,
-                            float *part, float *logits, float *stats);
+                            float *part, float *logits, float *stats, int n_kv_heads = 0);
 int launch_attention_combine(cudaStream_t st, const float *part_o, const float *part_ml, int n_splits,
                              const int32_t *cu_x, const int32_t *score_row, int n_seqs, int n_rows, int n_heads,
                              void *o, int ldo, float *stats);
@@ -280,11 +288,12 @@ int attention_list_splits(int n_seqs, int max_rows, int n_heads, int max_ctx);
 int launch_attention_list_split(cudaStream_t st, const void *q, int ldq, const void *k, const void *v, int ldkv,
                                 void *o, const int32_t *cu_q, const int32_t *cu_kv, const int32_t *kv_idx,
                                 const int32_t *q_kvlen, const int32_t *score_row, int n_seqs, int max_rows,
-                                int n_total, int n_heads, int n_splits, float *part, float *stats);
+                                int n_total, int n_heads, int n_splits, float *part, float *stats,
+                                int n_kv_heads = 0);
 int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                     const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
                     const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,
-                    int head_dim, float *scratch, float *scores);
+                    int head_dim, float *scratch, float *scores, int n_kv_heads = 0);
 int launch_select_threshold(cudaStream_t st, const float *scores, const int32_t *cu_in, int n_seqs,
                             uint32_t prune_bp, int32_t *keep_idx, int32_t *drop_idx, int32_t *counts);
 // counts[s] = rows of sequence s whose score is not smaller than its (cu_keep[s+1] - cu_keep[s])-th largest

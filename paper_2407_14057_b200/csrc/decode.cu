@@ -252,6 +252,7 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
   if (!status) return LAZY_E_CUDA;
   const long long launches0 = g_launches;
   const int S = c->n_seqs, L = c->L, d = c->d, dt = c->dtype, KV = c->cap_kv;
+  const int dkv = c->dkv, qc = c->qkv_cols;
   const size_t rb = c->row_bytes();
   for (int s = 0; s < S; ++s) {
     if (c->n_tokens[s] + 1 > c->prompt_len[s] + c->cfg.max_new_tokens) return LAZY_E_CAPACITY;
@@ -323,8 +324,8 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
 
   char *x = c->x, *x2 = c->x2;
   for (int l = 0; l < L; ++l) {
-    char *kc = c->kcache + (size_t)l * KV * rb;
-    char *vc = c->vcache + (size_t)l * KV * rb;
+    char *kc = c->kcache + (size_t)l * KV * c->kv_row_bytes();
+    char *vc = c->vcache + (size_t)l * KV * c->kv_row_bytes();
     int32_t *kvp = c->kv_pos + (size_t)l * KV;
     int32_t *kvm = c->kv_map + (size_t)l * KV;
     float *sc = c->scores + (size_t)l * KV;
@@ -345,21 +346,21 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
                           ctx_rows, status));
       KLAUNCH_OK();
     }
-    if (gemv_small_m_eligible(dt, M, d) && c->dh == 128) {
+    if (gemv_small_m_eligible(dt, M, d) && c->dh == 128 && dkv % 128 == 0) {
       // one to four rows: one weight-streaming kernel does RMSNorm, the projection, RoPE and the cache write
       LAZY_TRY(launch_gemv_qkv_rope(st, x, c->w_qkv[l], c->qkv, c->g_attn[l], c->cfg.rms_eps, xpos, c->rope_table,
-                                    kc, vc, kvp, kv_row_new, M, d, c->max_pos, status));
+                                    kc, vc, kvp, kv_row_new, M, d, c->max_pos, status, dkv));
     } else {
       if (gemv_small_m_eligible(dt, M, d)) {
-        LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, 3 * d, d, 0, c->g_attn[l],
+        LAZY_TRY(launch_gemv_small_m(st, x, c->w_qkv[l], nullptr, nullptr, c->qkv, M, qc, d, 0, c->g_attn[l],
                                      c->cfg.rms_eps, 0, true));
       } else {
         LAZY_TRY(launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, M, d, c->cfg.rms_eps));
-        LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, 3 * d, d, status, c->gemm_scratch,
+        LAZY_TRY(launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, M, qc, d, status, c->gemm_scratch,
                              c->gemm_scratch_bytes, 0, true));
       }
       LAZY_TRY(launch_rope_kv(st, dt, c->qkv, xpos, c->rope_table, kc, vc, kvp, kv_row_new, M, c->H, c->dh,
-                              c->max_pos, status));
+                              c->max_pos, status, c->Hkv));
     }
     for (int s = 0; s < S; ++s) c->kv_count[l][s] += m_of[s];
     int max_ctx = 0;
@@ -368,24 +369,24 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     if (attention_decode_eligible(dt, c->dh, M, max_ctx) &&
         attention_decode_scratch_floats(M, c->H, max_ctx) * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
       float *logits = c->score_scratch, *stats = c->score_scratch + (size_t)c->H * n_ctx;
-      LAZY_TRY(launch_attention_decode(st, c->qkv, 3 * d, kc, vc, d, c->attn, d, dtab(T_CU_X), dtab(T_CU_CTX),
+      LAZY_TRY(launch_attention_decode(st, c->qkv, qc, kc, vc, dkv, c->attn, d, dtab(T_CU_X), dtab(T_CU_CTX),
                                        ctx_rows, q_kvlen, dtab(T_QROW), S, M, n_ctx, max_ctx, c->H,
-                                       (float *)c->act, logits, stats));
+                                       (float *)c->act, logits, stats, c->Hkv));
       LAZY_TRY(launch_score_mean(st, logits, stats, dtab(T_CU_CTX), S, n_ctx, c->H, sc));
     } else {
       // many rows in flight: the tile kernel, with the key list cut into slices when there are too few
       // (query tile, head) pairs to fill the machine
       const int splits = attention_list_split_eligible(dt, c->dh) ? attention_list_splits(S, max_m, c->H, max_ctx) : 1;
       if (splits > 1 && (size_t)M * c->H * splits * 130 * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
-        LAZY_TRY(launch_attention_list_split(st, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), dtab(T_CU_CTX),
+        LAZY_TRY(launch_attention_list_split(st, c->qkv, qc, kc, vc, dkv, c->attn, dtab(T_CU_X), dtab(T_CU_CTX),
                                              ctx_rows, q_kvlen, dtab(T_QROW), S, max_m, M, c->H, splits,
-                                             (float *)c->act, c->score_scratch + (size_t)c->H * n_ctx));
+                                             (float *)c->act, c->score_scratch + (size_t)c->H * n_ctx, c->Hkv));
       } else {
-        LAZY_TRY(launch_attention_ex(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, dtab(T_CU_X), nullptr,
-                                     dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh));
+        LAZY_TRY(launch_attention_ex(st, dt, c->qkv, qc, kc, vc, dkv, c->attn, dtab(T_CU_X), nullptr,
+                                     dtab(T_CU_CTX), ctx_rows, q_kvlen, S, max_m, M, c->H, c->dh, c->Hkv));
       }
-      LAZY_TRY(launch_score_ex(st, dt, c->qkv, 3 * d, kc, d, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
-                               n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc));
+      LAZY_TRY(launch_score_ex(st, dt, c->qkv, qc, kc, dkv, dtab(T_CU_CTX), nullptr, ctx_rows, dtab(T_QROW), S,
+                               n_ctx, max_ctx, c->H, c->dh, c->score_scratch, sc, c->Hkv));
     }
     LAZY_TRY(launch_gemm(st, dt, c->attn, c->w_o[l], x, x, M, d, d, status, c->gemm_scratch, c->gemm_scratch_bytes, 0,
                          true));

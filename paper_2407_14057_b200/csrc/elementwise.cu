@@ -276,11 +276,11 @@ template <typename T>
 __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ pos,
                                const float2 *__restrict__ table, T *__restrict__ kcache,
                                T *__restrict__ vcache, int32_t *__restrict__ kv_pos,
-                               const int32_t *__restrict__ kv_row, int n_heads, int head_dim,
+                               const int32_t *__restrict__ kv_row, int n_heads, int n_kv_heads, int head_dim,
                                int max_pos, DevStatus *status) {
   constexpr int V = Elem<T>::kPerVec;
   const int r = blockIdx.x;
-  const int d = n_heads * head_dim;
+  const int d = n_heads * head_dim, dkv = n_kv_heads * head_dim;  // a row of qkv = [q: d | k: dkv | v: dkv]
   const int half = head_dim / 2;
   int p = pos[r];
   if (p < 0 || p >= max_pos) {
@@ -288,14 +288,14 @@ __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ 
     p = 0;
   }
   const size_t krow = kv_row ? (size_t)kv_row[r] : (size_t)r;
-  T *row = qkv + (size_t)r * 3 * d;
+  T *row = qkv + (size_t)r * (d + 2 * dkv);
   const float2 *tab = table + (size_t)p * half;
   const int vec_per_half = half / V;
-  const int pairs = n_heads * vec_per_half;  // vector pairs per q (and per k)
+  const int pairs_q = n_heads * vec_per_half, pairs_k = n_kv_heads * vec_per_half;  // vector pairs of q, of k
   const int tid = blockIdx.y * blockDim.x + threadIdx.x, tstep = gridDim.y * blockDim.x;
-  for (int t = tid; t < 2 * pairs; t += tstep) {
-    const int which = t / pairs;  // 0 = q, 1 = k
-    const int u = t - which * pairs;
+  for (int t = tid; t < pairs_q + pairs_k; t += tstep) {
+    const int which = t >= pairs_q;  // 0 = q, 1 = k
+    const int u = t - which * pairs_q;
     const int h = u / vec_per_half;
     const int i0 = (u - h * vec_per_half) * V;
     T *base = row + which * d + h * head_dim;
@@ -317,29 +317,30 @@ __global__ void rope_kv_kernel(T *__restrict__ qkv, const int32_t *__restrict__ 
       a.store(base + i0);
       b.store(base + half + i0);
     } else {
-      T *kd = kcache + krow * d + h * head_dim;
+      T *kd = kcache + krow * dkv + h * head_dim;
       a.store(kd + i0);
       b.store(kd + half + i0);
     }
   }
-  const uint4 *vs = reinterpret_cast<const uint4 *>(row + 2 * d);
-  uint4 *vd = reinterpret_cast<uint4 *>(vcache + krow * d);
-  for (int i = tid; i < d / V; i += tstep) vd[i] = vs[i];
+  const uint4 *vs = reinterpret_cast<const uint4 *>(row + d + dkv);
+  uint4 *vd = reinterpret_cast<uint4 *>(vcache + krow * dkv);
+  for (int i = tid; i < dkv / V; i += tstep) vd[i] = vs[i];
   if (tid == 0 && kv_pos) kv_pos[krow] = p;
 }
 
 int launch_rope_kv(cudaStream_t st, int dtype, void *qkv, const int32_t *pos, const float *table,
                    void *kcache, void *vcache, int32_t *kv_pos, const int32_t *kv_row, int n,
-                   int n_heads, int head_dim, int max_pos, DevStatus *status) {
+                   int n_heads, int head_dim, int max_pos, DevStatus *status, int n_kv_heads) {
   if (n == 0) return LAZY_OK;
+  if (n_kv_heads <= 0) n_kv_heads = n_heads;
   const dim3 grid(n, n <= 16 ? 8 : 1);  // a handful of rows (decode): spread each over several CTAs
   if (dtype == LAZY_F32)
     rope_kv_kernel<float><<<grid, 128, 0, st>>>((float *)qkv, pos, (const float2 *)table,
                                              (float *)kcache, (float *)vcache, kv_pos, kv_row,
-                                             n_heads, head_dim, max_pos, status);
+                                             n_heads, n_kv_heads, head_dim, max_pos, status);
   else
     rope_kv_kernel<bf16><<<grid, 128, 0, st>>>((bf16 *)qkv, pos, (const float2 *)table, (bf16 *)kcache,
-                                            (bf16 *)vcache, kv_pos, kv_row, n_heads, head_dim,
+                                            (bf16 *)vcache, kv_pos, kv_row, n_heads, n_kv_heads, head_dim,
                                             max_pos, status);
   LAZY_COUNT_LAUNCH();
   return launch_ok();

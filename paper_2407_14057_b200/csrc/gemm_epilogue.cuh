@@ -21,6 +21,7 @@ struct RopeArgs {
   int32_t *kv_pos;        // position tag per cache row (may be NULL)
   const int32_t *kv_row;  // cache row of GEMM row r (NULL: r)
   int d_model, max_pos;
+  int d_kv;               // width of a K / V cache row: n_kv_heads * head_dim (= d_model without grouping)
 };
 
 // ---- the last, partial wave ------------------------------------------------------------------------------
@@ -238,8 +239,9 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
   bf16 *crow = C + (size_t)row * ldc;
   if (EPI == EPI_QKV_ROPE) {
     // section of the fused projection this tile belongs to: 0 = q, 1 = k, 2 = v
-    const int sect = n0 / rope.d_model;
-    const int col_in = n0 - sect * rope.d_model;
+    // output columns are [q: d_model | k: d_kv | v: d_kv]
+    const int sect = n0 < rope.d_model ? 0 : (n0 < rope.d_model + rope.d_kv ? 1 : 2);
+    const int col_in = n0 - (sect == 0 ? 0 : (sect == 1 ? rope.d_model : rope.d_model + rope.d_kv));
     int p = 0;
     size_t krow = 0;
     if (row < M) {
@@ -251,7 +253,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       krow = rope.kv_row ? (size_t)rope.kv_row[row] : (size_t)row;
     }
     bf16 *dst = sect == 0 ? crow + n0
-                          : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_model + col_in;
+                          : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_kv + col_in;
     if (sect == 2) {
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {

@@ -317,16 +317,19 @@ bool gemm_res_rows_supported(int dtype, int M, int K) {
   return dtype == LAZY_BF16 && !gemv_small_m_eligible(dtype, M, K);
 }
 
-bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim) {
-  return dtype == LAZY_BF16 && head_dim == 128 && d_model % BN == 0;
+bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim, int d_kv) {
+  if (d_kv <= 0) d_kv = d_model;
+  return dtype == LAZY_BF16 && head_dim == 128 && d_model % BN == 0 && d_kv % BN == 0;
 }
 
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
-                         void *scratch, size_t scratch_bytes) {
+                         void *scratch, size_t scratch_bytes, int d_kv) {
   if (M == 0) return LAZY_OK;
+  if (d_kv <= 0) d_kv = d_model;
   RopeArgs r;
+  r.d_kv = d_kv;
   r.pos = pos;
   r.table = (const float2 *)table;
   r.kcache = (bf16 *)kcache;
@@ -335,7 +338,7 @@ int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void
   r.kv_row = kv_row;
   r.d_model = d_model;
   r.max_pos = max_pos;
-  return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, 3 * d_model, d_model, status, r, scratch,
+  return launch_tc<EPI_QKV_ROPE>(st, h, w_qkv, w_qkv, nullptr, qkv, M, d_model + 2 * d_kv, d_model, status, r, scratch,
                                  scratch_bytes, 0);
 }
 

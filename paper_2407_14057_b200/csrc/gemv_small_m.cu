@@ -32,18 +32,21 @@ struct GemvRope {
   int32_t *kv_pos;        // position tag per cache row
   const int32_t *kv_row;  // cache row of input row m
   int d_model, max_pos;
+  int d_kv;               // width of a K / V cache row (n_kv_heads * 128)
   DevStatus *status;
 };
 
 // The weight rows a warp streams for its n-th task.  Plain: output column n.  SwiGLU: gate row n and up
 // row n.  QKV: task n = (section q/k/v, head, i < 64) -> rows of output columns i and i + 64 of that head.
 template <int MODE>
-__device__ __forceinline__ void gv_task_rows(int n, const bf16 *B0, const bf16 *B1, int K, int d_model,
+__device__ __forceinline__ void gv_task_rows(int n, const bf16 *B0, const bf16 *B1, int K, int d_model, int d_kv,
                                              const uint4 *&w0, const uint4 *&w1, int &col0) {
   if (MODE == GV_QKV_ROPE) {
-    const int half_d = d_model >> 1;
-    const int sect = n / half_d, u = n - sect * half_d;
-    col0 = sect * d_model + (u >> 6) * 128 + (u & 63);
+    // d_model / 2 tasks for q, then d_kv / 2 each for k and v
+    const int tq = d_model >> 1, tk = d_kv >> 1;
+    const int sect = n < tq ? 0 : (n < tq + tk ? 1 : 2);
+    const int u = n - (sect == 0 ? 0 : (sect == 1 ? tq : tq + tk));
+    col0 = (sect == 0 ? 0 : (sect == 1 ? d_model : d_model + d_kv)) + (u >> 6) * 128 + (u & 63);
     w0 = reinterpret_cast<const uint4 *>(B0 + (size_t)col0 * K);
     w1 = reinterpret_cast<const uint4 *>(B0 + (size_t)(col0 + 64) * K);
   } else {
@@ -74,7 +77,7 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   if (n_first < N) {
     const uint4 *w0, *w1;
     int col0;
-    gv_task_rows<MODE>(n_first, B0, B1, K, rope.d_model, w0, w1, col0);
+    gv_task_rows<MODE>(n_first, B0, B1, K, rope.d_model, rope.d_kv, w0, w1, col0);
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int v = lane + 32 * u;
@@ -132,7 +135,7 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
   for (int n = blockIdx.x * (GV_THREADS / 32) + warp; n < N; n += warps_total) {
     const uint4 *w0, *w1;
     int col0;
-    gv_task_rows<MODE>(n, B0, B1, K, rope.d_model, w0, w1, col0);
+    gv_task_rows<MODE>(n, B0, B1, K, rope.d_model, rope.d_kv, w0, w1, col0);
     float acc0[M_ROWS], acc1[M_ROWS];
 #pragma unroll
     for (int m = 0; m < M_ROWS; ++m) acc0[m] = acc1[m] = 0.f;
@@ -183,7 +186,9 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
       float u = SWIGLU ? warp_sum(acc1[m]) : 0.f;
       if (MODE == GV_QKV_ROPE) {
         if (lane == 0) {
-          const int d = rope.d_model, sect = col0 / d, cin = col0 - sect * d;  // cin: column i of its head
+          const int d = rope.d_model, dkv = rope.d_kv;
+          const int sect = col0 < d ? 0 : (col0 < d + dkv ? 1 : 2);
+          const int cin = col0 - (sect == 0 ? 0 : (sect == 1 ? d : d + dkv));  // column inside q, k or v
           int p = rope.pos[m];
           if (p < 0 || p >= rope.max_pos) {
             dev_fail(rope.status, LAZY_E_CAPACITY, W_ROPE_POS, m, p);
@@ -196,8 +201,8 @@ gemv_small_m_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ B0, con
             o1 = u * cs.x + g * cs.y;
           }
           const size_t krow = (size_t)rope.kv_row[m];
-          bf16 *dst = sect == 0 ? reinterpret_cast<bf16 *>(C) + (size_t)m * 3 * d + cin
-                                : (sect == 1 ? rope.kcache : rope.vcache) + krow * d + cin;
+          bf16 *dst = sect == 0 ? reinterpret_cast<bf16 *>(C) + (size_t)m * (d + 2 * dkv) + cin
+                                : (sect == 1 ? rope.kcache : rope.vcache) + krow * dkv + cin;
           dst[0] = __float2bfloat16_rn(o0);
           dst[64] = __float2bfloat16_rn(o1);
           if (n == 0) rope.kv_pos[krow] = p;
@@ -272,9 +277,10 @@ int launch_gemv_small_m(cudaStream_t st, const void *A, const void *B0, const vo
 // decode step calls this, with the context's own (constant) weights: always a programmatic dependent.
 int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void *qkv, const void *gain, float eps,
                          const int32_t *pos, const float *table, void *kcache, void *vcache, int32_t *kv_pos,
-                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status) {
+                         const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status, int d_kv) {
+  if (d_kv <= 0) d_kv = d_model;
   if (((uintptr_t)x & 15) || ((uintptr_t)w_qkv & 15) || ((uintptr_t)gain & 15) || !pos || !table || !kcache ||
-      !vcache || !kv_pos || !kv_row || (d_model % 128))
+      !vcache || !kv_pos || !kv_row || (d_model % 128) || (d_kv % 128))
     return LAZY_E_BADARG;
   GemvRope r;
   r.pos = pos;
@@ -284,9 +290,10 @@ int launch_gemv_qkv_rope(cudaStream_t st, const void *x, const void *w_qkv, void
   r.kv_pos = kv_pos;
   r.kv_row = kv_row;
   r.d_model = d_model;
+  r.d_kv = d_kv;
   r.max_pos = max_pos;
   r.status = status;
-  const int tasks = 3 * d_model / 2;
+  const int tasks = (d_model + 2 * d_kv) / 2;
 #define GV_CASE(m) \
   case m: return launch_one<m, GV_QKV_ROPE>(st, x, w_qkv, nullptr, nullptr, qkv, tasks, d_model, gain, eps, 0, true, r);
   switch (M) {

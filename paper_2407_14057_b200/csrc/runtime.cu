@@ -93,6 +93,7 @@ int validate_cfg(const lazy_model_cfg *c) {
       c->head_dim < 1 || c->d_ffn < 1 || c->vocab < 1)
     return LAZY_E_BADARG;
   if (c->n_heads * c->head_dim != c->d_model) return LAZY_E_BADARG;
+  if (c->n_kv_heads < 0 || (c->n_kv_heads > 0 && c->n_heads % c->n_kv_heads)) return LAZY_E_BADARG;
   if (c->dtype != LAZY_BF16 && c->dtype != LAZY_F32) return LAZY_E_BADARG;
   // 16-byte vectors everywhere; RoPE pairs 16-byte vectors of the two halves of a head;
   // the generic attention kernel gives each lane head_dim/32 output columns.
@@ -143,7 +144,7 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->x = k.take(R * rb);
   c->x2 = k.take(R * rb);
   c->h = k.take(R * rb);
-  c->qkv = k.take(R * rb * 3);
+  c->qkv = k.take(R * (size_t)c->qkv_cols * c->eb);
   c->attn = k.take(R * rb);
   c->act = k.take(R * (size_t)c->F * c->eb);
   c->h_last = k.take((size_t)c->S * rb);
@@ -174,8 +175,8 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->revived_pos.assign(P, nullptr);
   for (int p = 0; p < P; ++p) c->revived_pos[p] = (int32_t *)k.take(KV * 4);
   c->rope_table = (float *)k.take((size_t)c->max_pos * c->dh * 4);
-  c->kcache = k.take((size_t)L * KV * rb);
-  c->vcache = k.take((size_t)L * KV * rb);
+  c->kcache = k.take((size_t)L * KV * c->kv_row_bytes());
+  c->vcache = k.take((size_t)L * KV * c->kv_row_bytes());
   c->kv_pos = (int32_t *)k.take((size_t)L * KV * 4);
   c->aux_rows = k.take((size_t)P * KV * rb);
   c->aux_pos = (int32_t *)k.take((size_t)P * KV * 4);
@@ -197,6 +198,9 @@ static void fill_shape(lazy_ctx *c, const lazy_model_cfg *cfg, const lazy_schedu
   c->d = cfg->d_model;
   c->H = cfg->n_heads;
   c->dh = cfg->head_dim;
+  c->Hkv = cfg->n_kv_heads > 0 ? cfg->n_kv_heads : cfg->n_heads;
+  c->dkv = c->Hkv * cfg->head_dim;
+  c->qkv_cols = cfg->d_model + 2 * c->dkv;
   c->F = cfg->d_ffn;
   c->V = cfg->vocab;
   c->dtype = cfg->dtype;
@@ -405,7 +409,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   if (!status) return LAZY_E_CUDA;
   const long long launches0 = g_launches;
   const int P = c->P, L = c->L, d = c->d, dt = c->dtype;
-  const size_t rb = c->row_bytes();
+  const int dkv = c->dkv, qc = c->qkv_cols;
+  const size_t rb = c->row_bytes(), kvb = c->kv_row_bytes();
   LAZY_TRY(reset_gemm_counters(c, st));
   c->ev_kind.clear();
   c->ev_flops.clear();
@@ -495,8 +500,8 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
   for (int l = 0; l < L; ++l) {
     const int n = c->seg_cu[g][n_seqs];
     const int32_t *pos = c->pos_seg[g];
-    char *kc = c->kcache + (size_t)l * c->cap_kv * rb;
-    char *vc = c->vcache + (size_t)l * c->cap_kv * rb;
+    char *kc = c->kcache + (size_t)l * c->cap_kv * kvb;
+    char *vc = c->vcache + (size_t)l * c->cap_kv * kvb;
     int32_t *kvp = c->kv_pos + (size_t)l * c->cap_kv;
     float *sc = c->scores + (size_t)l * c->cap_kv;
     int seg_max = 0;
@@ -514,21 +519,21 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       attn_flops += 2.0 * d * ns * (ns + 1.0);
     }
     TIMED(LAZY_K_RMSNORM, 0, 2.0 * n * rb, launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
-    if (gemm_qkv_rope_eligible(dt, d, c->dh)) {
+    if (gemm_qkv_rope_eligible(dt, d, c->dh, dkv)) {
       // rotary embedding and the K/V cache write ride in the projection's epilogue
-      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
+      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
             launch_gemm_qkv_rope(st, c->h, c->w_qkv[l], c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n,
-                                 d, c->max_pos, status, c->gemm_scratch, c->gemm_scratch_bytes));
+                                 d, c->max_pos, status, c->gemm_scratch, c->gemm_scratch_bytes, dkv));
     } else {
-      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * 3 * d * d, 0,
-            launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, 3 * d, d, status, c->gemm_scratch,
+      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
+            launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, qc, d, status, c->gemm_scratch,
                         c->gemm_scratch_bytes));
       TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
             launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
-                           c->max_pos, status));
+                           c->max_pos, status, c->Hkv));
     }
     bool fused_score = false;
-    if (attention_tc_eligible(dt, c->dh, 3 * d, d)) {
+    if (attention_tc_eligible(dt, c->dh, qc, dkv)) {
       // Eq. 1 comes from the last row's softmax numerators, which the attention kernel leaves in this layer's
       // slice of the score scratch; the head means of all layers since the previous cut are taken in one
       // launch when the next cut (or the end of the prefill) needs them.
@@ -538,9 +543,10 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
         const int q0 = c->seg_cu[g][s], ns = c->seg_cu[g][s + 1] - q0;
         const double fl = 2.0 * d * (double)ns * (ns + 1.0);
         TIMED(LAZY_K_ATTENTION, fl, 0,
-              launch_attention_tc(st, c->qkv, 3 * d, q0 + ns, kc, vc, d, c->seq_base[s] + ns, c->attn, c->H,
+              launch_attention_tc(st, c->qkv, qc, q0 + ns, kc, vc, dkv, c->seq_base[s] + ns, c->attn, c->H,
                                   nullptr, nullptr, 1, ns, q0, ns, c->seq_base[s], status,
-                                  c->score_scratch + (size_t)l * c->score_layer_stride, cdiv(seg_max, 64), n_seqs, s));
+                                  c->score_scratch + (size_t)l * c->score_layer_stride, cdiv(seg_max, 64), n_seqs, s,
+                                  c->Hkv));
       }
       fused_score = true;
       const bool last_of_group = c->point_at[l + 1] >= 0 || l == L - 1;
@@ -554,13 +560,13 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       }
     } else {
       TIMED(LAZY_K_ATTENTION, attn_flops, 0,
-            launch_attention(st, dt, c->qkv, 3 * d, kc, vc, d, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
-                             c->H, c->dh));
+            launch_attention(st, dt, c->qkv, qc, kc, vc, dkv, c->attn, d_cu(g), d_base, n_seqs, seg_max, n,
+                             c->H, c->dh, c->Hkv));
     }
     if (!fused_score)
       TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
-            launch_score(st, dt, c->qkv, 3 * d, kc, d, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
-                         c->score_scratch, sc));
+            launch_score(st, dt, c->qkv, qc, kc, dkv, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
+                         c->score_scratch, sc, c->Hkv));
     TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status,
                                                       c->gemm_scratch, c->gemm_scratch_bytes, 0, true));
 
@@ -761,7 +767,7 @@ int lazy_get_kv(lazy_ctx *c, void *stream, int32_t layer, int32_t seq, int32_t *
   if (!c->have_prefill) return LAZY_E_STATE;
   if (seq >= c->n_seqs) return LAZY_E_BADARG;
   const int cnt = c->kv_count[layer][seq];
-  const size_t rb = c->row_bytes();
+  const size_t rb = c->kv_row_bytes();  // K / V rows: n_kv_heads * head_dim wide
   const size_t row0 = (size_t)layer * c->cap_kv + c->seq_base[seq];
   if (h_count) *h_count = cnt;
   cudaStream_t st = (cudaStream_t)stream;

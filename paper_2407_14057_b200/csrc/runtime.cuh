@@ -11,6 +11,7 @@
 struct lazy_ctx {
   lazy_model_cfg cfg;
   int L, d, H, dh, F, V, dtype, eb;
+  int Hkv, dkv, qkv_cols;  // key/value heads, width of a K / V cache row, width of a row of the fused projection
   int P;  // schedule points
   std::vector<int> sched_layer;
   std::vector<uint32_t> sched_bp;
@@ -89,6 +90,7 @@ struct lazy_ctx {
   ~lazy_ctx();
 
   size_t row_bytes() const { return (size_t)d * eb; }
+  size_t kv_row_bytes() const { return (size_t)dkv * eb; }
   int seg_of_layer(int l) const {  // segment whose rows enter layer l
     int g = 0;
     for (int p = 0; p < P; ++p)

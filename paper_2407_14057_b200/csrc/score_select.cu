@@ -25,7 +25,7 @@ __global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *_
                                     const int32_t *__restrict__ kv_base,
                                     const int32_t *__restrict__ key_rows,
                                     const int32_t *__restrict__ q_rows, int n_total, int head_dim,
-                                    float *__restrict__ logits) {
+                                    float *__restrict__ logits, int kv_group) {
   constexpr int V = Elem<T>::kPerVec;
   const int seq = blockIdx.z, h = blockIdx.y;
   const int q_start = cu_q[seq];
@@ -57,7 +57,7 @@ __global__ void score_logits_kernel(const T *__restrict__ q, int ldq, const T *_
     if (j < j_end) {
       Vec16<T> kv;
       const size_t krow = key_rows ? (size_t)key_rows[q_start + j] : kb + j;
-      kv.load(k + krow * ldkv + h * head_dim + sub * V);
+      kv.load(k + krow * ldkv + (h / kv_group) * head_dim + sub * V);
       float kf[V];
       kv.unpack(kf);
 #pragma unroll
@@ -398,16 +398,18 @@ size_t score_scratch_floats(int n_seqs, int n_total, int n_heads) {
 
 int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                  const int32_t *cu_q, const int32_t *kv_base, int n_seqs, int n_total, int max_len,
-                 int n_heads, int head_dim, float *scratch, float *scores) {
+                 int n_heads, int head_dim, float *scratch, float *scores, int n_kv_heads) {
   return launch_score_ex(st, dtype, q, ldq, k, ldkv, cu_q, kv_base, nullptr, nullptr, n_seqs, n_total,
-                         max_len, n_heads, head_dim, scratch, scores);
+                         max_len, n_heads, head_dim, scratch, scores, n_kv_heads);
 }
 
 int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const void *k, int ldkv,
                     const int32_t *cu_q, const int32_t *kv_base, const int32_t *key_rows,
                     const int32_t *q_rows, int n_seqs, int n_total, int max_len, int n_heads,
-                    int head_dim, float *scratch, float *scores) {
+                    int head_dim, float *scratch, float *scores, int n_kv_heads) {
   if (n_total == 0 || n_seqs == 0) return LAZY_OK;
+  const int kv_group = kv_group_of(n_heads, n_kv_heads);
+  if (kv_group < 1) return LAZY_E_BADARG;
   const int V = dtype == LAZY_F32 ? 4 : 8;
   const int lpk = head_dim / V;
   if (head_dim % V || lpk < 1 || lpk > 32 || (lpk & (lpk - 1))) return LAZY_E_BADARG;
@@ -419,11 +421,11 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
   if (dtype == LAZY_F32)
     score_logits_kernel<float><<<grid, threads, 0, st>>>((const float *)q, ldq, (const float *)k, ldkv,
                                                          cu_q, kv_base, key_rows, q_rows, n_total, head_dim,
-                                                         logits);
+                                                         logits, kv_group);
   else
     score_logits_kernel<bf16><<<grid, threads, 0, st>>>((const bf16 *)q, ldq, (const bf16 *)k, ldkv,
                                                         cu_q, kv_base, key_rows, q_rows, n_total, head_dim,
-                                                        logits);
+                                                        logits, kv_group);
   LAZY_COUNT_LAUNCH();
   score_stats_kernel<<<dim3(n_heads, n_seqs), 256, 0, st>>>(logits, cu_q, n_total, n_heads, stats);
   LAZY_COUNT_LAUNCH();

@@ -222,3 +222,14 @@ def test_decode_errors():
         eng.lazy_decode_step(tok, lg, None)                # caches were sized for one new token
     assert e.value.status == -3
     eng.close()
+
+
+def test_decode_grouped_query_attention():
+    """Decode steps with revival on 2 key/value heads for 4 query heads: fp32 generic kernels, then the bf16
+    weight-streaming path (RoPE and cache write in the QKV kernel's epilogue) and split-key attention."""
+    rv = run_decode_case(synth.TINY.with_layers(3).with_kv_heads(2), ((1, 6000), (2, 3000)), [60, 25], torch.float32,
+                         seed=14, steps=4)
+    assert rv > 0
+    rv = run_decode_case(synth.SMALL.with_kv_heads(2), ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16,
+                         seed=15, steps=4)
+    assert rv > 0

@@ -360,3 +360,28 @@ def test_threshold_selection_equals_count_selection_without_ties_bf16():
         eng.close()
     assert all(np.array_equal(a, b) for a, b in zip(out[0][1], out[1][1]))
     assert torch.equal(out[0][0], out[1][0])
+
+
+# ----------------------------------------------------------------------------- grouped-query attention
+def test_grouped_query_attention_prefill_fp32():
+    """Fewer key/value heads than query heads (2 of 4, then 1 of 4): the whole pruned prefill against the
+    oracle on the generic fp32 kernels, varlen batch included; caches hold key/value heads only."""
+    for kvh in (2, 1):
+        shape = synth.TINY.with_layers(3).with_kv_heads(kvh)
+        run_model_case(shape, ((1, 6000), (2, 3000)), [90, 1, 47], torch.float32, seed=30 + kvh)
+
+
+def test_grouped_query_attention_prefill_bf16_tensor_cores():
+    """head_dim 128, 4 query heads on 2 key/value heads: QKV projection with RoPE and the cache write in its
+    epilogue over [q | k | v] sections of different widths, tcgen05 attention reading key/value head h // 2."""
+    shape = synth.SMALL.with_kv_heads(2)
+    run_model_case(shape, ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16, seed=33)
+    run_model_case(shape.with_layers(3), ((1, 6000), (2, 3000)), [200, 65, 1, 131], torch.bfloat16, seed=34)
+
+
+def test_grouped_query_attention_wide_shape_bf16():
+    """Two layers of a 7B-class grouped shape (d=4096, 32 query heads on 8 key/value heads, ffn 11008), 700-token
+    prompt with a cut: the widths at which the fused projection is 6144 columns wide and the caches 1024."""
+    shape = synth.ModelShape(n_layers=2, d_model=4096, n_heads=32, head_dim=128, d_ffn=11008, vocab=4096,
+                             n_kv_heads=8)
+    run_model_case(shape, ((1, 5000),), [700], torch.bfloat16, seed=35, perturb=False)
