@@ -190,6 +190,55 @@ def select_threshold(scores: np.ndarray, prune_bp: int) -> Tuple[np.ndarray, np.
     return keep, drop
 
 
+# --------------------------------------------------------------------------- fp8 projections
+# Optional 8-bit mode of the four projections of a layer (QKV, output, gate/up, down): both operands of the
+# product are e4m3 numbers (4 exponent bits, 3 mantissa bits, largest finite value 448, no infinities) times
+# a scale.  Weights arrive already rounded (a per-matrix scale folded in by whoever made them: the oracle is
+# handed the de-quantised values).  Activations are quantised per ROW on the way into the product, in the
+# arithmetic the CUDA path uses for the decision (float32): scale = max|x| / 448 (1 for an all-zero row),
+# code = round-to-nearest-even of x / scale onto the e4m3 grid.  The product itself is exact (float64) here.
+E4M3_MAX = 448.0
+
+
+def round_e4m3(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest e4m3 number (ties to even), saturating at +-448.  Written out on
+    the bit level: 3 mantissa bits above 2^-6 (normal numbers), a fixed step of 2^-9 below (subnormals)."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.minimum(np.abs(x).astype(np.float64), E4M3_MAX)
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)                               # below 2^-6 the grid no longer refines
+    step = np.exp2(e - 3.0)                               # 8 steps per binade
+    q = np.round(a / step) * step                         # numpy rounds halves to even
+    q = np.minimum(q, E4M3_MAX)
+    return (np.sign(x) * q).astype(np.float32)
+
+
+def quant_rows_e4m3(x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Per-row e4m3 quantisation of activations.  Returns (codes as float32 values on the e4m3 grid,
+    scale per row as float32); the de-quantised activation is codes * scale."""
+    x32 = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x32), axis=-1, keepdims=True)
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    codes = round_e4m3((x32 / scale).astype(np.float32))
+    return codes, scale[..., 0]
+
+
+def _bf16_round(x: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 (ties to even) of every element, as float32."""
+    u = np.ascontiguousarray(np.asarray(x, dtype=np.float32)).view(np.uint32)
+    r = ((u >> np.uint32(16)) & np.uint32(1)) + np.uint32(0x7FFF)
+    return ((u + r) & np.uint32(0xFFFF0000)).view(np.float32)
+
+
+def _linear(cfg, x, w):
+    """x @ w^T.  With cfg.fp8 the activation rows are quantised to e4m3 first (see above), from their
+    bfloat16 values: that is what the CUDA path holds when it takes the rounding decisions."""
+    if getattr(cfg, "fp8", False):
+        codes, scale = quant_rows_e4m3(_bf16_round(x))
+        x = f64(codes) * f64(scale)[..., None]
+    return f64(x) @ f64(w).T
+
+
 def kv_heads(cfg) -> int:
     """Key/value heads of the shape (grouped-query attention when fewer than the query heads)."""
     return int(getattr(cfg, "n_kv_heads", 0) or cfg.n_heads)
@@ -202,7 +251,7 @@ def _layer_qkv(cfg, lw, x, pos):
     Hkv = kv_heads(cfg)
     dkv = Hkv * dh
     h = rmsnorm(x, lw["g_attn"], cfg.rms_eps)
-    qkv = h @ f64(lw["w_qkv"]).T
+    qkv = _linear(cfg, h, lw["w_qkv"])
     n = x.shape[0]
     q = rope(qkv[:, :d].reshape(n, H, dh), pos, cfg.rope_theta)
     k = rope(qkv[:, d:d + dkv].reshape(n, Hkv, dh), pos, cfg.rope_theta)
@@ -210,15 +259,15 @@ def _layer_qkv(cfg, lw, x, pos):
     return q, k, v
 
 
-def _o_proj(o, lw):
+def _o_proj(cfg, o, lw):
     """Output projection of the concatenated heads."""
-    return o @ f64(lw["w_o"]).T
+    return _linear(cfg, o, lw["w_o"])
 
 
 def mlp(cfg, lw, x):
     """SwiGLU MLP of a pre-norm block: (silu(h Wg^T) * (h Wu^T)) Wd^T, h = rmsnorm(x)."""
     h = rmsnorm(x, lw["g_mlp"], cfg.rms_eps)
-    return (silu(h @ f64(lw["w_gate"]).T) * (h @ f64(lw["w_up"]).T)) @ f64(lw["w_down"]).T
+    return _linear(cfg, silu(_linear(cfg, h, lw["w_gate"])) * _linear(cfg, h, lw["w_up"]), lw["w_down"])
 
 
 def lm_head(cfg, W, x_row):
@@ -330,7 +379,7 @@ def prefill(cfg, W, ids, schedule, forced_keep: Optional[Dict[int, Sequence[int]
             cache.kv[int(p)] = (k[r], v[r])
         st._count(l, pos)
         o, s = attend(q, k, v, pos, pos, -1)
-        x = x + _o_proj(o, lw)
+        x = x + _o_proj(cfg, o, lw)
         if keep_records:
             st.scores.append(s)
             st.score_pos.append(pos.copy())
@@ -376,7 +425,7 @@ def layer_step(cfg, lw, x, pos, keep_pos: Optional[Sequence[int]] = None):
     pos = np.asarray(pos).astype(np.int64)
     q, k, v = _layer_qkv(cfg, lw, x, pos)
     o, s = attend(q, k, v, pos, pos, -1)
-    y = x + _o_proj(o, lw)
+    y = x + _o_proj(cfg, o, lw)
     if keep_pos is not None:
         want = set(int(p) for p in keep_pos)
         keep = np.asarray([r for r in range(len(pos)) if int(pos[r]) in want], dtype=np.int64)
@@ -434,7 +483,7 @@ def decode_step(cfg, W, st: LazyState, token_id: int,
         ctx = np.concatenate([T, np.asarray([p], dtype=np.int64)])
         kc, vc = cache.rows(ctx)
         o, s = attend(q, kc, vc, xpos, ctx, int(np.nonzero(xpos == p)[0][0]))
-        x = x + _o_proj(o, lw)
+        x = x + _o_proj(cfg, o, lw)
         st.scores.append(s)
         st.score_pos.append(ctx.copy())
         st.rows_pos.append(xpos.copy())
@@ -495,7 +544,7 @@ def prune_op(cfg, lw, x, pos, keep_bp: int, forced_keep_rows: Optional[Sequence[
     n = x.shape[0]
     q, k, v = _layer_qkv(cfg, lw, x, pos)
     o, s = attend(q, k, v, pos, pos, -1)
-    y = x + _o_proj(o, lw)
+    y = x + _o_proj(cfg, o, lw)
     if forced_keep_rows is not None:
         want = set(int(r) for r in forced_keep_rows)
         keep = np.asarray([r for r in range(n) if r in want], dtype=np.int64)

@@ -17,6 +17,7 @@ Stand-ins (no dataset or checkpoint is read):
 from __future__ import annotations
 
 import dataclasses
+import math
 from typing import Dict, List, Sequence, Tuple
 
 import torch
@@ -33,6 +34,7 @@ class ModelShape:
     rms_eps: float = 1e-6
     rope_theta: float = 1e4
     n_kv_heads: int = 0          # key/value heads; 0 = as many as query heads (no grouping)
+    fp8: bool = False            # the four projections of a layer multiply e4m3 operands
 
     @property
     def kv_heads(self) -> int:
@@ -40,6 +42,9 @@ class ModelShape:
 
     def with_kv_heads(self, n_kv_heads: int) -> "ModelShape":
         return dataclasses.replace(self, n_kv_heads=n_kv_heads)
+
+    def with_fp8(self, on: bool = True) -> "ModelShape":
+        return dataclasses.replace(self, fp8=on)
 
     def with_layers(self, n_layers: int) -> "ModelShape":
         return dataclasses.replace(self, n_layers=n_layers)
@@ -170,3 +175,26 @@ def make_scores(n: int, kind: str, seed: int) -> torch.Tensor:
     if kind == "random":
         return torch.rand(n, generator=g, dtype=torch.float32)
     raise ValueError(kind)
+
+
+PROJECTIONS = ("w_qkv", "w_o", "w_gate", "w_up", "w_down")
+
+
+def quantize_projections_e4m3(W: Dict[str, object]) -> Dict[str, object]:
+    """8-bit copies of the projection matrices of every layer: per matrix a power-of-two scale >= max|w| / 448
+    and the e4m3 codes of w / scale (torch's float8_e4m3fn cast: round to nearest even).  The bf16 / fp32
+    matrices in W are REPLACED by their de-quantised values codes * scale, which a power-of-two scale makes
+    exactly representable in bf16 (four significant bits), so the 8-bit path, the bf16 path and the oracle
+    all see the very same weights.  Returns {"layers": [{name: (codes as uint8, scale)}]}."""
+    out = {"layers": []}
+    for lw in W["layers"]:
+        q = {}
+        for name in PROJECTIONS:
+            w = lw[name].float()
+            amax = float(w.abs().max())
+            scale = 2.0 ** math.ceil(math.log2(amax / 448.0)) if amax > 0 else 1.0
+            codes = (w / scale).to(torch.float8_e4m3fn)
+            q[name] = (codes.view(torch.uint8), scale)
+            lw[name] = (codes.float() * scale).to(lw[name].dtype)
+        out["layers"].append(q)
+    return out

@@ -619,3 +619,67 @@ def test_threshold_prefill_equals_count_prefill_without_ties_and_keeps_all_ties(
     # decode keeps using the state's reading
     assert t.selection == "threshold"
     O.decode_step(shape, W, t, O.greedy(t.logits))
+
+
+# ----------------------------------------------------------------------------- e4m3 projections
+def test_round_e4m3_hand_worked_and_against_the_library_cast():
+    """e4m3: 3 mantissa bits, so 8 steps per binade; ties go to the even mantissa; largest value 448;
+    below 2^-6 the step stays 2^-9."""
+    x = np.array([0.3, 17.0, 19.0, 21.0, 448.0, 500.0, -1000.0, 1.0625, 1.1875, 2.0 ** -7, 2.0 ** -10, 0.0, -0.3],
+                 dtype=np.float32)
+    want = [0.3125, 16.0, 20.0, 20.0, 448.0, 448.0, -448.0, 1.0, 1.25, 2.0 ** -7, 2.0 ** -9 * 0.0, 0.0, -0.3125]
+    # 17 lies between 16 and 18: tie, even mantissa 000 -> 16; 19 between 18 (001) and 20 (010) -> 20;
+    # 21 between 20 and 22 (011): tie -> 20; 1.0625 between 1.0 and 1.125 -> 1.0; 1.1875 between 1.125 (001)
+    # and 1.25 (010) -> 1.25; 2^-10 is half a subnormal step: tie between 0 and 2^-9 -> 0 (even)
+    assert O.round_e4m3(x).tolist() == want
+    g = torch.Generator().manual_seed(5)
+    r = (torch.randn(20000, generator=g) * torch.logspace(-4, 2.5, 20000)).float()
+    r = r.clamp(-448, 448)
+    lib = r.to(torch.float8_e4m3fn).float().numpy()
+    assert np.array_equal(O.round_e4m3(r.numpy()), lib)
+
+
+def test_quant_rows_e4m3_properties():
+    rng = np.random.default_rng(9)
+    x = (rng.standard_normal((7, 96)) * rng.uniform(0.01, 30, (7, 1))).astype(np.float32)
+    x[3] = 0.0
+    codes, scale = O.quant_rows_e4m3(x)
+    assert scale[3] == 1.0 and np.all(codes[3] == 0)
+    for r in (0, 1, 2, 4, 5, 6):
+        assert scale[r] == np.float32(np.abs(x[r]).max()) / np.float32(448.0)
+        assert np.abs(codes[r]).max() == 448.0                       # the largest element lands on the top code
+        assert np.array_equal(codes[r], O.round_e4m3(x[r] / scale[r]))
+        assert np.max(np.abs(codes[r] * scale[r] - x[r])) <= np.abs(x[r]).max() / 448.0 * 16.0 + 1e-12   # half a top-binade step
+        rel = np.abs(codes[r] * scale[r] - x[r]) / np.abs(x[r]).clip(1e-30)
+        assert np.max(rel[np.abs(x[r]) > scale[r] * 2.0 ** -6]) <= 2.0 ** -4 + 1e-6        # 3 mantissa bits
+
+
+def test_fp8_mode_changes_only_the_projection_inputs():
+    """With fp8 on, every projection sees de-quantised e4m3 rows of its bf16 input and nothing else changes: a
+    layer computed by hand from the pieces equals layer_step, and the distance to the exact run is the
+    quantisation noise (a few per cent), not zero and not large."""
+    shape = MINI.with_fp8()
+    W = mini_weights(seed=33)
+    synth.quantize_projections_e4m3(W)
+    Wn = weights_to_np(W)
+    ids = to_np(synth.make_prompt(shape.vocab, 21, seed=33))
+    a = O.prefill(shape, Wn, ids, ((1, 5000),))
+    b = O.prefill(MINI, Wn, ids, ((1, 5000),))
+    d = rel_err(a.hidden_out[0], b.hidden_out[0])
+    assert 1e-4 < d < 0.2
+    lw = Wn["layers"][0]
+    x = O.f64(Wn["tok_embed"])[ids]
+    pos = np.arange(21)
+
+    def lin(v, w):
+        c, s = O.quant_rows_e4m3(O._bf16_round(v))
+        return (O.f64(c) * O.f64(s)[:, None]) @ O.f64(w).T
+    h = O.rmsnorm(x, lw["g_attn"], shape.rms_eps)
+    qkv = lin(h, lw["w_qkv"])
+    dm = shape.d_model
+    q = O.rope(qkv[:, :dm].reshape(21, 4, 16), pos, shape.rope_theta)
+    k = O.rope(qkv[:, dm:2 * dm].reshape(21, 4, 16), pos, shape.rope_theta)
+    v = qkv[:, 2 * dm:].reshape(21, 4, 16)
+    o, _ = O.attend(q, k, v, pos, pos, -1)
+    y = x + lin(o, lw["w_o"])
+    assert np.allclose(y, a.hidden_after_attn[0], rtol=0, atol=1e-12)
