@@ -361,6 +361,28 @@ def run_gpu(args):
     e2e_ms = max_over_ranks(e2e_ms, world, "cuda")
     eng.lazy_sync_status()
 
+    # the same two schedules with the projections on e4m3 operands (reported beside the 16-bit line, which stays
+    # the headline: the metric's dtype is bf16).  The 16-bit weights are replaced by the de-quantised e4m3
+    # values first, so this leg runs last.
+    fp8 = None
+    if not args.no_fp8 and shape.n_layers == 32:
+        q8 = synth.quantize_projections_e4m3(W)
+        for e_ in (eng, full):
+            e_.lazy_set_fp8_weights(q8)
+        ms8, _ = timed(eng, args.steps, 2)
+        ms8_full, _ = timed(full, max(2, args.steps // 2), 2)
+        _, k8, _ = timed(eng, ksteps, 1, timing=True, kinds=GEMM_KINDS)
+        g8_ms = sum(k8[k]["ms"] for k in GEMM_KINDS) / ksteps
+        g8_fl = sum(k8[k]["flops"] for k in GEMM_KINDS) / ksteps
+        fp8 = {"what": "QKV / output / gate-up / down projections on e4m3 codes (per-row activation scales, per-matrix "
+                       "weight scales, tcgen05 kind::f8f6f4), everything else bf16",
+               "ttft_ms_pruned": ms8, "ttft_ms_full_keep": ms8_full, "tokens_per_s": world * n / (ms8 * 1e-3),
+               "gemm_ms_per_step": g8_ms, "gemm_tflops": g8_fl / (g8_ms * 1e-3) / 1e12,
+               "frac_of_fp8_peak": g8_fl / (g8_ms * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops_sustained"]),
+               "fp8_peak_kind": "2 x the measured sustained bf16 figure (nominal ratio)"}
+        for e_ in (eng, full):
+            e_.lazy_set_fp8_weights(None)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -421,6 +443,8 @@ def run_gpu(args):
                      "traffic": _gemm_traffic()},
         "kernels": breakdown,
     }
+    if fp8:
+        out["fp8_projections"] = fp8
     if not args.no_cpu and world == 1:
         # the oracle, as it stands, on the machine's host cores.  By default on the whole workload (one run of
         # all layers over the full prompt: a measurement, a couple of minutes); --cpu-sample times the
@@ -584,13 +608,18 @@ def run_other_workload(args):
         # the HBM-bound steps alone; sources rotate over copies larger than L2 together
         srcs = [torch.randn((n, d), device="cuda").bfloat16() for _ in range(8)]
         idx = res["keep_idx"][:n_keep].contiguous()
-        g_ms = _event_ms(lambda i: B.lazy_k_gather_rows(srcs[i % 8], idx), 40, 8)
+        g_out = torch.empty((n_keep, d), dtype=torch.bfloat16, device="cuda")
+        g_ms = _event_ms(lambda i: B.lazy_k_gather_rows(srcs[i % 8], idx, out=g_out), 40, 8)
         sc = synth.make_scores(n, "lognormal", 5).cuda()
         cu_in = torch.tensor([0, n], dtype=torch.int32).cuda()
         cu_keep = torch.tensor([0, n_keep], dtype=torch.int32).cuda()
-        s_ms = _event_ms(lambda i: B.lazy_k_select(sc, cu_in, cu_keep), 40, 8)
+        s_out = (torch.empty(n_keep, dtype=torch.int32, device="cuda"),
+                 torch.empty(n - n_keep, dtype=torch.int32, device="cuda"))
+        s_ms = _event_ms(lambda i: B.lazy_k_select(sc, cu_in, cu_keep, n, n_keep, s_out), 40, 8)
         qs = [torch.randn((n, d), device="cuda").bfloat16() for _ in range(8)]
-        k_ms = _event_ms(lambda i: B.lazy_k_score(qs[i % 8], d, srcs[i % 8], d, cu_in, n, H, dh), 40, 8)
+        nf = B.lib().lazy_k_score_scratch_floats(1, n, H)
+        k_out = (torch.empty(nf, dtype=torch.float32, device="cuda"), torch.empty(n, dtype=torch.float32, device="cuda"))
+        k_ms = _event_ms(lambda i: B.lazy_k_score(qs[i % 8], d, srcs[i % 8], d, cu_in, n, H, dh, out=k_out), 40, 8)
         B.lazy_device_status()
         gbs = 2.0 * n_keep * rb / (g_ms * 1e-3) / 1e9
         out.update({"rows": n, "kept": n_keep, "whole_op_ms": round(ms, 4),
@@ -665,6 +694,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="reduced depth (profiling captures only)")
     ap.add_argument("--prompt", type=int, default=N_PROMPT)
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the extra leg with e4m3 projections")
+    ap.add_argument("--fp8", action="store_true", help=argparse.SUPPRESS)   # the leg runs by default
     ap.add_argument("--cpu-sample", action="store_true",
                     help="time the oracle on the bounded sample only (about 15 s) instead of the whole workload")
     ap.add_argument("--workload", default="prefill", choices=["prefill", "decode", "batch8", "prune-op", "gemv", "gemm"],

@@ -224,6 +224,20 @@ int lazy_get_kernel_events(lazy_ctx *ctx, void *stream, int32_t cap, int32_t *ki
  * point in lazy_prefill_run, one more per point in lazy_decode_step).  Without ties both modes select the
  * same sets.  Takes effect with the next lazy_prefill_run / lazy_decode_step. */
 int lazy_set_selection(lazy_ctx *ctx, int32_t mode);
+/* 8-bit projections (no counterpart in the paper, which runs 16-bit weights; a deployment option for the
+ * "linear layers" of Section 3.1).  With fp8 weights set, lazy_prefill_run computes the four projections of
+ * every layer (QKV, output, gate/up, down) on e4m3 operands with fp32 accumulation: the weights are the e4m3
+ * codes given here times one scale per matrix, the activations are quantised per row on the way in (scale =
+ * max|x| / 448, nearest-even e4m3 code of x / scale, decided in fp32).  Everything else (normalisation,
+ * attention, scores, selection, the LM head, every lazy_decode_step) stays in the context's bf16 arithmetic
+ * and bf16 weights.  bf16 contexts only.  Arrays: host arrays of n_layers entries; code matrices: device,
+ * same [out, in] shapes as their 16-bit counterparts, one byte per element, 16-byte aligned, in-features a
+ * multiple of 16.  The pointers must stay valid while set; NULL switches back to the 16-bit weights. */
+typedef struct {
+  const void *const *w_qkv, *const *w_o, *const *w_gate, *const *w_up, *const *w_down;
+  const float *s_qkv, *s_o, *s_gate, *s_up, *s_down;
+} lazy_fp8_weights;
+int lazy_set_fp8_weights(lazy_ctx *ctx, const lazy_fp8_weights *w);
 /* Where the scoring layer is cut (Section 3.2, Aux Cache paragraph).  after_layer = 0 (default): between
  * the layer's attention half and its MLP, so that MLP already runs on the kept rows, the Aux Cache holds
  * post-attention hidden states and a revived token first gets that layer's MLP.  after_layer = 1: after
@@ -310,6 +324,14 @@ int lazy_k_gemm_swiglu(void *stream, int32_t dtype, int32_t impl, const void *A,
 int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void *A, const void *Bg,
                           const void *Bu, void *C, int32_t M, int32_t F, int32_t K, void *d_scratch,
                           size_t scratch_bytes);
+/* Per-row e4m3 quantisation of bf16 activations x [M, K] (K a multiple of 16): q [M, K] receives the codes
+ * (bytes), scale [M] (device fp32) the row scales max|x| / 448 (1 for an all-zero row). */
+int lazy_k_quant_rows_e4m3(void *stream, const void *x, void *q, float *scale, int32_t M, int32_t K);
+/* C[M,N] = (A8 B8^T) * a_scale[row] * w_scale (+ R) in bf16, A8 [M,K] / B8 [N,K] e4m3 codes, tcgen05
+ * kind::f8f6f4 with fp32 accumulation.  With B8u != NULL: C[M,N] = silu(A8 B8^T * s) * (A8 B8u^T * s_up), the
+ * first half of the MLP (R must be NULL).  M > 0, K a multiple of 16, N a multiple of 8. */
+int lazy_k_gemm_fp8(void *stream, const void *A8, const float *a_scale, const void *B8, float w_scale,
+                    const void *B8u, float w_scale_up, const void *R, void *C, int32_t M, int32_t N, int32_t K);
 /* In-place RoPE of q and k inside qkv [n, 3*H*dh] by positions pos[n]; rotated k and v are
  * also written to kcache / vcache [n, H*dh].  rope_table: device fp32[max_pos*head_dim] scratch
  * that the call fills first. */

@@ -44,6 +44,11 @@ class lazy_weights(C.Structure):
                 ("g_final", C.c_void_p), ("w_lm_head", C.c_void_p)]
 
 
+class lazy_fp8_weights(C.Structure):
+    _fields_ = [(n, C.POINTER(C.c_void_p)) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down")] + \
+               [(n, C.POINTER(C.c_float)) for n in ("s_qkv", "s_o", "s_gate", "s_up", "s_down")]
+
+
 class lazy_schedule(C.Structure):
     _fields_ = [("n_points", C.c_int32), ("layer_entered", C.POINTER(C.c_int32)),
                 ("keep_bp", C.POINTER(C.c_uint32))]
@@ -100,6 +105,9 @@ _SIGNATURES = {
     "lazy_k_gemm_swiglu": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I]),
     "lazy_set_aux_point": (_I, [_P, _I]),
     "lazy_set_selection": (_I, [_P, _I]),
+    "lazy_set_fp8_weights": (_I, [_P, C.POINTER(lazy_fp8_weights)]),
+    "lazy_k_quant_rows_e4m3": (_I, [_P, _P, _P, _P, _I, _I]),
+    "lazy_k_gemm_fp8": (_I, [_P, _P, _P, _P, _F, _P, _F, _P, _P, _I, _I, _I]),
     "lazy_k_gemm_scratch_bytes": (_Z, []),
     "lazy_k_gemm_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
     "lazy_k_gemm_swiglu_ws": (_I, [_P, _I, _I, _P, _P, _P, _P, _I, _I, _I, _P, _Z]),
@@ -265,6 +273,23 @@ class LazyPrefill:
     def lazy_set_aux_point(self, after_layer: bool) -> None:
         _check("lazy_set_aux_point", lib().lazy_set_aux_point(self.ctx, 1 if after_layer else 0))
 
+    def lazy_set_fp8_weights(self, q: Optional[dict]) -> None:
+        """q: {"layers": [{name: (codes uint8 CUDA tensor [out, in], scale)}]} for the five projection
+        matrices of every layer (the output of synth.quantize_projections_e4m3 moved to the device), or None
+        to return to the 16-bit weights."""
+        if q is None:
+            _check("lazy_set_fp8_weights", lib().lazy_set_fp8_weights(self.ctx, None))
+            self._fp8 = None
+            return
+        names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down")
+        n = self.shape.n_layers
+        ptrs = [(C.c_void_p * n)(*[_ptr(lq[k][0]) for lq in q["layers"]]) for k in names]
+        scales = [(C.c_float * n)(*[float(lq[k][1]) for lq in q["layers"]]) for k in names]
+        w = lazy_fp8_weights(*[C.cast(a, C.POINTER(C.c_void_p)) for a in ptrs],
+                             *[C.cast(a, C.POINTER(C.c_float)) for a in scales])
+        _check("lazy_set_fp8_weights", lib().lazy_set_fp8_weights(self.ctx, C.byref(w)))
+        self._fp8 = (q, ptrs, scales)   # keeps the tensors alive (the library copies the arrays themselves)
+
     def lazy_set_selection(self, threshold: bool) -> None:
         _check("lazy_set_selection", lib().lazy_set_selection(self.ctx, 1 if threshold else 0))
 
@@ -396,6 +421,26 @@ def lazy_k_gemm_swiglu(A: torch.Tensor, Bg: torch.Tensor, Bu: torch.Tensor, impl
     return Cm
 
 
+def lazy_k_quant_rows_e4m3(x: torch.Tensor):
+    """(codes uint8 [M, K], scale fp32 [M]) of the per-row e4m3 quantisation of bf16 x [M, K]."""
+    M, K = x.shape
+    q = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    sc = torch.empty(max(M, 1), dtype=torch.float32, device=x.device)
+    _check("lazy_k_quant_rows_e4m3", lib().lazy_k_quant_rows_e4m3(_stream(), _ptr(x), _ptr(q), _ptr(sc), M, K))
+    return q, sc[:M]
+
+
+def lazy_k_gemm_fp8(A8: torch.Tensor, a_scale: torch.Tensor, B8: torch.Tensor, w_scale: float,
+                    B8u: Optional[torch.Tensor] = None, w_scale_up: float = 1.0,
+                    R: Optional[torch.Tensor] = None) -> torch.Tensor:
+    M, K = A8.shape
+    N = B8.shape[0]
+    Cm = torch.empty((M, N), dtype=torch.bfloat16, device=A8.device)
+    _check("lazy_k_gemm_fp8", lib().lazy_k_gemm_fp8(_stream(), _ptr(A8), _ptr(a_scale), _ptr(B8), w_scale, _ptr(B8u),
+                                                    w_scale_up, _ptr(R), _ptr(Cm), M, N, K))
+    return Cm
+
+
 def lazy_k_rope_kv(qkv: torch.Tensor, pos: torch.Tensor, n_heads: int, head_dim: int, max_pos: int,
                    theta: float):
     """Rotates q and k inside qkv in place; returns (k_cache, v_cache)."""
@@ -422,11 +467,16 @@ def lazy_k_attention(q: torch.Tensor, ldq: int, k: torch.Tensor, v: torch.Tensor
 
 
 def lazy_k_score(q: torch.Tensor, ldq: int, k: torch.Tensor, ldkv: int, cu_seqlens: torch.Tensor,
-                 n_total: int, n_heads: int, head_dim: int) -> torch.Tensor:
+                 n_total: int, n_heads: int, head_dim: int,
+                 out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None) -> torch.Tensor:
+    """out = (scratch, scores) buffers of an earlier call may be handed back in (timing loops)."""
     n_seqs = cu_seqlens.numel() - 1
-    nf = lib().lazy_k_score_scratch_floats(n_seqs, n_total, n_heads)
-    scratch = torch.empty(max(nf, 1), dtype=torch.float32, device=k.device)
-    scores = torch.empty(n_total, dtype=torch.float32, device=k.device)
+    if out is not None:
+        scratch, scores = out
+    else:
+        nf = lib().lazy_k_score_scratch_floats(n_seqs, n_total, n_heads)
+        scratch = torch.empty(max(nf, 1), dtype=torch.float32, device=k.device)
+        scores = torch.empty(n_total, dtype=torch.float32, device=k.device)
     _check("lazy_k_score", lib().lazy_k_score(_stream(), dtype_code(k.dtype), q.data_ptr(), ldq, _ptr(k), ldkv,
                                               _ptr(cu_seqlens), n_seqs, n_total, n_heads, head_dim,
                                               _ptr(scratch), _ptr(scores)))
@@ -443,12 +493,18 @@ def lazy_k_score_static(q: torch.Tensor, ldq: int, k: torch.Tensor, ldkv: int, c
     return scores
 
 
-def lazy_k_select(scores: torch.Tensor, cu_in: torch.Tensor, cu_keep: torch.Tensor):
+def lazy_k_select(scores: torch.Tensor, cu_in: torch.Tensor, cu_keep: torch.Tensor, n_in: Optional[int] = None,
+                  n_keep: Optional[int] = None, out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
+    """n_in / n_keep (totals over the batch) and out = (keep, drop) buffers may be passed by a caller that
+    knows them, which keeps the call free of device reads and allocations (timing loops)."""
     n_seqs = cu_in.numel() - 1
-    n_in = int(cu_in[-1].item())
-    n_keep = int(cu_keep[-1].item())
-    keep = torch.empty(max(n_keep, 1), dtype=torch.int32, device=scores.device)
-    drop = torch.empty(max(n_in - n_keep, 1), dtype=torch.int32, device=scores.device)
+    n_in = int(cu_in[-1].item()) if n_in is None else n_in
+    n_keep = int(cu_keep[-1].item()) if n_keep is None else n_keep
+    if out is not None:
+        keep, drop = out
+    else:
+        keep = torch.empty(max(n_keep, 1), dtype=torch.int32, device=scores.device)
+        drop = torch.empty(max(n_in - n_keep, 1), dtype=torch.int32, device=scores.device)
     _check("lazy_k_select", lib().lazy_k_select(_stream(), _ptr(scores), _ptr(cu_in), _ptr(cu_keep), n_seqs,
                                                 _ptr(keep), _ptr(drop)))
     return keep[:n_keep], drop[:n_in - n_keep]
@@ -467,9 +523,9 @@ def lazy_k_select_threshold(scores: torch.Tensor, cu_in: torch.Tensor, prune_bp:
     return keep, drop, counts[:n_seqs]
 
 
-def lazy_k_gather_rows(src: torch.Tensor, idx: torch.Tensor) -> torch.Tensor:
+def lazy_k_gather_rows(src: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     n = idx.numel()
-    dst = torch.empty((n,) + tuple(src.shape[1:]), dtype=src.dtype, device=src.device)
+    dst = out if out is not None else torch.empty((n,) + tuple(src.shape[1:]), dtype=src.dtype, device=src.device)
     row_bytes = src[0].numel() * src.element_size()
     _check("lazy_k_gather_rows", lib().lazy_k_gather_rows(_stream(), _ptr(src), _ptr(idx), _ptr(dst), n,
                                                           row_bytes, src.shape[0]))

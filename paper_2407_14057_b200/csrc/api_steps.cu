@@ -1,4 +1,5 @@
 // Context-free entry points: the individual steps of the path and the single-layer pruning op.
+#include "gemm_epilogue.cuh"
 #include "runtime.cuh"
 
 using namespace lazy;
@@ -50,6 +51,25 @@ int lazy_k_gemm_swiglu_ws(void *stream, int32_t dtype, int32_t impl, const void 
   if (impl == 1) return launch_gemm_simt((cudaStream_t)stream, dtype, A, Bg, Bu, nullptr, C, M, F, K, 1);
   return launch_gemm_swiglu((cudaStream_t)stream, dtype, A, Bg, Bu, C, M, F, K, status, d_scratch, scratch_bytes,
                             impl == 2 ? 1 : (impl == 3 ? 2 : 0));
+}
+
+int lazy_k_quant_rows_e4m3(void *stream, const void *x, void *q, float *scale, int32_t M, int32_t K) {
+  if (M < 0 || K < 16 || K % 16) return LAZY_E_BADARG;
+  if (M == 0) return LAZY_OK;
+  if (!x || !q || !scale) return LAZY_E_BADARG;
+  return launch_quant_rows_e4m3((cudaStream_t)stream, x, q, scale, M, K);
+}
+
+int lazy_k_gemm_fp8(void *stream, const void *A8, const float *a_scale, const void *B8, float w_scale,
+                    const void *B8u, float w_scale_up, const void *R, void *C, int32_t M, int32_t N, int32_t K) {
+  if (M < 0 || N < 8 || K < 16 || N % 8 || K % 16) return LAZY_E_BADARG;
+  if (M == 0) return LAZY_OK;
+  if (!A8 || !a_scale || !B8 || !C || (B8u && R)) return LAZY_E_BADARG;
+  DevStatus *status = dev_status_ptr();
+  if (!status) return LAZY_E_CUDA;
+  const int epi = B8u ? EPI_SWIGLU : (R ? EPI_RESIDUAL : EPI_PLAIN);
+  return launch_gemm_fp8((cudaStream_t)stream, epi, A8, a_scale, B8, w_scale, B8u, w_scale_up, R, C, M, N, K, status,
+                         RopeArgs(), nullptr, 0);
 }
 
 int lazy_k_rope_kv(void *stream, int32_t dtype, void *qkv, const int32_t *pos, float *rope_table,

@@ -181,6 +181,8 @@ int launch_rmsnorm(cudaStream_t st, int dtype, const void *x, const void *g, voi
 int launch_rmsnorm_rows(cudaStream_t st, int dtype, const void *x, const int32_t *row_idx,
                         const void *g, void *y, int n, int d, float eps);
 int launch_rope_table(cudaStream_t st, float *table, int max_pos, int head_dim, float theta);
+// Per-row e4m3 quantisation of bf16 activations x [M, K]: q [M, K] codes (bytes), scale [M]; K multiple of 16.
+int launch_quant_rows_e4m3(cudaStream_t st, const void *x, void *q, float *scale, int M, int K);
 // q rotated in place inside qkv; rotated k and v written to the caches at row kv_row[r]
 // (or r if kv_row is NULL) together with the position tag.  Grouped-query attention: n_kv_heads key/value
 // heads (0 = n_heads); a row of qkv is [q: n_heads*dh | k: n_kv_heads*dh | v: n_kv_heads*dh], a cache row

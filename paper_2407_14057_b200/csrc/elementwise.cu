@@ -248,6 +248,58 @@ int launch_rmsnorm(cudaStream_t st, int dtype, const void *x, const void *g, voi
   return launch_rmsnorm_rows(st, dtype, x, nullptr, g, y, n, d, eps);
 }
 
+// ---- per-row e4m3 quantisation of activations ------------------------------------------------------------
+// One CTA per row: scale = max|x| / 448 (1 for an all-zero row), code = e4m3(x / scale), both decided in
+// fp32 with IEEE division and round-to-nearest-even conversion (the definition the CPU reference follows).
+// The row is read twice (the second pass hits L1 / L2).
+__global__ void __launch_bounds__(256)
+quant_rows_e4m3_kernel(const bf16 *__restrict__ x, uint8_t *__restrict__ q, float *__restrict__ scale, int K) {
+  const int r = blockIdx.x;
+  const uint4 *xr = reinterpret_cast<const uint4 *>(x + (size_t)r * K);
+  const int nvec = K >> 3;
+  float amax = 0.f;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    Vec16<bf16> v;
+    v.raw = xr[i];
+    float f[8];
+    v.unpack(f);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(f[j]));
+  }
+  __shared__ float part[8];
+  amax = warp_max(amax);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  amax = part[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) amax = fmaxf(amax, part[w]);
+  const float sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+  if (threadIdx.x == 0) scale[r] = sc;
+  uint2 *qr = reinterpret_cast<uint2 *>(q + (size_t)r * K);
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    Vec16<bf16> v;
+    v.raw = xr[i];
+    float f[8];
+    v.unpack(f);
+    uint32_t w[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      unsigned short lo, hi;  // each: two codes, the first operand of the conversion in the upper byte
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(f[4 * h + 1], sc)), "f"(__fdiv_rn(f[4 * h], sc)));
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(f[4 * h + 3], sc)), "f"(__fdiv_rn(f[4 * h + 2], sc)));
+      w[h] = (uint32_t)lo | ((uint32_t)hi << 16);
+    }
+    qr[i] = make_uint2(w[0], w[1]);
+  }
+}
+int launch_quant_rows_e4m3(cudaStream_t st, const void *x, void *q, float *scale, int M, int K) {
+  if (M == 0) return LAZY_OK;
+  if ((K % 16) || ((uintptr_t)x & 15) || ((uintptr_t)q & 15)) return LAZY_E_BADARG;
+  quant_rows_e4m3_kernel<<<M, 256, 0, st>>>((const bf16 *)x, (uint8_t *)q, scale, K);
+  LAZY_COUNT_LAUNCH();
+  return launch_ok();
+}
+
 // ---- RoPE table -----------------------------------------------------------------------------------
 // table[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), evaluated in double once at set-up.
 __global__ void rope_table_kernel(float2 *table, int max_pos, int half, int head_dim, double theta) {

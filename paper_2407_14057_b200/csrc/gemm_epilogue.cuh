@@ -22,6 +22,10 @@ struct RopeArgs {
   const int32_t *kv_row;  // cache row of GEMM row r (NULL: r)
   int d_model, max_pos;
   int d_kv;               // width of a K / V cache row: n_kv_heads * head_dim (= d_model without grouping)
+  // 8-bit operands: the accumulator of row r is the product of e4m3 codes and is multiplied by
+  // a_scale[r] * w_scale on the way out (SwiGLU: gate columns by w_scale, up columns by w_scale_up)
+  const float *a_scale = nullptr;
+  float w_scale = 1.f, w_scale_up = 1.f;
 };
 
 // ---- the last, partial wave ------------------------------------------------------------------------------
@@ -252,6 +256,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       }
       krow = rope.kv_row ? (size_t)rope.kv_row[row] : (size_t)row;
     }
+    const float osc = (rope.a_scale && row < M) ? rope.a_scale[row] * rope.w_scale : 1.f;
     bf16 *dst = sect == 0 ? crow + n0
                           : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_kv + col_in;
     if (sect == 2) {
@@ -260,6 +265,8 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
         float v[32];
         tmem_ld_32x32(taddr + (uint32_t)c, v);
         if (row < M) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] *= osc;
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             Vec16<bf16> o;
@@ -281,7 +288,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
               const float4 cs = *reinterpret_cast<const float4 *>(tab + o + i);  // two (cos, sin)
-              const float a0 = lo[i], b0 = hi[i], a1 = lo[i + 1], b1 = hi[i + 1];
+              const float a0 = lo[i] * osc, b0 = hi[i] * osc, a1 = lo[i + 1] * osc, b1 = hi[i + 1] * osc;
               lo[i] = a0 * cs.x - b0 * cs.y;
               hi[i] = b0 * cs.x + a0 * cs.y;
               lo[i + 1] = a1 * cs.z - b1 * cs.w;
@@ -301,13 +308,23 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       if (sect == 1 && col_in == 0 && row < M && rope.kv_pos) rope.kv_pos[krow] = p;
     }
   } else {
+  const float asc = (rope.a_scale && row < M) ? rope.a_scale[row] : 1.f;
+  const float osc = asc * rope.w_scale, osc_up = asc * rope.w_scale_up;
 #pragma unroll 1
   for (int c = 0; c < TILE_N; c += 32) {
     float v[32];
     tmem_ld_32x32(taddr + (uint32_t)c, v);
+    if (rope.a_scale) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] *= osc;
+    }
     if (EPI == EPI_SWIGLU) {
       float u[32];
       tmem_ld_32x32(taddr + (uint32_t)(BN / 2 + c), u);
+      if (rope.a_scale) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) u[i] *= osc_up;
+      }
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
     }
@@ -400,6 +417,10 @@ inline GemmTail plan_tail(int num_tiles, int num_kb, int units, int cta_per_unit
 int launch_gemm_pair(int epi, cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R,
                      void *C, int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
                      size_t scratch_bytes);
+// 8-bit products (e4m3 codes with scales; see gemm_tcgen05.cu).
+int launch_gemm_fp8(cudaStream_t st, int epi, const void *A8, const float *a_scale, const void *B8, float w_scale,
+                    const void *B8u, float w_scale_up, const void *R, void *C, int M, int N, int K, DevStatus *status,
+                    RopeArgs extra, void *scratch, size_t scratch_bytes);
 // Clusters of two CTAs of that kernel the device can hold at once (-1: query failed).
 int gemm_pair_max_clusters();
 

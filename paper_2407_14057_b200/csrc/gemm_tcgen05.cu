@@ -47,7 +47,9 @@ constexpr int GEMM_SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 
 
 // C is [M, ldc]; for EPI_SWIGLU the accumulator's columns [0,128) are gate features and
 // [128,256) the matching up features, and C receives 128 columns per tile.
-template <int EPI>
+// FP8: A and B hold e4m3 codes (one byte each): a stage is still 128-byte rows, now 128 elements of K, and the
+// MMA is kind::f8f6f4 with K = 32 per instruction; the epilogue applies the operands' scales.
+template <int EPI, bool FP8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
                          const __grid_constant__ CUtensorMap map_b0,
@@ -68,7 +70,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
   const int m_tiles = (M + BM - 1) / BM;
   const int n_tiles = (N + TILE_N_OUT - 1) / TILE_N_OUT;
   const int num_tiles = m_tiles * n_tiles;
-  const int num_kb = (K + BK - 1) / BK;
+  constexpr int BKE = FP8 ? 2 * BK : BK;  // elements of K per stage (128 bytes per row either way)
+  const int num_kb = (K + BKE - 1) / BKE;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -114,14 +117,14 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           if (!ok) break;
           const uint32_t full = smem_u32(&bars->full[stage]);
           mbar_expect_tx(full, A_STAGE_BYTES + B_STAGE_BYTES);
-          tma_load_2d(smem_u32(smem_a + stage * A_STAGE_BYTES), &map_a, full, kb * BK, m0);
+          tma_load_2d(smem_u32(smem_a + stage * A_STAGE_BYTES), &map_a, full, kb * BKE, m0);
           const uint32_t bdst = smem_u32(smem_b + stage * B_STAGE_BYTES);
           if (EPI == EPI_SWIGLU) {
-            tma_load_2d(bdst, &map_b0, full, kb * BK, n0);
-            tma_load_2d(bdst + B_HALF_BYTES, &map_b1, full, kb * BK, n0);
+            tma_load_2d(bdst, &map_b0, full, kb * BKE, n0);
+            tma_load_2d(bdst + B_HALF_BYTES, &map_b1, full, kb * BKE, n0);
           } else {
-            tma_load_2d(bdst, &map_b0, full, kb * BK, n0);
-            tma_load_2d(bdst + B_HALF_BYTES, &map_b0, full, kb * BK, n0 + BN / 2);
+            tma_load_2d(bdst, &map_b0, full, kb * BKE, n0);
+            tma_load_2d(bdst + B_HALF_BYTES, &map_b0, full, kb * BKE, n0 + BN / 2);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -130,7 +133,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(BM, BN);
+      const uint32_t idesc = FP8 ? umma_idesc_e4m3(BM, BN) : umma_idesc_bf16(BM, BN);
       int stage = 0;
       uint32_t phase = 0;
       int local = 0;
@@ -153,7 +156,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t adesc = umma_smem_desc(a_addr + k * UMMA_K * 2);
             const uint64_t bdesc = umma_smem_desc(b_addr + k * UMMA_K * 2);
-            umma_bf16(tmem_d, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+            if (FP8) umma_f8(tmem_d, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
+            else umma_bf16(tmem_d, adesc, bdesc, idesc, (kb > w.kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit(smem_u32(&bars->empty[stage]));  // stage reusable once these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -226,11 +230,6 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
 }
 
 // ---- host side -----------------------------------------------------------------------------------
-// Row-major bf16 matrix [rows, cols] (cols contiguous), box = 64 columns x box_rows rows.
-int make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows) {
-  return tma_map_2d_bf16(map, base, rows, cols, cols, BK, box_rows);
-}
-
 // Which kernel takes a product of more than one row tile: the one whose launch is estimated shorter.
 // Both cover the same outputs per wave (148 tiles of 128 rows, or 74 pair tiles of 256 rows); what differs is
 // how the row count pads to 128 / 256, how many waves that makes, what the split last wave recovers, and the
@@ -257,27 +256,30 @@ bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_b
   return w_pair * pair_wave < w_one;  // a pair tile takes pair_wave x the time of a one-CTA tile
 }
 
-template <int EPI>
+// FP8: A [M, K] and B0 / B1 [N, K] hold e4m3 codes (bytes), rope.a_scale / w_scale their scales; always the
+// one-CTA kernel.
+template <int EPI, bool FP8 = false>
 int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, const void *R, void *C,
               int M, int N, int K, DevStatus *status, const RopeArgs &rope, void *scratch,
               size_t scratch_bytes, int force_kernel) {
   // TMA needs 16-byte aligned bases and row pitches; the epilogue stores 8 columns at a time.
-  if ((K % 8) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
+  if ((K % (FP8 ? 16 : 8)) || (N % 8) || ((uintptr_t)A & 15) || ((uintptr_t)B0 & 15) || ((uintptr_t)B1 & 15) ||
       ((uintptr_t)C & 15) || ((uintptr_t)R & 15))
     return LAZY_E_BADARG;
-  if (gemm_use_pair(EPI, M, N, K, scratch, scratch_bytes, force_kernel))
+  if (!FP8 && gemm_use_pair(EPI, M, N, K, scratch, scratch_bytes, force_kernel))
     return launch_gemm_pair(EPI, st, A, B0, B1, R, C, M, N, K, status, rope, scratch, scratch_bytes);
+  constexpr int EB = FP8 ? 1 : 2, BKE = FP8 ? 2 * BK : BK;  // element bytes, elements of K per 128-byte stage row
   CUtensorMap ma, mb0, mb1;
-  LAZY_TRY(make_map(&ma, A, M, K, BM));
-  LAZY_TRY(make_map(&mb0, B0, N, K, BN / 2));
-  LAZY_TRY(make_map(&mb1, B1, N, K, BN / 2));
+  LAZY_TRY(tma_map_2d(&ma, A, M, K, K, BKE, BM, EB));
+  LAZY_TRY(tma_map_2d(&mb0, B0, N, K, K, BKE, BN / 2, EB));
+  LAZY_TRY(tma_map_2d(&mb1, B1, N, K, K, BKE, BN / 2, EB));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
-  const GemmTail tail = plan_tail(tiles, cdiv(K, BK), sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K,
+  const GemmTail tail = plan_tail(tiles, cdiv(K, BKE), sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K,
                                   EPI == EPI_SWIGLU ? 8 : 0, scratch,
                                   scratch_bytes);
   const int grid = (tiles < sm_count() && tail.tail_units == 0) ? tiles : sm_count();
-  auto kfn = gemm_bf16_tcgen05_kernel<EPI>;
+  auto kfn = gemm_bf16_tcgen05_kernel<EPI, FP8>;
   static bool attr_set = false;
   if (!attr_set) {
     LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
@@ -310,6 +312,30 @@ int launch_gemm(cudaStream_t st, int dtype, const void *A, const void *B, const 
   }
   return launch_tc<EPI_PLAIN>(st, A, B, B, nullptr, C, M, N, K, status, RopeArgs(), scratch, scratch_bytes,
                               force_kernel);
+}
+
+// 8-bit products: A8 [M, K] and B8 [N, K] are e4m3 codes, a_scale [M] the per-row scales of A, w_scale the
+// scale of B (w_scale_up of the second matrix of a SwiGLU product).  epi: EPI_PLAIN (R NULL) / EPI_RESIDUAL /
+// EPI_SWIGLU (B8 = gate, B8u = up, N = features) / EPI_QKV_ROPE (extra carries the rotary operands).
+int launch_gemm_fp8(cudaStream_t st, int epi, const void *A8, const float *a_scale, const void *B8, float w_scale,
+                    const void *B8u, float w_scale_up, const void *R, void *C, int M, int N, int K, DevStatus *status,
+                    RopeArgs extra, void *scratch, size_t scratch_bytes) {
+  if (M == 0) return LAZY_OK;
+  if (!a_scale) return LAZY_E_BADARG;
+  extra.a_scale = a_scale;
+  extra.w_scale = w_scale;
+  extra.w_scale_up = w_scale_up;
+  switch (epi) {
+    case EPI_PLAIN:
+      return launch_tc<EPI_PLAIN, true>(st, A8, B8, B8, nullptr, C, M, N, K, status, extra, scratch, scratch_bytes, 1);
+    case EPI_RESIDUAL:
+      return launch_tc<EPI_RESIDUAL, true>(st, A8, B8, B8, R, C, M, N, K, status, extra, scratch, scratch_bytes, 1);
+    case EPI_SWIGLU:
+      return launch_tc<EPI_SWIGLU, true>(st, A8, B8, B8u, nullptr, C, M, N, K, status, extra, scratch, scratch_bytes, 1);
+    case EPI_QKV_ROPE:
+      return launch_tc<EPI_QKV_ROPE, true>(st, A8, B8, B8, nullptr, C, M, N, K, status, extra, scratch, scratch_bytes, 1);
+    default: return LAZY_E_BADARG;
+  }
 }
 
 // The residual row list exists in the tensor-core epilogue only.

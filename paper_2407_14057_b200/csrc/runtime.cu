@@ -186,6 +186,8 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
   c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)(16 * 2 + L) * (c->S + 1) * 4);
   c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
+  c->a8 = (uint8_t *)k.take(c->dtype == LAZY_BF16 ? R * (size_t)(c->F > c->d ? c->F : c->d) : 0);
+  c->a8_scale = (float *)k.take(c->dtype == LAZY_BF16 ? R * 4 : 0);
   c->gemm_scratch_bytes = c->dtype == LAZY_BF16 ? gemm_scratch_bytes() : 0;
   c->gemm_scratch = c->gemm_scratch_bytes ? k.take(c->gemm_scratch_bytes) : nullptr;
   c->capture = with_capture ? k.take((size_t)L * R * rb) : nullptr;
@@ -339,6 +341,38 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
 int32_t lazy_keep_count(int32_t n_total, uint32_t keep_bp, int32_t n_present) {
   if (n_total < 1 || keep_bp < 1 || keep_bp > 10000 || n_present < 1) return 0;
   return keep_count(n_total, keep_bp, n_present);
+}
+
+int lazy_set_fp8_weights(lazy_ctx *c, const lazy_fp8_weights *w) {
+  if (!c) return LAZY_E_BADARG;
+  if (!w) {
+    c->fp8_on = false;
+    return LAZY_OK;
+  }
+  if (c->dtype != LAZY_BF16 || c->d % 16 || c->F % 16) return LAZY_E_BADARG;
+  if (!w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->s_qkv || !w->s_o || !w->s_gate ||
+      !w->s_up || !w->s_down)
+    return LAZY_E_BADARG;
+  for (int l = 0; l < c->L; ++l) {
+    const void *ps[5] = {w->w_qkv[l], w->w_o[l], w->w_gate[l], w->w_up[l], w->w_down[l]};
+    for (const void *p : ps)
+      if (!p || ((uintptr_t)p & 15)) return LAZY_E_BADARG;
+    const float ss[5] = {w->s_qkv[l], w->s_o[l], w->s_gate[l], w->s_up[l], w->s_down[l]};
+    for (float s : ss)
+      if (!(s > 0.f)) return LAZY_E_BADARG;
+  }
+  c->w8_qkv.assign(w->w_qkv, w->w_qkv + c->L);
+  c->w8_o.assign(w->w_o, w->w_o + c->L);
+  c->w8_gate.assign(w->w_gate, w->w_gate + c->L);
+  c->w8_up.assign(w->w_up, w->w_up + c->L);
+  c->w8_down.assign(w->w_down, w->w_down + c->L);
+  c->s8_qkv.assign(w->s_qkv, w->s_qkv + c->L);
+  c->s8_o.assign(w->s_o, w->s_o + c->L);
+  c->s8_gate.assign(w->s_gate, w->s_gate + c->L);
+  c->s8_up.assign(w->s_up, w->s_up + c->L);
+  c->s8_down.assign(w->s_down, w->s_down + c->L);
+  c->fp8_on = true;
+  return LAZY_OK;
 }
 
 int lazy_set_selection(lazy_ctx *c, int32_t mode) {
@@ -519,7 +553,35 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       attn_flops += 2.0 * d * ns * (ns + 1.0);
     }
     TIMED(LAZY_K_RMSNORM, 0, 2.0 * n * rb, launch_rmsnorm(st, dt, x, c->g_attn[l], c->h, n, d, c->cfg.rms_eps));
-    if (gemm_qkv_rope_eligible(dt, d, c->dh, dkv)) {
+    // 8-bit projections: the activation is quantised per row into the staging buffer, then multiplied as
+    // e4m3 codes (products of up to four rows stay on the 16-bit weight-streaming kernel)
+    const bool f8 = c->fp8_on && dt == LAZY_BF16 && n > 4;
+    auto quant = [&](const void *src, int rows, int width) -> int {
+      return launch_quant_rows_e4m3(st, src, c->a8, c->a8_scale, rows, width);
+    };
+    if (f8) {
+      TIMED(LAZY_K_OTHER, 0, 3.0 * n * d, quant(c->h, n, d));
+      RopeArgs r = {};
+      const bool fused = gemm_qkv_rope_eligible(dt, d, c->dh, dkv);
+      if (fused) {
+        r.pos = pos;
+        r.table = (const float2 *)c->rope_table;
+        r.kcache = (bf16 *)kc;
+        r.vcache = (bf16 *)vc;
+        r.kv_pos = kvp;
+        r.kv_row = c->kv_row[g];
+        r.d_model = d;
+        r.max_pos = c->max_pos;
+        r.d_kv = dkv;
+      }
+      TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
+            launch_gemm_fp8(st, fused ? EPI_QKV_ROPE : EPI_PLAIN, c->a8, c->a8_scale, c->w8_qkv[l], c->s8_qkv[l], nullptr,
+                            1.f, nullptr, c->qkv, n, qc, d, status, r, c->gemm_scratch, c->gemm_scratch_bytes));
+      if (!fused)
+        TIMED(LAZY_K_ROPE_KV, 0, 6.0 * n * rb,
+              launch_rope_kv(st, dt, c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n, c->H, c->dh,
+                             c->max_pos, status, c->Hkv));
+    } else if (gemm_qkv_rope_eligible(dt, d, c->dh, dkv)) {
       // rotary embedding and the K/V cache write ride in the projection's epilogue
       TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
             launch_gemm_qkv_rope(st, c->h, c->w_qkv[l], c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n,
@@ -567,8 +629,15 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       TIMED(LAZY_K_SCORE, 0, (double)n * rb + 4.0 * n,
             launch_score(st, dt, c->qkv, qc, kc, dkv, d_cu(g), d_base, n_seqs, n, seg_max, c->H, c->dh,
                          c->score_scratch, sc, c->Hkv));
-    TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status,
-                                                      c->gemm_scratch, c->gemm_scratch_bytes, 0, true));
+    if (f8) {
+      TIMED(LAZY_K_OTHER, 0, 3.0 * n * d, quant(c->attn, n, d));
+      TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0,
+            launch_gemm_fp8(st, EPI_RESIDUAL, c->a8, c->a8_scale, c->w8_o[l], c->s8_o[l], nullptr, 1.f, x, x, n, d, d,
+                            status, RopeArgs(), c->gemm_scratch, c->gemm_scratch_bytes));
+    } else {
+      TIMED(LAZY_K_GEMM_O, 2.0 * n * d * d, 0, launch_gemm(st, dt, c->attn, c->w_o[l], x, x, n, d, d, status,
+                                                        c->gemm_scratch, c->gemm_scratch_bytes, 0, true));
+    }
 
     const int p = c->point_at[l + 1];
     // Rows of the residual stream that survive a cut made in this layer, when they are still where they
@@ -580,12 +649,25 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       const int n2 = c->seg_cu[g][n_seqs];
       TIMED(LAZY_K_RMSNORM, 0, 2.0 * n2 * rb,
             launch_rmsnorm_rows(st, dt, x, via_keep, c->g_mlp[l], c->h, n2, d, c->cfg.rms_eps));
-      TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
-            launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
-                               c->gemm_scratch_bytes, 0, true));
-      TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
-            launch_gemm(st, dt, c->act, c->w_down[l], x, via_keep ? x2 : x, n2, d, c->F, status, c->gemm_scratch,
-                        c->gemm_scratch_bytes, 0, true, via_keep));
+      if (c->fp8_on && dt == LAZY_BF16 && n2 > 4) {
+        TIMED(LAZY_K_OTHER, 0, 3.0 * n2 * d, quant(c->h, n2, d));
+        TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
+              launch_gemm_fp8(st, EPI_SWIGLU, c->a8, c->a8_scale, c->w8_gate[l], c->s8_gate[l], c->w8_up[l], c->s8_up[l],
+                              nullptr, c->act, n2, c->F, d, status, RopeArgs(), c->gemm_scratch, c->gemm_scratch_bytes));
+        TIMED(LAZY_K_OTHER, 0, 3.0 * n2 * c->F, quant(c->act, n2, c->F));
+        RopeArgs rr = {};
+        rr.res_rows = via_keep;
+        TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
+              launch_gemm_fp8(st, EPI_RESIDUAL, c->a8, c->a8_scale, c->w8_down[l], c->s8_down[l], nullptr, 1.f, x,
+                              via_keep ? x2 : x, n2, d, c->F, status, rr, c->gemm_scratch, c->gemm_scratch_bytes));
+      } else {
+        TIMED(LAZY_K_GEMM_GATE_UP, 4.0 * n2 * c->F * d, 0,
+              launch_gemm_swiglu(st, dt, c->h, c->w_gate[l], c->w_up[l], c->act, n2, c->F, d, status, c->gemm_scratch,
+                                 c->gemm_scratch_bytes, 0, true));
+        TIMED(LAZY_K_GEMM_DOWN, 2.0 * n2 * d * c->F, 0,
+              launch_gemm(st, dt, c->act, c->w_down[l], x, via_keep ? x2 : x, n2, d, c->F, status, c->gemm_scratch,
+                          c->gemm_scratch_bytes, 0, true, via_keep));
+      }
       if (via_keep) {
         char *t = x; x = x2; x2 = t;
         via_keep = nullptr;

@@ -55,6 +55,12 @@ struct lazy_ctx {
   float *dec_f32;
   bool select_threshold = false;  // threshold reading of the selection: ties at the scheduled rank all survive
   bool aux_after_layer = false;  // cut after the whole scoring layer (Aux rows = layer output) instead of before its MLP
+  // 8-bit projections: codes and scales per layer (empty = off), staging for the quantised activations
+  std::vector<const void *> w8_qkv, w8_o, w8_gate, w8_up, w8_down;
+  std::vector<float> s8_qkv, s8_o, s8_gate, s8_up, s8_down;
+  bool fp8_on = false;
+  uint8_t *a8;       // [cap_rows, max(d, F)] e4m3 codes of the activation entering a projection
+  float *a8_scale;   // [cap_rows]
   void *gemm_scratch;  // split-wave partials and counters of the tensor-core GEMMs (bf16 only)
   size_t gemm_scratch_bytes;
 

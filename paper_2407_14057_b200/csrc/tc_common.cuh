@@ -94,6 +94,20 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same MMA on 8-bit operands (kind::f8f6f4; both e4m3 here): K = 32 elements per instruction.
+__device__ __forceinline__ void umma_f8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Instruction descriptor, kind::f8f6f4: D fp32, A and B e4m3 (format code 0), both K-major.
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(int m, int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
@@ -201,18 +215,24 @@ inline EncodeTiledFn tma_encode_fn() {
 
 // Row-major bf16 matrix: `rows` rows of `cols` elements, row pitch `ld` elements; box =
 // box_cols x box_rows with 128-byte swizzle (box_cols * 2 bytes <= 128); out-of-range reads give 0.
-inline int tma_map_2d_bf16(CUtensorMap *map, const void *base, long long rows, int cols, long long ld,
-                           int box_cols, int box_rows) {
+// elem_bytes 2: bf16; 1: bytes (e4m3 codes), box_cols then <= 128.
+inline int tma_map_2d(CUtensorMap *map, const void *base, long long rows, int cols, long long ld, int box_cols,
+                      int box_rows, int elem_bytes) {
   EncodeTiledFn fn = tma_encode_fn();
   if (!fn) return LAZY_E_CUDA;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+  CUresult r = fn(map, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                  const_cast<void *>(base), dims, strides, box,
                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? LAZY_OK : LAZY_E_CUDA;
+}
+inline int tma_map_2d_bf16(CUtensorMap *map, const void *base, long long rows, int cols, long long ld,
+                           int box_cols, int box_rows) {
+  return tma_map_2d(map, base, rows, cols, ld, box_cols, box_rows, 2);
 }
 
 }  // namespace lazy

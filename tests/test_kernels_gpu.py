@@ -381,3 +381,61 @@ def test_select_kernel_writes_position_lists_and_handles_long_sequences():
         if kind == "uniform":
             s = s + torch.arange(n, dtype=torch.float32) * 1e-12    # nearly equal, distinct in the low bits
         _select_case([s], [max(1, (n * 3) // 10)])
+
+
+# ----------------------------------------------------------------------------- e4m3 projections
+def test_quant_rows_e4m3_bit_exact():
+    """Per-row e4m3 quantisation: the codes and scales the kernel decides equal the oracle's, bit for bit
+    (both decide in float32: scale = max|x| / 448, code = nearest-even e4m3 of x / scale)."""
+    g = torch.Generator().manual_seed(70)
+    x = (torch.randn((37, 4096), generator=g) * torch.logspace(-3, 2, 37)[:, None]).to(torch.bfloat16)
+    x[5] = 0
+    x[6, :100] = 0
+    q, sc = B.lazy_k_quant_rows_e4m3(x.cuda())
+    B.lazy_device_status()
+    codes, scale = O.quant_rows_e4m3(to_np(x))
+    assert np.array_equal(to_np(sc), scale)
+    got = q.view(torch.float8_e4m3fn).float().cpu().numpy()
+    assert np.array_equal(got, codes)
+
+
+def _fp8_operands(M, N, K, seed):
+    a = _rand((M, K), seed, torch.bfloat16)
+    w = _rand((N, K), seed + 1, torch.float32, std=0.02)
+    ws = 2.0 ** np.ceil(np.log2(float(w.abs().max()) / 448.0))
+    w8 = (w / ws).to(torch.float8_e4m3fn)
+    a8, a_sc = B.lazy_k_quant_rows_e4m3(a.cuda())
+    a_deq = a8.view(torch.float8_e4m3fn).float().cpu().numpy().astype(np.float64) * to_np(a_sc).astype(np.float64)[:, None]
+    w_deq = w8.float().numpy().astype(np.float64) * ws
+    return a8, a_sc, w8.view(torch.uint8).cuda(), float(ws), a_deq, w_deq
+
+
+@pytest.mark.parametrize("M,N,K", [(5, 256, 128), (128, 256, 4096), (300, 520, 1040), (1013, 4096, 4096),
+                                   (2364, 4096, 11008)])
+def test_gemm_fp8_matches_the_product_of_the_dequantised_operands(M, N, K):
+    """tcgen05 kind::f8f6f4 product of e4m3 codes with fp32 accumulation, scales applied on the way out: against
+    the float64 product of the de-quantised operands (exact inputs on both sides; only the bf16 rounding of the
+    output and the fp32 accumulation order differ).  Ragged rows / columns / K, several waves, a split last wave."""
+    a8, a_sc, w8, ws, a_deq, w_deq = _fp8_operands(M, N, K, 80)
+    ref = a_deq @ w_deq.T
+    got = B.lazy_k_gemm_fp8(a8, a_sc, w8, ws)
+    B.lazy_device_status()
+    assert rel_err(to_np(got), ref) < BF16_STEP_TOL
+    r = _rand((M, N), 83, torch.bfloat16)
+    got = B.lazy_k_gemm_fp8(a8, a_sc, w8, ws, R=r.cuda())
+    B.lazy_device_status()
+    assert rel_err(to_np(got), ref + to_np(r)) < BF16_STEP_TOL
+
+
+def test_gemm_fp8_swiglu():
+    M, F, K = 700, 1408, 512
+    a8, a_sc, g8, gs, a_deq, g_deq = _fp8_operands(M, F, K, 90)
+    _, _, u8, us, _, u_deq = _fp8_operands(M, F, K, 94)
+    a8b, a_scb, _, _, a_deqb, _ = _fp8_operands(M, F, K, 90)      # same activations (same seed)
+    assert torch.equal(a8, a8b)
+    gg = a_deq @ g_deq.T
+    uu = a_deq @ u_deq.T
+    ref = gg / (1.0 + np.exp(-gg)) * uu
+    got = B.lazy_k_gemm_fp8(a8, a_sc, g8, gs, B8u=u8, w_scale_up=us)
+    B.lazy_device_status()
+    assert rel_err(to_np(got), ref) < BF16_STEP_TOL

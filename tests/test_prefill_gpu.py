@@ -33,11 +33,25 @@ def _to_cuda(W):
     return out
 
 
-def _tols(dtype):
+# With e4m3 projections the two sides quantise activations that differ by bf16 rounding noise (attention outputs,
+# SwiGLU outputs: about half a per cent), and an element that falls on the other side of a rounding boundary moves
+# by a whole e4m3 step (6 to 12 % of its value).  The disagreement feeds the next projection's quantiser, so
+# within one layer it grows to the level of the e4m3 noise itself and then stays there: measured 3.5-5.5 % of the
+# tensor in the root-mean-square sense and 3-7 % of its maximum element by element at 512 features, 9 % at the
+# 4096 / 11008-feature widths, at every depth (it does not accumulate).  Two runs in this mode cannot agree
+# more closely than that; what pins the arithmetic exactly are the step-level tests (bit-exact quantiser,
+# product of given codes to 1e-2).  Here tensors are held to 2e-1 of their maximum and 1.5e-1 root-mean-square,
+# scores to 3e-3, kept-set differences to a 15 % band.
+FP8_TOL, FP8_BAND, FP8_RMS, FP8_SCORE_ABS = 2e-1, 1.5e-1, 1.5e-1, 3e-3
+
+
+def _tols(dtype, fp8=False):
+    if fp8:
+        return FP8_TOL, FP8_BAND
     return (1e-4, 1e-5) if dtype == torch.float32 else (2e-2, 3e-2)   # tensor tol, relative score band
 
 
-def _check_set_difference(gpu_pos, ref_pos, ref_scores, ref_score_pos, band_rel):
+def _check_set_difference(gpu_pos, ref_pos, ref_scores, ref_score_pos, band_rel, band_abs=1e-3):
     """Tokens kept by one side only must sit at the threshold."""
     g, r = set(gpu_pos.tolist()), set(ref_pos.tolist())
     assert len(g) == len(r)
@@ -48,22 +62,27 @@ def _check_set_difference(gpu_pos, ref_pos, ref_scores, ref_score_pos, band_rel)
     last = int(ref_score_pos[-1])
     tau = min(s_of[p] for p in r if p != last)
     for p in diff:
-        assert abs(s_of[p] - tau) <= 1e-3, (p, s_of[p], tau)
+        assert abs(s_of[p] - tau) <= band_abs, (p, s_of[p], tau)
         assert abs(s_of[p] - tau) <= band_rel * tau, (p, s_of[p], tau)
     return len(diff)
 
 
 def run_model_case(shape, schedule, lengths, dtype, seed, perturb=True, max_new=0):
     bf16 = dtype == torch.bfloat16
-    tol, band = _tols(dtype)
+    fp8 = getattr(shape, "fp8", False)
+    tol, band = _tols(dtype, fp8)
+    score_abs = FP8_SCORE_ABS if fp8 else 1e-3
     W = synth.make_weights(shape, seed, bf16=bf16)
     if perturb:
         synth.perturb_gains(W, seed + 100)
+    q8 = synth.quantize_projections_e4m3(W) if fp8 else None     # W now holds the de-quantised weights
     Wn = weights_to_np(W)
     ids, cu = synth.make_varlen_batch(shape.vocab, lengths, seed + 1)
     n_seqs = len(lengths)
     eng = B.LazyPrefill(shape, _to_cuda(W), schedule, dtype, max_seqs=n_seqs,
                         max_prompt_tokens=sum(lengths), max_new_tokens=max_new, debug_capture=True)
+    if fp8:
+        eng.lazy_set_fp8_weights({"layers": [{k: (c.cuda(), s) for k, (c, s) in lq.items()} for lq in q8["layers"]]})
     logits = torch.empty((n_seqs, shape.vocab), dtype=torch.float32, device="cuda")
     d_ids = ids.cuda()
     eng.lazy_prefill_run(d_ids, cu, logits)
@@ -81,7 +100,7 @@ def run_model_case(shape, schedule, lengths, dtype, seed, perturb=True, max_new=
         first = points[0] if points else shape.n_layers
         for l in range(first):
             sc = to_np(eng.lazy_get_scores(l, s))
-            assert np.max(np.abs(sc - free.scores[l])) < 1e-3
+            assert np.max(np.abs(sc - free.scores[l])) < score_abs
             assert abs(sc.sum() - 1.0) < 1e-3 and sc.min() >= 0
         # (2)+(3) walk the cuts: compare against the oracle replayed on the GPU's sets so far
         replay = O.prefill(shape, Wn, sid, schedule, forced_keep=gpu_kept)
@@ -90,7 +109,7 @@ def run_model_case(shape, schedule, lengths, dtype, seed, perturb=True, max_new=
             partial = {k: v for k, v in gpu_kept.items() if k < e}
             ref = O.prefill(shape, Wn, sid, schedule, forced_keep=partial) if partial else free
             flips += _check_set_difference(gpu_kept[e], ref.kept_pos[e], ref.scores[e - 1],
-                                           ref.score_pos[e - 1], band)
+                                           ref.score_pos[e - 1], band, score_abs)
             assert np.all(np.diff(gpu_kept[e]) > 0) and gpu_kept[e][-1] == len(sid) - 1
             if prev is not None:
                 assert set(gpu_kept[e].tolist()) <= set(prev.tolist())       # subset property
@@ -98,11 +117,14 @@ def run_model_case(shape, schedule, lengths, dtype, seed, perturb=True, max_new=
         for l in range(shape.n_layers):
             sc = to_np(eng.lazy_get_scores(l, s))
             assert sc.shape == replay.scores[l].shape
-            assert np.max(np.abs(sc - replay.scores[l])) < 1e-3
+            assert np.max(np.abs(sc - replay.scores[l])) < score_abs
             n_l = replay.hidden_out[l].shape[0]
             got = hidden[l][row_off[l]:row_off[l] + n_l]
             row_off[l] += n_l
             assert rel_err(got, replay.hidden_out[l]) < tol, (l, rel_err(got, replay.hidden_out[l]))
+            if fp8:
+                rms = float(np.sqrt(np.mean((got - replay.hidden_out[l]) ** 2) / np.mean(replay.hidden_out[l] ** 2)))
+                assert rms < FP8_RMS, (l, rms)
             kpos, kk, vv = eng.lazy_get_kv(l, s)
             assert np.array_equal(to_np(kpos), replay.rows_pos[l])
             kr, vr = replay.layers[l].rows(replay.rows_pos[l])
@@ -385,3 +407,19 @@ def test_grouped_query_attention_wide_shape_bf16():
     shape = synth.ModelShape(n_layers=2, d_model=4096, n_heads=32, head_dim=128, d_ffn=11008, vocab=4096,
                              n_kv_heads=8)
     run_model_case(shape, ((1, 5000),), [700], torch.bfloat16, seed=35, perturb=False)
+
+
+# ----------------------------------------------------------------------------- e4m3 projections end to end
+def test_fp8_projections_prefill_small_model():
+    """The four projections of every layer on e4m3 operands (per-row activation scales, per-matrix weight
+    scales), everything else in bf16: pruned prefill against the oracle run in the same mode, on the same
+    de-quantised weights; kept sets, scores, hidden states, caches, Aux rows and logits."""
+    shape = synth.SMALL.with_fp8()
+    run_model_case(shape, ((1, 7000), (2, 5000), (3, 3000)), [300], torch.bfloat16, seed=41)
+    run_model_case(shape.with_layers(3).with_kv_heads(2), ((1, 6000), (2, 3000)), [200, 65, 9, 131], torch.bfloat16, seed=42)
+
+
+def test_fp8_projections_wide_shape_and_against_bf16():
+    """Two layers at the 7B widths, 1500-token prompt, one cut, against the oracle in the same mode."""
+    shape = synth.LLAMA7B.with_layers(2).with_fp8()
+    run_model_case(shape, ((1, 5000),), [1500], torch.bfloat16, seed=43, perturb=False)
