@@ -216,9 +216,12 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
 }
 
 // Residual addend of the 32 output columns [col0, col0 + 32) of a row, as four 16-byte vectors (a vector
-// beyond N, or a row beyond M, is left as it is).  A thread asks for them well before it needs them: the
-// first 32 columns of a tile before it waits for the tile's accumulator, every later group while it works
-// on the group before, so the L2 latency of these row-strided reads stays off the epilogue's critical path.
+// beyond N, or a row beyond M, is left as it is).  These reads are row-strided (a thread owns a row), and a
+// group that is only asked for when the group before it is being worked on costs a full L2 round trip per
+// group: measured, a 256-column tile then spent ~14 000 clocks in its residual epilogue, nearly all of it
+// waiting.  So a thread keeps GEMM_RES_AHEAD groups in flight: the first ones are requested before it waits
+// for the tile's accumulator, and each group consumed is replaced by the request GEMM_RES_AHEAD groups on.
+constexpr int GEMM_RES_AHEAD = 4;
 __device__ __forceinline__ void gemm_residual_load(uint4 (&r)[4], const bf16 *__restrict__ R, const RopeArgs &extra,
                                                    int row, int col0, int M, int N, int ldc) {
   if (row >= M) return;
@@ -226,6 +229,55 @@ __device__ __forceinline__ void gemm_residual_load(uint4 (&r)[4], const bf16 *__
 #pragma unroll
   for (int j = 0; j < 4; ++j)
     if (col0 + 8 * j < N) r[j] = *reinterpret_cast<const uint4 *>(rrow + col0 + 8 * j);
+}
+// The first GEMM_RES_AHEAD groups of a tile whose first output column is n0.
+__device__ __forceinline__ void gemm_residual_prefetch(uint4 (&r)[GEMM_RES_AHEAD][4], const bf16 *__restrict__ R,
+                                                       const RopeArgs &extra, int row, int n0, int M, int N, int ldc) {
+#pragma unroll
+  for (int g = 0; g < GEMM_RES_AHEAD; ++g) gemm_residual_load(r[g], R, extra, row, n0 + 32 * g, M, N, ldc);
+}
+
+// Output staging of an epilogue warp.  A thread owns a row, so storing straight from registers makes every
+// warp-wide store touch 32 different rows with 16 bytes each: measured, a 256-column tile's stores then took
+// 8 000-9 000 clocks (more when all CTAs end a launch together), most of a tile's epilogue.  Instead the
+// warp writes 64-column groups of its 32 rows into a 4 KiB shared-memory buffer in the 128-byte-swizzled
+// layout and one lane hands the buffer to the TMA unit, which writes whole 128-byte lines and drops what
+// lies beyond M or N.  Two buffers alternate, so a group is staged while the one before it drains.
+constexpr int GEMM_STG_BYTES = 4096;                       // 32 rows x 64 bf16
+constexpr int GEMM_STG_PER_CTA = 4 * 2 * GEMM_STG_BYTES;   // four epilogue warps, two buffers each
+struct EpiStore {
+  const CUtensorMap *map;  // the output matrix: box 64 columns x 32 rows, 128-byte swizzle
+  uint32_t stg;            // shared-memory address of this warp's two buffers (1024-byte aligned)
+  int y0;                  // first output row of the warp's 32-row block of the current tile
+  uint32_t n_out;          // groups handed over so far: the next group takes buffer n_out & 1
+};
+// Buffer for the next group, free to be written (the store that last read it has done so).
+__device__ __forceinline__ uint32_t epi_stage_begin(const EpiStore &es) {
+  if ((threadIdx.x & 31) == 0) bulk_wait_group_read<1>();
+  __syncwarp();
+  return es.stg + (es.n_out & 1u) * GEMM_STG_BYTES;
+}
+// 16-byte chunk j (columns 8j .. 8j+7 of the group) of this thread's row.
+__device__ __forceinline__ void epi_stage_put(uint32_t buf, int j, const uint4 &v) {
+  const uint32_t lane = threadIdx.x & 31;
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128u + (((uint32_t)j ^ (lane & 7u)) << 4)),
+               "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+               : "memory");
+}
+// Hands the staged group to the TMA unit: columns [x, x + 64) of rows [y0, y0 + 32).
+__device__ __forceinline__ void epi_stage_commit(EpiStore &es, uint32_t buf, int x) {
+  fence_proxy_async_smem();
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) {
+    tma_store_2d(es.map, buf, x, es.y0);
+    bulk_commit_group();
+  }
+  ++es.n_out;
+}
+// Before the CTA exits: every store of this warp has completed.
+__device__ __forceinline__ void epi_stage_drain() {
+  if ((threadIdx.x & 31) == 0) bulk_wait_group_all();
+  __syncwarp();
 }
 
 // One thread, one row.  taddr: TMEM address of the row's first accumulator column (lane field set);
@@ -236,8 +288,8 @@ template <int EPI>
 __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n0, int M, int N, int ldc,
                                                   const bf16 *__restrict__ R, bf16 *__restrict__ C,
                                                   const RopeArgs &rope, DevStatus *status,
-                                                  uint4 (&res_next)[4]) {
-  // res_next (EPI_RESIDUAL): the addend of the tile's first 32 columns, loaded by the caller ahead of time
+                                                  uint4 (&res_q)[GEMM_RES_AHEAD][4], EpiStore &es) {
+  // res_q (EPI_RESIDUAL): the addends of the tile's first column groups, requested by the caller ahead of time
   constexpr int BN = GEMM_ACC_N;
   constexpr int TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   bf16 *crow = C + (size_t)row * ldc;
@@ -279,21 +331,36 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       const float2 *tab = rope.table + (size_t)p * 64;
 #pragma unroll 1
       for (int hc = 0; hc < BN; hc += 128) {  // the two heads of the tile
+        // q goes out through the staging buffers (columns [0,64) of the head in the first, [64,128) in the
+        // second); rotated k goes straight to its cache row, which need not be row `row` of anything
+        if (sect == 0) {
+          if ((threadIdx.x & 31) == 0) bulk_wait_group_read<0>();
+          __syncwarp();
+        }
 #pragma unroll 1
         for (int o = 0; o < 64; o += 32) {    // pairs (i, i + 64), 32 at a time
           float lo[32], hi[32];
           tmem_ld_32x32(taddr + (uint32_t)(hc + o), lo);
           tmem_ld_32x32(taddr + (uint32_t)(hc + o + 64), hi);
-          if (row < M) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float4 cs = *reinterpret_cast<const float4 *>(tab + o + i);  // two (cos, sin)
-              const float a0 = lo[i] * osc, b0 = hi[i] * osc, a1 = lo[i + 1] * osc, b1 = hi[i + 1] * osc;
-              lo[i] = a0 * cs.x - b0 * cs.y;
-              hi[i] = b0 * cs.x + a0 * cs.y;
-              lo[i + 1] = a1 * cs.z - b1 * cs.w;
-              hi[i + 1] = b1 * cs.z + a1 * cs.w;
+          for (int i = 0; i < 32; i += 2) {
+            const float4 cs = *reinterpret_cast<const float4 *>(tab + o + i);  // two (cos, sin)
+            const float a0 = lo[i] * osc, b0 = hi[i] * osc, a1 = lo[i + 1] * osc, b1 = hi[i + 1] * osc;
+            lo[i] = a0 * cs.x - b0 * cs.y;
+            hi[i] = b0 * cs.x + a0 * cs.y;
+            lo[i + 1] = a1 * cs.z - b1 * cs.w;
+            hi[i + 1] = b1 * cs.z + a1 * cs.w;
+          }
+          if (sect == 0) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              Vec16<bf16> ol, oh;
+              ol.pack(lo + j);
+              oh.pack(hi + j);
+              epi_stage_put(es.stg, (o >> 3) + (j >> 3), ol.raw);
+              epi_stage_put(es.stg + GEMM_STG_BYTES, (o >> 3) + (j >> 3), oh.raw);
             }
+          } else if (row < M) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
               Vec16<bf16> ol, oh;
@@ -304,13 +371,24 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
             }
           }
         }
+        if (sect == 0) {
+          fence_proxy_async_smem();
+          __syncwarp();
+          if ((threadIdx.x & 31) == 0) {
+            tma_store_2d(es.map, es.stg, n0 + hc, es.y0);
+            tma_store_2d(es.map, es.stg + GEMM_STG_BYTES, n0 + hc + 64, es.y0);
+            bulk_commit_group();
+          }
+          es.n_out += 2;
+        }
       }
       if (sect == 1 && col_in == 0 && row < M && rope.kv_pos) rope.kv_pos[krow] = p;
     }
   } else {
   const float asc = (rope.a_scale && row < M) ? rope.a_scale[row] : 1.f;
   const float osc = asc * rope.w_scale, osc_up = asc * rope.w_scale_up;
-#pragma unroll 1
+  // fully unrolled with the residual epilogue, whose ring of requested groups is indexed statically
+#pragma unroll(EPI == EPI_RESIDUAL ? TILE_N / 32 : 1)
   for (int c = 0; c < TILE_N; c += 32) {
     float v[32];
     tmem_ld_32x32(taddr + (uint32_t)c, v);
@@ -326,36 +404,42 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
         for (int i = 0; i < 32; ++i) u[i] *= osc_up;
       }
 #pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = v[i] / (1.f + __expf(-v[i])) * u[i];
+      // SiLU(g) * u with the approximate reciprocal: the IEEE division cost ~100 clocks per element of a
+      // thread's row here (a tile's epilogue was compute-bound at ~15 000 clocks), and the result is rounded
+      // to bf16 anyway
+      for (int i = 0; i < 32; ++i) v[i] = __fdividef(v[i], 1.f + __expf(-v[i])) * u[i];
     }
     uint4 res_cur[4];
     if (EPI == EPI_RESIDUAL) {
+      constexpr int kGroups = TILE_N / 32;
+      const int g = (c >> 5) % GEMM_RES_AHEAD;  // static after unrolling
 #pragma unroll
-      for (int j = 0; j < 4; ++j) res_cur[j] = res_next[j];
-      if (c + 32 < TILE_N) gemm_residual_load(res_next, R, rope, row, n0 + c + 32, M, N, ldc);
+      for (int j = 0; j < 4; ++j) res_cur[j] = res_q[g][j];
+      if ((c >> 5) + GEMM_RES_AHEAD < kGroups)
+        gemm_residual_load(res_q[g], R, rope, row, n0 + c + 32 * GEMM_RES_AHEAD, M, N, ldc);
     }
-    if (row < M) {
+    // the 32 columns go to the staging buffer of their 64-column group (rows beyond M and columns beyond N
+    // are staged too and dropped by the store)
+    uint32_t buf = es.stg + (es.n_out & 1u) * GEMM_STG_BYTES;
+    if ((c & 32) == 0) buf = epi_stage_begin(es);
 #pragma unroll
-      for (int j = 0; j < 32; j += 8) {
-        const int col = n0 + c + j;
-        if (col < N) {  // N is a multiple of 8: a vector is entirely inside or outside
-          float f[8];
+    for (int j = 0; j < 32; j += 8) {
+      float f[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) f[i] = v[j + i];
-          if (EPI == EPI_RESIDUAL) {
-            Vec16<bf16> rv;
-            rv.raw = res_cur[j >> 3];
-            float rf[8];
-            rv.unpack(rf);
+      for (int i = 0; i < 8; ++i) f[i] = v[j + i];
+      if (EPI == EPI_RESIDUAL) {
+        Vec16<bf16> rv;
+        rv.raw = res_cur[j >> 3];
+        float rf[8];
+        rv.unpack(rf);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) f[i] += rf[i];
-          }
-          Vec16<bf16> o;
-          o.pack(f);
-          o.store(crow + col);
-        }
+        for (int i = 0; i < 8; ++i) f[i] += rf[i];
       }
+      Vec16<bf16> o;
+      o.pack(f);
+      epi_stage_put(buf, ((c & 32) >> 3) + (j >> 3), o.raw);
     }
+    if (c & 32) epi_stage_commit(es, buf, n0 + c - 32);
   }
   }  // epilogue kinds
 }

@@ -42,8 +42,10 @@ struct __align__(8) GemmBarriers {
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr int GEMM_SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 /*align slack*/ +
-                                (int)sizeof(GemmBarriers);
+constexpr int RING_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+// operand ring | output staging of the epilogue warps | barriers
+constexpr int GEMM_SMEM_BYTES = RING_BYTES + GEMM_STG_PER_CTA + 1024 /*align slack*/ + (int)sizeof(GemmBarriers);
+static_assert(GEMM_SMEM_BYTES <= 232448, "shared memory per CTA");
 
 // C is [M, ldc]; for EPI_SWIGLU the accumulator's columns [0,128) are gate features and
 // [128,256) the matching up features, and C receives 128 columns per tile.
@@ -53,7 +55,8 @@ template <int EPI, bool FP8>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
                          const __grid_constant__ CUtensorMap map_b0,
-                         const __grid_constant__ CUtensorMap map_b1, const bf16 *__restrict__ R,
+                         const __grid_constant__ CUtensorMap map_b1,
+                         const __grid_constant__ CUtensorMap map_c, const bf16 *__restrict__ R,
                          bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
                          const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
@@ -62,7 +65,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
   uint8_t *smem = smem_raw + pad;  // 1024-byte aligned: required by the 128B swizzle atoms
   uint8_t *smem_a = smem;
   uint8_t *smem_b = smem + STAGES * A_STAGE_BYTES;
-  GemmBarriers *bars = reinterpret_cast<GemmBarriers *>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  GemmBarriers *bars = reinterpret_cast<GemmBarriers *>(smem + RING_BYTES + GEMM_STG_PER_CTA);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Output tiles: columns per tile as seen by the caller.
@@ -87,6 +90,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
     tma_prefetch_desc(&map_a);
     tma_prefetch_desc(&map_b0);
     tma_prefetch_desc(&map_b1);
+    tma_prefetch_desc(&map_c);
   }
   if (warp == 1) {  // TMEM allocation by one whole warp; the same warp frees it at the end
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -171,6 +175,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
     int local = 0;
     bool ok = true;
     GemmWork w;
+    EpiStore es = {&map_c, smem_u32(smem + RING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
     for (; ok && gemm_work_item(local, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
@@ -178,9 +183,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
       const int m0 = m_idx * BM, n0 = n_idx * TILE_N_OUT;
       const int row = m0 + quarter * 32 + lane;
-      uint4 res_first[4] = {};
+      uint4 res_first[GEMM_RES_AHEAD][4] = {};
       if (EPI == EPI_RESIDUAL && w.mode != 1)  // requested now, needed once the accumulator is complete
-        gemm_residual_load(res_first, R, rope, row, n0, M, N, ldc);
+        gemm_residual_prefetch(res_first, R, rope, row, n0, M, N, ldc);
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -203,7 +208,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
           gemm_fixup_row(taddr, tail.partials + (size_t)(blockIdx.x + 1) * GEMM_SLOT_FLOATS, 1, n_parts, smem,
                          row_in_tile);
         }
-        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first);
+        es.y0 = m0 + quarter * 32;
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first, es);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + w.tail_idx, 1u) == 3u) {  // last warp through: clean for the next launch
@@ -216,6 +222,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[acc]));
     }
+    epi_stage_drain();  // the staging buffers must not go away under a store that still reads them
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -273,6 +280,8 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   LAZY_TRY(tma_map_2d(&ma, A, M, K, K, BKE, BM, EB));
   LAZY_TRY(tma_map_2d(&mb0, B0, N, K, K, BKE, BN / 2, EB));
   LAZY_TRY(tma_map_2d(&mb1, B1, N, K, K, BKE, BN / 2, EB));
+  CUtensorMap mc;  // the output: 64-column x 32-row boxes written from the epilogue's staging buffers
+  LAZY_TRY(tma_map_2d_bf16(&mc, C, M, N, N, 64, 32));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
   const GemmTail tail = plan_tail(tiles, cdiv(K, BKE), sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K,
@@ -285,7 +294,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
     LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
     attr_set = true;
   }
-  kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N,
+  kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, (const bf16 *)R, (bf16 *)C, M, N, K, N,
                                                   status, rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();

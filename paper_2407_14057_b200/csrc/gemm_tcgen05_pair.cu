@@ -36,13 +36,17 @@ struct __align__(8) PairBarriers {
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr int PAIR_SMEM_BYTES = PSTAGES * (PA_BYTES + PB_BYTES) + 1024 /*align slack*/ + (int)sizeof(PairBarriers);
+constexpr int PRING_BYTES = PSTAGES * (PA_BYTES + PB_BYTES);
+// operand ring | output staging of the epilogue warps | barriers
+constexpr int PAIR_SMEM_BYTES = PRING_BYTES + GEMM_STG_PER_CTA + 1024 /*align slack*/ + (int)sizeof(PairBarriers);
+static_assert(PAIR_SMEM_BYTES <= 232448, "shared memory per CTA");
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PTHREADS, 1)
 gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                               const __grid_constant__ CUtensorMap map_b0,
-                              const __grid_constant__ CUtensorMap map_b1, const bf16 *__restrict__ R,
+                              const __grid_constant__ CUtensorMap map_b1,
+                              const __grid_constant__ CUtensorMap map_c, const bf16 *__restrict__ R,
                               bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
                               const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
@@ -51,7 +55,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   uint8_t *smem = smem_raw + pad;
   uint8_t *smem_a = smem;
   uint8_t *smem_b = smem + PSTAGES * PA_BYTES;
-  PairBarriers *bars = reinterpret_cast<PairBarriers *>(smem + PSTAGES * (PA_BYTES + PB_BYTES));
+  PairBarriers *bars = reinterpret_cast<PairBarriers *>(smem + PRING_BYTES + GEMM_STG_PER_CTA);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();  // 0 = leader
@@ -76,6 +80,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     tma_prefetch_desc(&map_a);
     tma_prefetch_desc(&map_b0);
     tma_prefetch_desc(&map_b1);
+    tma_prefetch_desc(&map_c);
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(&bars->tmem_base), PTMEM_COLS);  // same warp in both CTAs
   tc_fence_before();
@@ -160,6 +165,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     int local = 0;
     bool ok = true;
     GemmWork w;
+    EpiStore es = {&map_c, smem_u32(smem + PRING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
     for (; ok && gemm_work_item(local, pair, n_pairs, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
@@ -167,9 +173,10 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       gemm_tile_coords(w.tile, m_tiles, n_tiles, tail.m_band, m_idx, n_idx);
       const int m0 = m_idx * (2 * PBM) + (int)rank * PBM, n0 = n_idx * TILE_N_OUT;
       const int row = m0 + quarter * 32 + lane;
-      uint4 res_first[4] = {};
+      es.y0 = m0 + quarter * 32;
+      uint4 res_first[GEMM_RES_AHEAD][4] = {};
       if (EPI == EPI_RESIDUAL && w.mode != 1)  // requested now, needed once the accumulator is complete
-        gemm_residual_load(res_first, R, rope, row, n0, M, N, ldc);
+        gemm_residual_prefetch(res_first, R, rope, row, n0, M, N, ldc);
       ok = mbar_wait(smem_u32(&bars->tmem_full[acc]), acc_phase, abort_flag, status, W_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -195,7 +202,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           gemm_fixup_row(taddr, tail.partials + (size_t)(2 * (pair + 1) + (int)rank) * GEMM_SLOT_FLOATS, 2, n_parts,
                          smem, row_in_tile);
         }
-        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first);
+        gemm_epilogue_row<EPI>(taddr, row, n0, M, N, ldc, R, C, rope, status, res_first, es);
         if (w.mode == 2) {
           __syncwarp();
           if (lane == 0 && atomicAdd(tail.done + flag_idx, 1u) == 3u) {
@@ -208,6 +215,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(cluster_map_shared(smem_u32(&bars->tmem_empty[acc]), 0));
     }
+    epi_stage_drain();  // the staging buffers must not go away under a store that still reads them
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -230,6 +238,8 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
   LAZY_TRY(tma_map_2d_bf16(&ma, A, M, K, K, PBK, PBM));
   LAZY_TRY(tma_map_2d_bf16(&mb0, B0, N, K, K, PBK, PBN / 2));
   LAZY_TRY(tma_map_2d_bf16(&mb1, B1, N, K, K, PBK, PBN / 2));
+  CUtensorMap mc;  // the output: 64-column x 32-row boxes written from the epilogue's staging buffers
+  LAZY_TRY(tma_map_2d_bf16(&mc, C, M, N, N, 64, 32));
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? PBN / 2 : PBN;
   const int tiles = cdiv(M, 2 * PBM) * cdiv(N, TILE_N_OUT);
   auto kfn = gemm_bf16_tcgen05_pair_kernel<EPI>;
@@ -257,7 +267,7 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
   const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), gemm_m_band(M, K, 2 * PBM), M, K,
                                   EPI == EPI_SWIGLU ? 8 : 0, scratch, scratch_bytes);
   const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
-  kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
+  kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
                                                     rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
