@@ -221,7 +221,7 @@ __device__ __forceinline__ bool gemm_tail_wait(const unsigned *flag, unsigned ta
 // group: measured, a 256-column tile then spent ~14 000 clocks in its residual epilogue, nearly all of it
 // waiting.  So a thread keeps GEMM_RES_AHEAD groups in flight: the first ones are requested before it waits
 // for the tile's accumulator, and each group consumed is replaced by the request GEMM_RES_AHEAD groups on.
-constexpr int GEMM_RES_AHEAD = 4;
+constexpr int GEMM_RES_AHEAD = 8;
 __device__ __forceinline__ void gemm_residual_load(uint4 (&r)[4], const bf16 *__restrict__ R, const RopeArgs &extra,
                                                    int row, int col0, int M, int N, int ldc) {
   if (row >= M) return;
