@@ -259,7 +259,7 @@ bool gemm_use_pair(int epi, int M, int N, int K, void *scratch, size_t scratch_b
             scratch, scratch_bytes, &w_one);
   plan_tail(cdiv(M, 2 * BM) * cdiv(N, tile_n), num_kb, max_pairs, 2, cdiv(M, 2 * BM), gemm_m_band(M, K, 2 * BM), M, K,
             extra, scratch, scratch_bytes, &w_pair);
-  const double pair_wave = epi == EPI_SWIGLU ? 1.0 : 0.94;
+  const double pair_wave = 0.95;
   return w_pair * pair_wave < w_one;  // a pair tile takes pair_wave x the time of a one-CTA tile
 }
 
