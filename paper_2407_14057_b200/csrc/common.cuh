@@ -214,7 +214,7 @@ bool gemm_res_rows_supported(int dtype, int M, int K);
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
-                         void *scratch = nullptr, size_t scratch_bytes = 0, int d_kv = 0);
+                         void *scratch = nullptr, size_t scratch_bytes = 0, int d_kv = 0, int kv_rows = 0);
 // Weight-streaming kernel for M <= 4 rows (decode); same results as the tensor-core GEMM.  With gain the
 // rows of A are RMS-normalised on the way in; with c_f32 the output is fp32 (LM head).
 bool gemv_small_m_eligible(int dtype, int M, int K);

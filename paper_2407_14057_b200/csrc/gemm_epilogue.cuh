@@ -17,7 +17,8 @@ struct RopeArgs {
   const int32_t *res_rows = nullptr;  // [M] row of R added to output row r (NULL: r)
   const int32_t *pos;     // [M] original positions
   const float2 *table;    // [max_pos][64] (cos, sin)
-  bf16 *kcache, *vcache;  // [rows, d_model]
+  bf16 *kcache, *vcache;  // [kv_rows, d_kv]
+  int kv_rows = 0;        // rows of the two caches (extent of their tensor maps)
   int32_t *kv_pos;        // position tag per cache row (may be NULL)
   const int32_t *kv_row;  // cache row of GEMM row r (NULL: r)
   int d_model, max_pos;
@@ -247,6 +248,7 @@ constexpr int GEMM_STG_BYTES = 4096;                       // 32 rows x 64 bf16
 constexpr int GEMM_STG_PER_CTA = 4 * 2 * GEMM_STG_BYTES;   // four epilogue warps, two buffers each
 struct EpiStore {
   const CUtensorMap *map;  // the output matrix: box 64 columns x 32 rows, 128-byte swizzle
+  const CUtensorMap *map_k, *map_v;  // QKV epilogue: the layer's K and V caches (same box), else unused
   uint32_t stg;            // shared-memory address of this warp's two buffers (1024-byte aligned)
   int y0;                  // first output row of the warp's 32-row block of the current tile
   uint32_t n_out;          // groups handed over so far: the next group takes buffer n_out & 1
@@ -265,14 +267,17 @@ __device__ __forceinline__ void epi_stage_put(uint32_t buf, int j, const uint4 &
                : "memory");
 }
 // Hands the staged group to the TMA unit: columns [x, x + 64) of rows [y0, y0 + 32).
-__device__ __forceinline__ void epi_stage_commit(EpiStore &es, uint32_t buf, int x) {
+__device__ __forceinline__ void epi_stage_commit(EpiStore &es, uint32_t buf, const CUtensorMap *map, int x, int y) {
   fence_proxy_async_smem();
   __syncwarp();
   if ((threadIdx.x & 31) == 0) {
-    tma_store_2d(es.map, buf, x, es.y0);
+    tma_store_2d(map, buf, x, y);
     bulk_commit_group();
   }
   ++es.n_out;
+}
+__device__ __forceinline__ void epi_stage_commit(EpiStore &es, uint32_t buf, int x) {
+  epi_stage_commit(es, buf, es.map, x, es.y0);
 }
 // Before the CTA exits: every store of this warp has completed.
 __device__ __forceinline__ void epi_stage_drain() {
@@ -311,14 +316,33 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
     const float osc = (rope.a_scale && row < M) ? rope.a_scale[row] * rope.w_scale : 1.f;
     bf16 *dst = sect == 0 ? crow + n0
                           : (sect == 1 ? rope.kcache : rope.vcache) + krow * rope.d_kv + col_in;
+    // Where the warp's 32 rows go as one box: q always (rows of C); k and v when all 32 rows are real and
+    // their cache rows are consecutive (one sequence, or a block inside one sequence of a packed batch).
+    // Otherwise k / v are stored row by row from registers.
+    const size_t krow0 = __shfl_sync(0xffffffffu, krow, 0);
+    const bool block_ok = rope.kv_rows > 0 &&
+                          __all_sync(0xffffffffu, row < M && krow == krow0 + (size_t)(threadIdx.x & 31));
+    const bool staged = sect == 0 || block_ok;
+    const CUtensorMap *omap = sect == 0 ? es.map : (sect == 1 ? es.map_k : es.map_v);
+    const int ox = sect == 0 ? n0 : col_in, oy = sect == 0 ? es.y0 : (int)krow0;
     if (sect == 2) {
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         float v[32];
         tmem_ld_32x32(taddr + (uint32_t)c, v);
-        if (row < M) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] *= osc;
+        for (int i = 0; i < 32; ++i) v[i] *= osc;
+        if (staged) {
+          uint32_t buf = es.stg + (es.n_out & 1u) * GEMM_STG_BYTES;
+          if ((c & 32) == 0) buf = epi_stage_begin(es);
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            Vec16<bf16> o;
+            o.pack(v + j);
+            epi_stage_put(buf, ((c & 32) >> 3) + (j >> 3), o.raw);
+          }
+          if (c & 32) epi_stage_commit(es, buf, omap, ox + c - 32, oy);
+        } else if (row < M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             Vec16<bf16> o;
@@ -331,9 +355,8 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
       const float2 *tab = rope.table + (size_t)p * 64;
 #pragma unroll 1
       for (int hc = 0; hc < BN; hc += 128) {  // the two heads of the tile
-        // q goes out through the staging buffers (columns [0,64) of the head in the first, [64,128) in the
-        // second); rotated k goes straight to its cache row, which need not be row `row` of anything
-        if (sect == 0) {
+        // a head goes out through both staging buffers: columns [0,64) in the first, [64,128) in the second
+        if (staged) {
           if ((threadIdx.x & 31) == 0) bulk_wait_group_read<0>();
           __syncwarp();
         }
@@ -351,7 +374,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
             lo[i + 1] = a1 * cs.z - b1 * cs.w;
             hi[i + 1] = b1 * cs.z + a1 * cs.w;
           }
-          if (sect == 0) {
+          if (staged) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
               Vec16<bf16> ol, oh;
@@ -371,12 +394,12 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
             }
           }
         }
-        if (sect == 0) {
+        if (staged) {
           fence_proxy_async_smem();
           __syncwarp();
           if ((threadIdx.x & 31) == 0) {
-            tma_store_2d(es.map, es.stg, n0 + hc, es.y0);
-            tma_store_2d(es.map, es.stg + GEMM_STG_BYTES, n0 + hc + 64, es.y0);
+            tma_store_2d(omap, es.stg, ox + hc, oy);
+            tma_store_2d(omap, es.stg + GEMM_STG_BYTES, ox + hc + 64, oy);
             bulk_commit_group();
           }
           es.n_out += 2;

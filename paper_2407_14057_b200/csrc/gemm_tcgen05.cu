@@ -56,7 +56,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
                          const __grid_constant__ CUtensorMap map_b0,
                          const __grid_constant__ CUtensorMap map_b1,
-                         const __grid_constant__ CUtensorMap map_c, const bf16 *__restrict__ R,
+                         const __grid_constant__ CUtensorMap map_c,
+                         const __grid_constant__ CUtensorMap map_k,
+                         const __grid_constant__ CUtensorMap map_v, const bf16 *__restrict__ R,
                          bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
                          const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
@@ -175,7 +177,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a,
     int local = 0;
     bool ok = true;
     GemmWork w;
-    EpiStore es = {&map_c, smem_u32(smem + RING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
+    EpiStore es = {&map_c, &map_k, &map_v, smem_u32(smem + RING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
     for (; ok && gemm_work_item(local, blockIdx.x, gridDim.x, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
@@ -282,6 +284,12 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
   LAZY_TRY(tma_map_2d(&mb1, B1, N, K, K, BKE, BN / 2, EB));
   CUtensorMap mc;  // the output: 64-column x 32-row boxes written from the epilogue's staging buffers
   LAZY_TRY(tma_map_2d_bf16(&mc, C, M, N, N, 64, 32));
+  CUtensorMap mk = mc, mv = mc;  // QKV epilogue: rotated k and v go to the layer's cache rows
+  if (EPI == EPI_QKV_ROPE && rope.kv_rows > 0) {
+    if (((uintptr_t)rope.kcache & 15) || ((uintptr_t)rope.vcache & 15)) return LAZY_E_BADARG;
+    LAZY_TRY(tma_map_2d_bf16(&mk, rope.kcache, rope.kv_rows, rope.d_kv, rope.d_kv, 64, 32));
+    LAZY_TRY(tma_map_2d_bf16(&mv, rope.vcache, rope.kv_rows, rope.d_kv, rope.d_kv, 64, 32));
+  }
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int tiles = cdiv(M, BM) * cdiv(N, TILE_N_OUT);
   const GemmTail tail = plan_tail(tiles, cdiv(K, BKE), sm_count(), 1, cdiv(M, BM), gemm_m_band(M, K, BM), M, K,
@@ -294,7 +302,7 @@ int launch_tc(cudaStream_t st, const void *A, const void *B0, const void *B1, co
     LAZY_CUDA_OK(cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES));
     attr_set = true;
   }
-  kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, (const bf16 *)R, (bf16 *)C, M, N, K, N,
+  kfn<<<grid, GEMM_THREADS, GEMM_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, mk, mv, (const bf16 *)R, (bf16 *)C, M, N, K, N,
                                                   status, rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
@@ -360,10 +368,11 @@ bool gemm_qkv_rope_eligible(int dtype, int d_model, int head_dim, int d_kv) {
 int launch_gemm_qkv_rope(cudaStream_t st, const void *h, const void *w_qkv, void *qkv, const int32_t *pos,
                          const float *table, void *kcache, void *vcache, int32_t *kv_pos,
                          const int32_t *kv_row, int M, int d_model, int max_pos, DevStatus *status,
-                         void *scratch, size_t scratch_bytes, int d_kv) {
+                         void *scratch, size_t scratch_bytes, int d_kv, int kv_rows) {
   if (M == 0) return LAZY_OK;
   if (d_kv <= 0) d_kv = d_model;
   RopeArgs r;
+  r.kv_rows = kv_rows > 0 ? kv_rows : 0;  // 0: extent unknown, k and v are stored row by row
   r.d_kv = d_kv;
   r.pos = pos;
   r.table = (const float2 *)table;

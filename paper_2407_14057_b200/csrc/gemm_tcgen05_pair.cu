@@ -46,7 +46,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PTHREADS, 1)
 gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                               const __grid_constant__ CUtensorMap map_b0,
                               const __grid_constant__ CUtensorMap map_b1,
-                              const __grid_constant__ CUtensorMap map_c, const bf16 *__restrict__ R,
+                              const __grid_constant__ CUtensorMap map_c,
+                         const __grid_constant__ CUtensorMap map_k,
+                         const __grid_constant__ CUtensorMap map_v, const bf16 *__restrict__ R,
                               bf16 *__restrict__ C, int M, int N, int K, int ldc, DevStatus *status,
                               const RopeArgs rope, const GemmTail tail) {
   extern __shared__ uint8_t smem_raw[];
@@ -165,7 +167,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     int local = 0;
     bool ok = true;
     GemmWork w;
-    EpiStore es = {&map_c, smem_u32(smem + PRING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
+    EpiStore es = {&map_c, &map_k, &map_v, smem_u32(smem + PRING_BYTES) + (uint32_t)(quarter * 2 * GEMM_STG_BYTES), 0, 0u};
     for (; ok && gemm_work_item(local, pair, n_pairs, num_tiles, num_kb, tail, w); ++local) {
       const int acc = local & 1;
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
@@ -240,6 +242,12 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
   LAZY_TRY(tma_map_2d_bf16(&mb1, B1, N, K, K, PBK, PBN / 2));
   CUtensorMap mc;  // the output: 64-column x 32-row boxes written from the epilogue's staging buffers
   LAZY_TRY(tma_map_2d_bf16(&mc, C, M, N, N, 64, 32));
+  CUtensorMap mk = mc, mv = mc;  // QKV epilogue: rotated k and v go to the layer's cache rows
+  if (EPI == EPI_QKV_ROPE && rope.kv_rows > 0) {
+    if (((uintptr_t)rope.kcache & 15) || ((uintptr_t)rope.vcache & 15)) return LAZY_E_BADARG;
+    LAZY_TRY(tma_map_2d_bf16(&mk, rope.kcache, rope.kv_rows, rope.d_kv, rope.d_kv, 64, 32));
+    LAZY_TRY(tma_map_2d_bf16(&mv, rope.vcache, rope.kv_rows, rope.d_kv, rope.d_kv, 64, 32));
+  }
   constexpr int TILE_N_OUT = (EPI == EPI_SWIGLU) ? PBN / 2 : PBN;
   const int tiles = cdiv(M, 2 * PBM) * cdiv(N, TILE_N_OUT);
   auto kfn = gemm_bf16_tcgen05_pair_kernel<EPI>;
@@ -267,7 +275,7 @@ int launch_pair(cudaStream_t st, const void *A, const void *B0, const void *B1, 
   const GemmTail tail = plan_tail(tiles, cdiv(K, PBK), max_pairs, 2, cdiv(M, 2 * PBM), gemm_m_band(M, K, 2 * PBM), M, K,
                                   EPI == EPI_SWIGLU ? 8 : 0, scratch, scratch_bytes);
   const int pairs = (tiles < max_pairs && tail.tail_units == 0) ? tiles : max_pairs;
-  kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
+  kfn<<<2 * pairs, PTHREADS, PAIR_SMEM_BYTES, st>>>(ma, mb0, mb1, mc, mk, mv, (const bf16 *)R, (bf16 *)C, M, N, K, N, status,
                                                     rope, tail);
   LAZY_COUNT_LAUNCH();
   return launch_ok();

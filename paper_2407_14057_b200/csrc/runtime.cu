@@ -567,6 +567,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
         r.pos = pos;
         r.table = (const float2 *)c->rope_table;
         r.kcache = (bf16 *)kc;
+        r.kv_rows = c->cap_kv;
         r.vcache = (bf16 *)vc;
         r.kv_pos = kvp;
         r.kv_row = c->kv_row[g];
@@ -585,7 +586,7 @@ int lazy_prefill_run(lazy_ctx *c, void *stream, const int32_t *d_prompt_ids,
       // rotary embedding and the K/V cache write ride in the projection's epilogue
       TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
             launch_gemm_qkv_rope(st, c->h, c->w_qkv[l], c->qkv, pos, c->rope_table, kc, vc, kvp, c->kv_row[g], n,
-                                 d, c->max_pos, status, c->gemm_scratch, c->gemm_scratch_bytes, dkv));
+                                 d, c->max_pos, status, c->gemm_scratch, c->gemm_scratch_bytes, dkv, c->cap_kv));
     } else {
       TIMED(LAZY_K_GEMM_QKV, 2.0 * n * qc * d, 0,
             launch_gemm(st, dt, c->h, c->w_qkv[l], nullptr, c->qkv, n, qc, d, status, c->gemm_scratch,
