@@ -681,6 +681,48 @@ def run_other_workload(args):
         out["gemm"] = rows
         out["note"] = "isolated back-to-back launches, weights rotating over three copies; impl: auto = chosen by shape"
 
+    elif args.workload == "gemm-sustained":
+        # Every projection shape of the bench line looped for about a second, so that the card settles at its
+        # power cap as it does inside the step, with the SM clock sampled during each loop; beside it the
+        # library's plain GEMM (torch.matmul, no epilogue) on the same operands, as the per-shape reference that
+        # the single roofline denominator (an 8192^3 product) cannot give.
+        ws = B.lazy_k_gemm_scratch()
+        row_list = [int(r) for r in args.rows.split(",")] if args.rows else [1013, 1688, 2364, 3376]
+
+        def sustained(fn, flops):
+            per = _event_ms(fn, 10, 5)
+            iters = max(20, int(1000.0 / per))
+            cs = ClockSampler(0)
+            cs.start()
+            ms = _event_ms(fn, iters, 0)
+            clk = cs.stop()
+            return {"us": round(ms * 1e3, 1), "tflops": round(flops / (ms * 1e-3) / 1e12), "sm_mhz": clk["sm_mhz"]}
+
+        rows = []
+        for M in row_list:
+            for name, N, K, sw in (("qkv", 12288, 4096, False), ("o", 4096, 4096, False),
+                                   ("gate_up", 11008, 4096, True), ("down", 4096, 11008, False)):
+                A = torch.randn(M, K, device="cuda").bfloat16()
+                Ws = [(torch.randn(N, K, device="cuda") * 0.02).bfloat16() for _ in range(3)]
+                Us = [(torch.randn(N, K, device="cuda") * 0.02).bfloat16() for _ in range(3)] if sw else None
+                W2 = [torch.cat([Ws[i], Us[i]], 0) for i in range(3)] if sw else Ws
+                R = None if sw else torch.randn(M, N, device="cuda").bfloat16()
+                Cm = torch.empty(M, N, device="cuda", dtype=torch.bfloat16)
+                C2 = torch.empty(M, N * (2 if sw else 1), device="cuda", dtype=torch.bfloat16)
+                fl = 2.0 * M * N * K * (2 if sw else 1)
+                if sw:
+                    ours = sustained(lambda i: B.lazy_k_gemm_swiglu(A, Ws[i % 3], Us[i % 3], out=Cm, scratch=ws), fl)
+                else:
+                    ours = sustained(lambda i: B.lazy_k_gemm(A, Ws[i % 3], R, out=Cm, scratch=ws), fl)
+                lib_ref = sustained(lambda i: torch.matmul(A, W2[i % 3].t(), out=C2), fl)
+                rows.append({"M": M, "product": name, "N": N, "K": K, "ours": ours, "library_plain_gemm": lib_ref})
+                del Ws, Us, W2
+                torch.cuda.empty_cache()
+        B.lazy_device_status()
+        out["gemm_sustained"] = rows
+        out["note"] = ("about one second of back-to-back launches per entry (power-capped clocks, sampled); the library "
+                       "entry is a plain product without residual / SwiGLU / rotary epilogue")
+
     out["clocks"] = sampler.stop()
     print(json.dumps(out), flush=True)
 
@@ -698,7 +740,7 @@ def main():
     ap.add_argument("--fp8", action="store_true", help=argparse.SUPPRESS)   # the leg runs by default
     ap.add_argument("--cpu-sample", action="store_true",
                     help="time the oracle on the bounded sample only (about 15 s) instead of the whole workload")
-    ap.add_argument("--workload", default="prefill", choices=["prefill", "decode", "batch8", "prune-op", "gemv", "gemm"],
+    ap.add_argument("--workload", default="prefill", choices=["prefill", "decode", "batch8", "prune-op", "gemv", "gemm", "gemm-sustained"],
                     help="prefill = the bench line; the others time the remaining configurations and single "
                          "kernels through the public binding and print one JSON object each")
     ap.add_argument("--rows", default="", help="--workload gemm: comma-separated row counts (default: the bench's)")
