@@ -70,6 +70,28 @@ def test_gemm_bf16_tensor_core(M, N, K, residual):
     assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-3 * np.max(np.abs(ref)))
 
 
+@pytest.mark.parametrize("impl", [2, 3])
+@pytest.mark.parametrize("M,N,K", [(130, 8, 64), (37, 72, 128), (200, 200, 256), (129, 136, 64), (300, 264, 320)])
+def test_gemm_bf16_narrow_and_ragged_output_widths(M, N, K, impl):
+    """Outputs narrower than one 64-column store box, or ending inside one, with row counts that end inside a
+    32-row box: the epilogues stage whole boxes and rely on the store unit to drop what lies outside the
+    matrix, so nothing may be written beyond it (the output sits inside a larger poisoned buffer) and every
+    element inside must be right.  Both tensor-core kernels, with and without the residual."""
+    A = _rand((M, K), 80, torch.bfloat16).cuda()
+    Bm = _rand((N, K), 81, torch.bfloat16, 0.05).cuda()
+    R = _rand((M, N), 82, torch.bfloat16).cuda()
+    ws = B.lazy_k_gemm_scratch()
+    ref0 = O.f64(to_np(A)) @ O.f64(to_np(Bm)).T
+    for res in (None, R):
+        guard = torch.full(((M + 64) * N + 256,), 777.0, dtype=torch.bfloat16, device="cuda")
+        out = guard[128:128 + M * N].view(M, N)
+        B.lazy_k_gemm(A, Bm, res, impl=impl, out=out, scratch=ws)
+        B.lazy_device_status()
+        ref = ref0 + (O.f64(to_np(res)) if res is not None else 0.0)
+        assert rel_err(to_np(out), ref) < BF16_STEP_TOL
+        assert torch.all(guard[:128] == 777.0) and torch.all(guard[128 + M * N:] == 777.0)
+
+
 def test_gemm_bf16_in_place_residual_and_cuda_core_cross_check():
     M, N, K = 200, 512, 1408
     A = _rand((M, K), 6, torch.bfloat16).cuda()
