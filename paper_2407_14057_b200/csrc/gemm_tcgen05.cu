@@ -8,13 +8,15 @@
 //               tcgen05.mma (M128 N256 K16) from one lane; tcgen05.commit releases ring stages
 //               ("empty" barriers) and publishes finished accumulators ("tmem full");
 //   warps 2-5   epilogue: tcgen05.ld their 32-lane quarter of the accumulator, apply the
-//               epilogue (plain / + residual / SiLU(gate)*up), convert to bf16, 16-byte stores.
+//               epilogue (plain / + residual / SiLU(gate)*up / rotary), convert to bf16, stage 64-column
+//               groups of the warp's 32 rows in shared memory and hand them to the TMA unit to store.
 // The second accumulator lets the epilogue of tile i overlap the MMAs of tile i+1.
 // Work items come from gemm_epilogue.cuh: whole tiles in a banded order, then, when it pays, K ranges
 // of the last partial wave of tiles (a dumped partial accumulator, or the part that adds the dumps and
 // finishes the tile).  The host side picks, per launch, this kernel or the CTA-pair kernel of
 // gemm_tcgen05_pair.cu (gemm_use_pair), and the weight-streaming kernel for up to four rows.
-// Ragged M, N, K rely on TMA zero fill for loads and on predicated stores.
+// Ragged M, N, K rely on TMA zero fill for loads and on the TMA unit dropping what a store box holds
+// beyond the matrix (row-by-row stores, where they remain, are predicated).
 // Every mbarrier wait is bounded (wall-clock limit); on expiry the kernel records
 // LAZY_E_TIMEOUT in the status word, every role leaves its loop, TMEM is released and the CTA
 // exits.  No cluster launch, no multicast.
