@@ -118,7 +118,8 @@ int lazy_prefill_init(const lazy_model_cfg *cfg, const lazy_weights *w, const la
  * Writes fp32 next-token logits [n_seqs, vocab] to d_logits (device) and leaves per-layer KV
  * caches and Aux Caches in the workspace for decode.  Resets any earlier generation state.
  * Row counts follow from (lengths, schedule) alone, so nothing is read back: the call only
- * enqueues work on `stream`. */
+ * enqueues work on `stream`.  `stream` must not be capturing into a CUDA graph: the call copies small
+ * index tables from host memory that does not outlive it, and a replay would read that memory again. */
 int lazy_prefill_run(lazy_ctx *ctx, void *stream, const int32_t *d_prompt_ids,
                      const int32_t *h_cu_seqlens, int32_t n_seqs, float *d_logits);
 

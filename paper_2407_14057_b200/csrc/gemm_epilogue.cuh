@@ -305,6 +305,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
     const int col_in = n0 - (sect == 0 ? 0 : (sect == 1 ? rope.d_model : rope.d_model + rope.d_kv));
     int p = 0;
     size_t krow = 0;
+    bool kv_valid = true;  // false: the row's cache row lies outside the caches; its k / v are dropped
     if (row < M) {
       p = rope.pos[row];
       if (p < 0 || p >= rope.max_pos) {
@@ -312,6 +313,13 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
         p = 0;
       }
       krow = rope.kv_row ? (size_t)rope.kv_row[row] : (size_t)row;
+      // a cache row outside the caches (a corrupted row table) is reported, and the row's k / v are dropped
+      // instead of being stored out of range (a box store must not start at such a row either)
+      if (rope.kv_rows > 0 && krow >= (size_t)rope.kv_rows) {
+        dev_fail(status, LAZY_E_CAPACITY, W_ROPE_POS, row, (int)krow);
+        kv_valid = false;
+        krow = 0;
+      }
     }
     const float osc = (rope.a_scale && row < M) ? rope.a_scale[row] * rope.w_scale : 1.f;
     bf16 *dst = sect == 0 ? crow + n0
@@ -320,8 +328,8 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
     // their cache rows are consecutive (one sequence, or a block inside one sequence of a packed batch).
     // Otherwise k / v are stored row by row from registers.
     const size_t krow0 = __shfl_sync(0xffffffffu, krow, 0);
-    const bool block_ok = rope.kv_rows > 0 &&
-                          __all_sync(0xffffffffu, row < M && krow == krow0 + (size_t)(threadIdx.x & 31));
+    const bool block_ok = rope.kv_rows > 0 && krow0 + 32 <= (size_t)rope.kv_rows &&
+                          __all_sync(0xffffffffu, row < M && kv_valid && krow == krow0 + (size_t)(threadIdx.x & 31));
     const bool staged = sect == 0 || block_ok;
     const CUtensorMap *omap = sect == 0 ? es.map : (sect == 1 ? es.map_k : es.map_v);
     const int ox = sect == 0 ? n0 : col_in, oy = sect == 0 ? es.y0 : (int)krow0;
@@ -342,7 +350,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
             epi_stage_put(buf, ((c & 32) >> 3) + (j >> 3), o.raw);
           }
           if (c & 32) epi_stage_commit(es, buf, omap, ox + c - 32, oy);
-        } else if (row < M) {
+        } else if (row < M && kv_valid) {
 #pragma unroll
           for (int j = 0; j < 32; j += 8) {
             Vec16<bf16> o;
@@ -383,7 +391,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
               epi_stage_put(es.stg, (o >> 3) + (j >> 3), ol.raw);
               epi_stage_put(es.stg + GEMM_STG_BYTES, (o >> 3) + (j >> 3), oh.raw);
             }
-          } else if (row < M) {
+          } else if (row < M && kv_valid) {
 #pragma unroll
             for (int j = 0; j < 32; j += 8) {
               Vec16<bf16> ol, oh;
@@ -405,7 +413,7 @@ __device__ __forceinline__ void gemm_epilogue_row(uint32_t taddr, int row, int n
           es.n_out += 2;
         }
       }
-      if (sect == 1 && col_in == 0 && row < M && rope.kv_pos) rope.kv_pos[krow] = p;
+      if (sect == 1 && col_in == 0 && row < M && kv_valid && rope.kv_pos) rope.kv_pos[krow] = p;
     }
   } else {
   const float asc = (rope.a_scale && row < M) ? rope.a_scale[row] : 1.f;
