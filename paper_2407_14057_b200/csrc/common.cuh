@@ -271,7 +271,8 @@ int launch_score(cudaStream_t st, int dtype, const void *q, int ldq, const void 
 // General form (decode): sequence s scores the key LIST key_rows[cu_q[s] .. cu_q[s+1]) (cache rows)
 // with the query in row q_rows[s].
 int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, const int32_t *cu_q,
-                      int n_seqs, int n_total, int n_heads, float *scores);
+                      int n_seqs, int n_total, int n_heads, float *scores, int n_layers = 1,
+                      size_t layer_stride = 0, size_t scores_stride = 0);
 // Split-key attention for one to eight query rows over key lists (decode); leaves the score row's
 // logits and softmax statistics for launch_score_mean.
 bool attention_decode_eligible(int dtype, int head_dim, int n_rows, int max_ctx);

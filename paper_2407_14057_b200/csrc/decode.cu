@@ -59,13 +59,22 @@ __global__ void map_build_kernel(const int32_t *tags, int32_t *map, int base, in
 // own).  Thread i < n (context list): the cache row of this layer holding that position.  A position
 // that is in flight gets its row from xmap (the row is being appended by this very step), so no thread
 // depends on a map entry another thread of this launch writes.
+// blockIdx.y = layer within the segment (the layers up to the next re-selection run on the same in-flight rows
+// and the same context list, so their bookkeeping is done in one launch): layer y appends at append_at +
+// y * append_stride, owns the map kv_map + y * rows_stride and receives kv_row_new / ctx_rows + y * rows_stride;
+// the visible lengths do not depend on the layer and are written by layer 0.
 __global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, const int32_t *seq_base,
                                    const int32_t *append_at, const int32_t *xpos, const int32_t *ctx_pos,
                                    const int32_t *xmap, int n_seqs, int m, int n, int32_t *kv_row_new,
-                                   int32_t *kv_map, int32_t *q_kvlen, int32_t *ctx_rows, DevStatus *status) {
+                                   int32_t *kv_map, int32_t *q_kvlen, int32_t *ctx_rows, DevStatus *status,
+                                   int append_stride, size_t rows_stride) {
   // the projection that follows is a programmatic dependent: it may start fetching weights now and
   // still waits for this grid before it reads the rows computed here; this grid is one too
   LAZY_PDL_ENTER();
+  append_at += (size_t)blockIdx.y * append_stride;
+  kv_map += (size_t)blockIdx.y * rows_stride;
+  kv_row_new += (size_t)blockIdx.y * rows_stride;
+  ctx_rows += (size_t)blockIdx.y * rows_stride;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     const int s = seq_of(cu_ctx, n_seqs, i);
@@ -91,7 +100,7 @@ __global__ void dec_prepare_kernel(const int32_t *cu_x, const int32_t *cu_ctx, c
       const int mid = (lo + hi) >> 1;
       if (list[mid] <= p) lo = mid + 1; else hi = mid;
     }
-    q_kvlen[i] = lo;
+    if (blockIdx.y == 0) q_kvlen[i] = lo;
   }
 }
 
@@ -263,9 +272,12 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
 
   // ---- integer scratch
   int32_t *I = c->dec_i32;
-  int32_t *ctx_pos = I, *ctx_pos2 = I + (size_t)KV, *ctx_rows = I + (size_t)2 * KV;
+  int32_t *ctx_pos = I, *ctx_pos2 = I + (size_t)KV;  // (slot 2 of the scratch is unused)
   int32_t *xpos = I + (size_t)3 * KV, *xpos2 = I + (size_t)4 * KV, *q_kvlen = I + (size_t)5 * KV;
-  int32_t *kv_row_new = I + (size_t)6 * KV, *new_src = I + (size_t)7 * KV, *xmap = I + (size_t)8 * KV;
+  int32_t *new_src = I + (size_t)7 * KV, *xmap = I + (size_t)8 * KV;  // (slot 6 unused)
+  // per layer: the cache rows the in-flight rows append to, and the cache rows of the context list
+  auto kv_row_new_of = [&](int l) { return c->dec_seg + (size_t)l * KV; };
+  auto ctx_rows_of = [&](int l) { return c->dec_seg + (size_t)(L + l) * KV; };
   int32_t *selmark = I + (size_t)9 * KV, *keep_idx = I + (size_t)10 * KV, *drop_idx = I + (size_t)11 * KV;
   int32_t *new_pos = I + (size_t)12 * KV, *drop_src = I + (size_t)13 * KV, *drop_dst = I + (size_t)14 * KV;
   int32_t *revived = I + (size_t)15 * KV;
@@ -323,7 +335,11 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
   KLAUNCH_OK();
 
   char *x = c->x, *x2 = c->x2;
+  int seg_end = -1;        // last layer of the segment whose bookkeeping has been launched
+  int score_from = -1;     // first layer of the segment whose head means are still to be taken (-1: none pending)
+  size_t score_stride = 0; // floats between two layers' logits + statistics in the score scratch
   for (int l = 0; l < L; ++l) {
+    int32_t *kv_row_new = kv_row_new_of(l), *ctx_rows = ctx_rows_of(l);
     char *kc = c->kcache + (size_t)l * KV * c->kv_row_bytes();
     char *vc = c->vcache + (size_t)l * KV * c->kv_row_bytes();
     int32_t *kvp = c->kv_pos + (size_t)l * KV;
@@ -337,14 +353,25 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     if (M > c->cap_rows) return LAZY_E_CAPACITY;
     c->stats.rows_computed[l] = M;
 
-    {  // bookkeeping first: the projection below may already write the rows' K/V into their cache rows
+    if (l > seg_end) {
+      // Bookkeeping first (the projection below may already write the rows' K/V into their cache rows), for
+      // every layer up to the next re-selection at once: they all run on these in-flight rows and this context.
+      seg_end = l;
+      while (seg_end + 1 < L && c->point_at[seg_end + 1] < 0) ++seg_end;
+      for (int ll = l + 1; ll <= seg_end; ++ll)
+        for (int s = 0; s < S; ++s)
+          if (c->kv_count[ll][s] + m_of[s] > c->prompt_len[s] + c->cfg.max_new_tokens) return LAZY_E_CAPACITY;
       const int n_thr = M > n_ctx ? M : n_ctx;
-      LAZY_TRY(launch_pdl(dec_prepare_kernel, dim3(cdiv(n_thr, 256)), dim3(256), 0, st, (const int32_t *)dtab(T_CU_X),
-                          (const int32_t *)dtab(T_CU_CTX), (const int32_t *)dtab(T_BASE),
-                          (const int32_t *)(d_append + (size_t)l * W), (const int32_t *)xpos,
-                          (const int32_t *)ctx_pos, (const int32_t *)xmap, S, M, n_ctx, kv_row_new, kvm, q_kvlen,
-                          ctx_rows, status));
+      LAZY_TRY(launch_pdl(dec_prepare_kernel, dim3(cdiv(n_thr, 256), seg_end - l + 1), dim3(256), 0, st,
+                          (const int32_t *)dtab(T_CU_X), (const int32_t *)dtab(T_CU_CTX),
+                          (const int32_t *)dtab(T_BASE), (const int32_t *)(d_append + (size_t)l * W),
+                          (const int32_t *)xpos, (const int32_t *)ctx_pos, (const int32_t *)xmap, S, M, n_ctx,
+                          kv_row_new, kvm, q_kvlen, ctx_rows, status, W, (size_t)KV));
       KLAUNCH_OK();
+      // room for every layer's score logits and statistics side by side? then their head means wait for the
+      // segment's last layer
+      score_stride = align_up((size_t)c->H * n_ctx + (size_t)2 * S * c->H, 64);
+      score_from = score_stride * (size_t)(seg_end - l + 1) <= c->score_scratch_cap ? l : -1;
     }
     if (gemv_small_m_eligible(dt, M, d) && c->dh == 128 && dkv % 128 == 0) {
       // one to four rows: one weight-streaming kernel does RMSNorm, the projection, RoPE and the cache write
@@ -368,11 +395,18 @@ int decode_step_impl(lazy_ctx *c, cudaStream_t st, const int32_t *d_new_ids, flo
     // the MLP activation buffer is idle during attention: it holds the split partials
     if (attention_decode_eligible(dt, c->dh, M, max_ctx) &&
         attention_decode_scratch_floats(M, c->H, max_ctx) * 4 <= (size_t)c->cap_rows * c->F * c->eb) {
-      float *logits = c->score_scratch, *stats = c->score_scratch + (size_t)c->H * n_ctx;
+      float *logits = c->score_scratch + (score_from >= 0 ? (size_t)(l - score_from) * score_stride : 0);
+      float *stats = logits + (size_t)c->H * n_ctx;
       LAZY_TRY(launch_attention_decode(st, c->qkv, qc, kc, vc, dkv, c->attn, d, dtab(T_CU_X), dtab(T_CU_CTX),
                                        ctx_rows, q_kvlen, dtab(T_QROW), S, M, n_ctx, max_ctx, c->H,
                                        (float *)c->act, logits, stats, c->Hkv));
-      LAZY_TRY(launch_score_mean(st, logits, stats, dtab(T_CU_CTX), S, n_ctx, c->H, sc));
+      if (score_from < 0) {
+        LAZY_TRY(launch_score_mean(st, logits, stats, dtab(T_CU_CTX), S, n_ctx, c->H, sc));
+      } else if (l == seg_end) {  // Eq. 1 head means of the whole segment, before its scores are needed
+        LAZY_TRY(launch_score_mean(st, c->score_scratch, c->score_scratch + (size_t)c->H * n_ctx, dtab(T_CU_CTX), S,
+                                   n_ctx, c->H, c->scores + (size_t)score_from * KV, seg_end - score_from + 1,
+                                   score_stride, (size_t)KV));
+      }
     } else {
       // many rows in flight: the tile kernel, with the key list cut into slices when there are too few
       // (query tile, head) pairs to fill the machine

@@ -162,7 +162,8 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
     size_t a = score_scratch_floats(c->S, c->cap_kv, c->H);
     c->score_layer_stride = align_up(attn_score_scratch_floats(c->S, c->H, c->cap_rows / 64 + 1), 64);
     size_t b = c->score_layer_stride * (size_t)c->L;
-    c->score_scratch = (float *)k.take((a > b ? a : b) * 4);
+    c->score_scratch_cap = a > b ? a : b;
+    c->score_scratch = (float *)k.take(c->score_scratch_cap * 4);
   }
   c->keep_idx.assign(P, nullptr);
   c->drop_idx.assign(P, nullptr);
@@ -186,6 +187,7 @@ static size_t carve(lazy_ctx *c, char *base, bool with_capture) {
   c->aux_map = (int32_t *)k.take((size_t)P * KV * 4);
   c->dec_i32 = (int32_t *)k.take((size_t)16 * KV * 4 + (size_t)(16 * 2 + L) * (c->S + 1) * 4);
   c->dec_f32 = (float *)k.take((size_t)2 * KV * 4);
+  c->dec_seg = (int32_t *)k.take((size_t)2 * L * KV * 4);
   c->a8 = (uint8_t *)k.take(c->dtype == LAZY_BF16 ? R * (size_t)(c->F > c->d ? c->F : c->d) : 0);
   c->a8_scale = (float *)k.take(c->dtype == LAZY_BF16 ? R * 4 : 0);
   c->gemm_scratch_bytes = c->dtype == LAZY_BF16 ? gemm_scratch_bytes() : 0;

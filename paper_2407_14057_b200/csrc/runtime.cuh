@@ -51,6 +51,8 @@ struct lazy_ctx {
   int32_t *aux_map;  // [P, cap_kv]: Aux row of (sequence base + position), -1 if absent
   std::vector<int32_t *> revived_pos;  // [P] x [cap_kv]: per in-flight row after a boundary, its
                                        // position if it came from the Aux Cache, else -1
+  int32_t *dec_seg;  // [2][L][cap_kv]: per layer of a decode segment, the cache rows appended to and the context's rows
+  size_t score_scratch_cap;  // floats in score_scratch
   int32_t *dec_i32;  // integer scratch of the decode step
   float *dec_f32;
   bool select_threshold = false;  // threshold reading of the selection: ties at the scheduled rank all survive

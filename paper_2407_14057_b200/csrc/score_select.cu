@@ -97,10 +97,16 @@ __global__ void score_stats_kernel(const float *__restrict__ logits, const int32
   }
 }
 
-// 8 lanes per key, each over a slice of the heads.
+// 8 lanes per key, each over a slice of the heads.  blockIdx.y = one of several layers whose logits / statistics
+// lie layer_stride floats apart and whose scores lie scores_stride floats apart (decode: the layers between two
+// re-selections attend over the same context, so their head means are taken in one launch).
 __global__ void score_mean_kernel(const float *__restrict__ logits, const float *__restrict__ stats,
                                   const int32_t *__restrict__ cu_q, int n_seqs, int n_total,
-                                  int n_heads, float *__restrict__ scores) {
+                                  int n_heads, float *__restrict__ scores, size_t layer_stride,
+                                  size_t scores_stride) {
+  logits += (size_t)blockIdx.y * layer_stride;
+  stats += (size_t)blockIdx.y * layer_stride;
+  scores += (size_t)blockIdx.y * scores_stride;
   // releases a following programmatic dependent (decode: the output projection's weight streaming can start
   // its weight reads now) and, launched as one itself, waits for the kernel before it
   LAZY_PDL_ENTER();
@@ -430,7 +436,7 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
   score_stats_kernel<<<dim3(n_heads, n_seqs), 256, 0, st>>>(logits, cu_q, n_total, n_heads, stats);
   LAZY_COUNT_LAUNCH();
   score_mean_kernel<<<cdiv(n_total, 32), 256, 0, st>>>(logits, stats, cu_q, n_seqs, n_total, n_heads,
-                                                        scores);
+                                                        scores, (size_t)0, (size_t)0);
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
@@ -438,11 +444,12 @@ int launch_score_ex(cudaStream_t st, int dtype, const void *q, int ldq, const vo
 // Eq. 1 mean over heads from logits [H, n_total] and per-(sequence, head) (max, 1/sum) pairs that
 // another kernel already produced.
 int launch_score_mean(cudaStream_t st, const float *logits, const float *stats, const int32_t *cu_q,
-                      int n_seqs, int n_total, int n_heads, float *scores) {
-  if (n_total == 0) return LAZY_OK;
-  if (!logits || !stats || !cu_q || !scores) return LAZY_E_BADARG;
-  LAZY_TRY(launch_pdl(score_mean_kernel, dim3(cdiv(n_total, 32)), dim3(256), 0, st, logits, stats, cu_q, n_seqs,
-                      n_total, n_heads, scores));
+                      int n_seqs, int n_total, int n_heads, float *scores, int n_layers, size_t layer_stride,
+                      size_t scores_stride) {
+  if (n_total == 0 || n_layers == 0) return LAZY_OK;
+  if (!logits || !stats || !cu_q || !scores || n_layers < 1) return LAZY_E_BADARG;
+  LAZY_TRY(launch_pdl(score_mean_kernel, dim3(cdiv(n_total, 32), n_layers), dim3(256), 0, st, logits, stats, cu_q,
+                      n_seqs, n_total, n_heads, scores, layer_stride, scores_stride));
   LAZY_COUNT_LAUNCH();
   return launch_ok();
 }
