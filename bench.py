@@ -610,6 +610,15 @@ def run_other_workload(args):
         idx = res["keep_idx"][:n_keep].contiguous()
         g_out = torch.empty((n_keep, d), dtype=torch.bfloat16, device="cuda")
         g_ms = _event_ms(lambda i: B.lazy_k_gather_rows(srcs[i % 8], idx, out=g_out), 40, 8)
+        # the same kernel on enough rows for the launch to outlast the host's per-call cost (a 40 MB gather is over
+        # before the next call has been issued): a random permutation of 32768 rows, sources rotating
+        big_n = 32768
+        big_src = [torch.randn((big_n, d), device="cuda").bfloat16() for _ in range(3)]
+        big_idx = torch.randperm(big_n, device="cuda").to(torch.int32)
+        big_out = torch.empty((big_n, d), dtype=torch.bfloat16, device="cuda")
+        gb_ms = _event_ms(lambda i: B.lazy_k_gather_rows(big_src[i % 3], big_idx, out=big_out), 20, 5)
+        del big_src, big_out
+        torch.cuda.empty_cache()
         sc = synth.make_scores(n, "lognormal", 5).cuda()
         cu_in = torch.tensor([0, n], dtype=torch.int32).cuda()
         cu_keep = torch.tensor([0, n_keep], dtype=torch.int32).cuda()
@@ -625,6 +634,10 @@ def run_other_workload(args):
         out.update({"rows": n, "kept": n_keep, "whole_op_ms": round(ms, 4),
                     "gather_rows": {"us": round(g_ms * 1e3, 2), "gbs": round(gbs, 1),
                                     "frac_of_hbm_peak": round(gbs / peaks["hbm_gbs"], 3)},
+                    "gather_rows_32768": {"us": round(gb_ms * 1e3, 2),
+                                          "gbs": round(2.0 * big_n * rb / (gb_ms * 1e-3) / 1e9, 1),
+                                          "frac_of_hbm_peak": round(2.0 * big_n * rb / (gb_ms * 1e-3) / 1e9
+                                                                    / peaks["hbm_gbs"], 3)},
                     "select": {"us": round(s_ms * 1e3, 2), "bytes": 8 * n},
                     "score_standalone": {"us": round(k_ms * 1e3, 2),
                                          "gbs": round(n * rb / (k_ms * 1e-3) / 1e9, 1)}})
